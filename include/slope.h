@@ -1,0 +1,152 @@
+/*
+ * slope.h -- C ABI of the B200 (sm_100a) SLoPe 2:4-sparse linear layer.
+ *
+ * The calls follow the thesis chapter "SLoPe: Double-Pruned Sparse Plus Lazy
+ * Low-Rank Adapter Pretraining of LLMs": Eq. (sparse_forward),
+ * Eq. (sparse_backward_weight), Eq. (sparse_backward_input), Eq. (concat),
+ * Algorithm 1 and the supplementary section "Implementation details".
+ *
+ * Common rules
+ *  - Every pointer is DEVICE memory owned by the caller unless a comment says
+ *    "host".  The library allocates no device memory.  Base pointers must be
+ *    16-byte aligned.  Matrices are dense, row-major, contiguous.
+ *  - bf16 = the upper 16 bits of an IEEE fp32.  GEMMs accumulate in fp32 and
+ *    round once (nearest-even) to bf16.
+ *  - `stream` is a cudaStream_t (NULL = the legacy default stream).  Calls are
+ *    asynchronous with respect to the host.
+ *  - Argument, shape, alignment and architecture errors are returned before
+ *    anything is launched.  d_out, d_in must be multiples of 128; tokens b a
+ *    multiple of 8 (b >= 8); adapter rank r in {0, 16, 32, ..., 128}.
+ *    There is no CPU fallback: on a device that is not sm_100 the calls return
+ *    SLOPE_ERR_UNSUPPORTED_ARCH.
+ *  - Device-side waits are bounded; a wait that runs out makes the kernel stop
+ *    and record SLOPE_ERR_TIMEOUT in a sticky status word, read (and cleared)
+ *    by slope_poll_status().
+ *  - Same inputs on the same device give bit-identical outputs.
+ *
+ * Compressed 2:4 format of a matrix A[rows x cols] pruned along its columns
+ *  - values  [rows x cols/2] bf16: for each group of 4 consecutive columns the
+ *    two kept entries, in ascending column order (bit copies of the source);
+ *  - metadata, rows*cols/8 bytes: one 4-bit code p0 | p1<<2 (p0 < p1 the kept
+ *    positions) per group, stored in the order the sparse tensor-core
+ *    instruction reads it.  The matrix is cut into 128x128 blocks, block
+ *    (rb, cb) at byte ((rb*(cols/128)) + cb) * 2048; inside a block the four
+ *    codes of row rr, columns [16*cs, 16*cs+16) form a 16-bit unit placed in
+ *    32-bit word (16*(rr/16) + 8*(cs%2) + rr%8)*4 + cs/2, low half if
+ *    (rr/8)%2 == 0, else high half;
+ *  - mask, [rows x cols/8] bytes: bit (j%8) of byte [i][j/8] is set when
+ *    element (i, j) was kept.  Masks are always in W's orientation.
+ */
+#ifndef SLOPE_H_
+#define SLOPE_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SLOPE_OK = 0,
+    SLOPE_ERR_INVALID_ARG = 1,      /* null pointer, bad enum value            */
+    SLOPE_ERR_SHAPE = 2,            /* dimension not supported                 */
+    SLOPE_ERR_ALIGNMENT = 3,        /* pointer not 16-byte aligned             */
+    SLOPE_ERR_UNSUPPORTED_ARCH = 4, /* current device is not sm_100            */
+    SLOPE_ERR_CUDA = 5,             /* a CUDA runtime / driver call failed     */
+    SLOPE_ERR_TIMEOUT = 6           /* a bounded device-side wait ran out      */
+} slope_status_t;
+
+/* Buffer sizes in bytes of the compressed format of a [rows x cols] matrix. */
+size_t slope_values_bytes(int rows, int cols);
+size_t slope_meta_bytes(int rows, int cols);
+size_t slope_mask_bytes(int rows, int cols);
+
+/*
+ * First pruning pass + compression (Algorithm 1, "backend.setup(W)"; the
+ * compression is described in the supplementary section on cuSPARSELt
+ * initialisation overhead).  For every row of W[d_out x d_in] and every group
+ * of 4 consecutive columns keep the two entries of largest magnitude (equal
+ * magnitudes: the lower column wins).  Writes the compressed W^R: values,
+ * metadata and (if mask1_bits != NULL) the element mask.
+ */
+slope_status_t slope_prune_24(const void* W, int d_out, int d_in,
+                              void* Wc_vals, void* Wc_meta, void* mask1_bits, void* stream);
+
+/*
+ * Second pruning pass (Section "Double-pruned Backward Pass"): transpose the
+ * already pruned W^R = W (.) mask1 and impose 2:4 again, now along d_out.
+ * Entries removed by the first pass take part with magnitude 0 and value +0.
+ * Writes the compressed TRANSPOSED matrix (W^{R,C})^T [d_in x d_out]: values
+ * [d_in x d_out/2], metadata, and (if mask2_bits != NULL) the mask of
+ * W^{R,C} in W's orientation [d_out x d_in/8] (a subset of mask1).
+ */
+slope_status_t slope_double_prune(const void* W, const void* mask1_bits, int d_out, int d_in,
+                                  void* WTc_vals, void* WTc_meta, void* mask2_bits, void* stream);
+
+/*
+ * Forward, Eq. (sparse_forward), optionally with the lazy adapter fused as in
+ * Eq. (concat):  Y[b x d_out] = X[b x d_in] (W^R)^T  (+ T[b x r] R[r x d_out]).
+ * Wc_vals / Wc_meta come from slope_prune_24.  T = X L is produced by
+ * slope_adapter_fwd_bwd(phase 0).  r = 0 (T, R ignored) leaves the adapter out.
+ */
+slope_status_t slope_linear_fwd(const void* X, int b, const void* Wc_vals, const void* Wc_meta,
+                                int d_out, int d_in, const void* T, const void* R, int r,
+                                void* Y, void* stream);
+
+/*
+ * Input gradient, Eq. (sparse_backward_input), with the double-pruned weight:
+ *   dX[b x d_in] = dY[b x d_out] W^{R,C}  (+ dT[b x r] L^T, L[d_in x r]).
+ * WTc_vals / WTc_meta come from slope_double_prune.  dT = dY R^T is produced by
+ * slope_adapter_fwd_bwd(phase 1).
+ */
+slope_status_t slope_linear_bwd_dx(const void* dY, int b, const void* WTc_vals, const void* WTc_meta,
+                                   int d_out, int d_in, const void* dT, const void* L, int r,
+                                   void* dX, void* stream);
+
+/*
+ * Weight gradient, Eq. (sparse_backward_weight), restricted to the first-pass
+ * mask and stored compressed (Algorithm 1 "pruneAndCompress"; output shape
+ * d_out x d_in/2 per "Implementation details"):
+ *   dWc[i][2g+t] = sum_n dY[n][i] X[n][4g + p_t(i,g)],  p_0 < p_1 kept by mask1.
+ */
+slope_status_t slope_linear_bwd_dw_masked(const void* dY, const void* X, int b, int d_out, int d_in,
+                                          const void* mask1_bits, void* dWc_vals, void* stream);
+
+/*
+ * Dense low-rank adapter GEMMs of Section "Lazy Low-rank Adapters" in the
+ * orientation of Eq. (concat): L[d_in x r], R[r x d_out].
+ *   phase 0:  T[b x r]  = X L
+ *   phase 1:  dT[b x r] = dY R^T,  dL[d_in x r] = X^T dT,  dR[r x d_out] = T^T dY
+ *             (dT and T are the bf16 tensors written by this call / phase 0).
+ * `workspace` is device scratch of at least slope_adapter_workspace_bytes()
+ * bytes, used by phase 1 for fixed-order split-K partial sums; unused pointers
+ * of the other phase may be NULL.
+ */
+size_t slope_adapter_workspace_bytes(int b, int d_out, int d_in, int r);
+slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY,
+                                     const void* L, const void* R,
+                                     int b, int d_out, int d_in, int r,
+                                     void* T, void* dT, void* dL, void* dR,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Diagnostic: rewrite tensor-core-order metadata as canonical metadata
+ * (uint16 [rows x cols/16], group g of a row at bits 4*(g%4) of unit g/4).
+ * Paper counterpart: none (the index storage of Eq. (index_bits) in a
+ * readable order).
+ */
+slope_status_t slope_meta_to_canonical(const void* meta_hw, int rows, int cols,
+                                       void* meta_canon, void* stream);
+
+/* Synchronises `stream`, returns and clears the sticky device status. */
+slope_status_t slope_poll_status(void* stream);
+
+/* Number of kernel launches issued by this library since load (host counter). */
+unsigned long long slope_launch_count(void);
+
+const char* slope_status_string(slope_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLOPE_H_ */

@@ -1,0 +1,448 @@
+// tcgen05 GEMM kernels for sm_100a.
+//
+// Both kernels are persistent and warp-specialised: warp 0 feeds shared memory with TMA,
+// warp 1 owns tensor memory and issues the MMAs (one elected thread), warps 2..5 drain the
+// fp32 accumulators from tensor memory, convert to bf16 and store.  Two accumulator stages
+// in tensor memory let the epilogue of tile t overlap the main loop of tile t+1.  Every
+// mbarrier wait is bounded (ptx.cuh); a role that gives up sets a CTA-wide flag, all roles
+// leave their loops, tensor memory is released and the kernel returns.
+#pragma once
+#include "ptx.cuh"
+
+namespace slope {
+
+constexpr int kGemmThreads = 192;
+constexpr int kBlockM = 128;
+
+struct PipeState {
+    int stage = 0;
+    uint32_t phase = 0;
+    __device__ __forceinline__ void advance(int nstages) {
+        if (++stage == nstages) { stage = 0; phase ^= 1u; }
+    }
+};
+
+// Give in-flight bulk copies time to land before the CTA's shared memory goes away.
+__device__ __forceinline__ void drain_after_abort() {
+    const unsigned long long t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+}
+
+// =====================================================================================
+// Sparse GEMM:  O[Ntok x M] (bf16) = ( A_2:4[M x K] * B[Ntok x K]^T  (+ A2[M x r] * B2[Ntok x r]^T) )^T
+//   A   compressed values [M x K/2] + tensor-core-order metadata   (sparse operand)
+//   B   activations, K contiguous
+//   A2  dense adapter factor on the weight side: either [M x r] (K contiguous) or [r x M]
+//   B2  dense adapter activations [Ntok x r]
+// Used for Eq. (sparse_forward) (M = d_out, K = d_in) and Eq. (sparse_backward_input)
+// (M = d_in, K = d_out, A = double-pruned transposed copy); the adapter product of
+// Eq. (concat) is accumulated into the same tensor-memory tile by extra dense MMAs.
+// Only the A operand of tcgen05.mma.sp can be sparse, hence the accumulator holds the
+// transposed output tile (lane = feature, column = token) and the epilogue transposes.
+// =====================================================================================
+struct SparseGemmParams {
+    int M, K, Ntok, r;
+    int a2_mn_major;              // 1: A2 is stored [r x M] (M contiguous)
+    const uint8_t* meta;          // metadata blocks of A
+    uint16_t* out;                // [Ntok x M]
+};
+
+template <int BLOCK_N, int STAGES>
+struct SparseCfg {
+    static constexpr int kABytes = kBlockM * 128;                // 128 rows x 64 compressed bf16
+    static constexpr int kBBytes = BLOCK_N * 256;                // BLOCK_N rows x 128 bf16 (two 64-wide boxes)
+    static constexpr int kEBytes = 2048;
+    static constexpr int kStageBytes = kABytes + kBBytes + kEBytes;
+    static constexpr int kBarBytes = 256;
+    static constexpr int kSmemBytes = STAGES * kStageBytes + kBarBytes + 1024;   // + alignment slack
+    static constexpr int kECol = 2 * BLOCK_N;                    // metadata columns after both accumulators
+    static_assert(BLOCK_N % 16 == 0 && BLOCK_N >= 16 && 2 * BLOCK_N + 8 <= 512, "tile does not fit tensor memory");
+    static_assert(kStageBytes % 1024 == 0, "stage must keep 1024-byte alignment for the 128-byte swizzle");
+};
+
+template <int BLOCK_N, int STAGES>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                   const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
+                   const SparseGemmParams p) {
+    using Cfg = SparseCfg<BLOCK_N, STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * Cfg::kStageBytes);
+    uint64_t* empty_bar = full_bar + STAGES;
+    uint64_t* tfull_bar = empty_bar + STAGES;
+    uint64_t* tempty_bar = tfull_bar + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_m = p.M / kBlockM;
+    const int num_n = (p.Ntok + BLOCK_N - 1) / BLOCK_N;
+    const int num_tiles = num_m * num_n;
+    const int num_kb = p.K / 128;
+    const int num_ab = (p.r + 63) / 64;
+    const int total_kb = num_kb + num_ab;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], 128); }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (elect_one()) {
+            tma_prefetch_desc(&tmA);
+            tma_prefetch_desc(&tmB);
+            PipeState ps;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                const int m_blk = tile % num_m, n_blk = tile / num_m;
+                for (int kb = 0; kb < total_kb; ++kb) {
+                    if (!mbar_wait(&empty_bar[ps.stage], ps.phase ^ 1u, abort_flag)) { ok = false; break; }
+                    uint8_t* sA = smem + ps.stage * Cfg::kStageBytes;
+                    uint8_t* sB = sA + Cfg::kABytes;
+                    uint8_t* sE = sB + Cfg::kBBytes;
+                    uint64_t* bar = &full_bar[ps.stage];
+                    if (kb < num_kb) {
+                        mbar_expect_tx(bar, Cfg::kABytes + Cfg::kBBytes + Cfg::kEBytes);
+                        tma_load_2d(sA, &tmA, bar, kb * 64, m_blk * kBlockM);
+                        tma_load_2d(sB, &tmB, bar, kb * 128, n_blk * BLOCK_N);
+                        tma_load_2d(sB + BLOCK_N * 128, &tmB, bar, kb * 128 + 64, n_blk * BLOCK_N);
+                        bulk_load_1d(sE, p.meta + (static_cast<size_t>(m_blk) * num_kb + kb) * 2048, 2048, bar);
+                    } else {
+                        const int ab = kb - num_kb;
+                        mbar_expect_tx(bar, Cfg::kABytes + BLOCK_N * 128);
+                        if (p.a2_mn_major) {
+                            tma_load_2d(sA, &tmA2, bar, m_blk * kBlockM, ab * 64);
+                            tma_load_2d(sA + 8192, &tmA2, bar, m_blk * kBlockM + 64, ab * 64);
+                        } else {
+                            tma_load_2d(sA, &tmA2, bar, ab * 64, m_blk * kBlockM);
+                        }
+                        tma_load_2d(sB, &tmB2, bar, ab * 64, n_blk * BLOCK_N);
+                    }
+                    ps.advance(STAGES);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (elect_one()) {
+            constexpr uint32_t idesc_sp = make_idesc_bf16(kBlockM, BLOCK_N, false, false, true);
+            const uint32_t idesc_ad = make_idesc_bf16(kBlockM, BLOCK_N, p.a2_mn_major != 0, false, false);
+            PipeState ps;
+            bool ok = true;
+            int it = 0;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
+                const int acc = it & 1;
+                const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
+                if (!mbar_wait(&tempty_bar[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * BLOCK_N;
+                for (int kb = 0; kb < total_kb; ++kb) {
+                    if (!mbar_wait(&full_bar[ps.stage], ps.phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t sA = smem_u32(smem + ps.stage * Cfg::kStageBytes);
+                    const uint32_t sB = sA + Cfg::kABytes;
+                    const uint32_t sE = sB + Cfg::kBBytes;
+                    if (kb < num_kb) {
+                        const uint32_t e_tmem = tmem_base + Cfg::kECol + (kb & 1) * 4;
+                        tmem_cp_128x128b(e_tmem, make_smem_desc(sE, 128, 128, kSwizzleNone));
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint64_t ad = make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
+                            const uint64_t bd =
+                                make_smem_desc(sB + (j >> 1) * (BLOCK_N * 128) + (j & 1) * 64, 16, 1024, kSwizzle128B);
+                            umma_bf16_sp(d_tmem, ad, bd, e_tmem + (j & 2), idesc_sp | (j & 1), (kb | j) != 0 ? 1u : 0u);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint64_t ad = p.a2_mn_major
+                                                    ? make_smem_desc(sA + j * 2048, 8192, 1024, kSwizzle128B)
+                                                    : make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
+                            const uint64_t bd = make_smem_desc(sB + j * 32, 16, 1024, kSwizzle128B);
+                            umma_bf16(d_tmem, ad, bd, idesc_ad, 1u);
+                        }
+                    }
+                    umma_commit(&empty_bar[ps.stage]);
+                    ps.advance(STAGES);
+                }
+                if (ok) umma_commit(&tfull_bar[acc]);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int q = warp & 3;                       // tensor-memory lane quadrant of this warp
+        bool ok = true;
+        int it = 0;
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
+            const int m_blk = tile % num_m, n_blk = tile / num_m;
+            const int acc = it & 1;
+            const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
+            if (!mbar_wait(&tfull_bar[acc], acc_phase, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t t_row = tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
+            const int m = m_blk * kBlockM + q * 32 + lane;
+            uint16_t* out_col = p.out + m;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BLOCK_N; c0 += 16) {
+                uint32_t v[16];
+                tmem_ld_16(t_row + c0, v);
+                tmem_ld_wait();
+                const int n0 = n_blk * BLOCK_N + c0;
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const int n = n0 + c;
+                    if (n < p.Ntok) out_col[static_cast<size_t>(n) * p.M] = to_bf16(__uint_as_float(v[c]));
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&tempty_bar[acc]);
+        }
+    }
+
+    __syncwarp();
+    if (*abort_flag) drain_after_abort();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// =====================================================================================
+// Dense GEMM:  D[M x N] = A[M x K] * B[N x K]^T, bf16 in, fp32 accumulate.
+//   A_MN / B_MN: the operand is stored with its M (resp. N) index contiguous, i.e. as
+//   [K x M] (resp. [K x N]) row-major; otherwise K is contiguous.
+// Epilogues:
+//   kEpiStore    bf16 D, row-major, leading dimension N
+//   kEpiMasked   Eq. (sparse_backward_weight) + Algorithm 1 "pruneAndCompress": keep, per
+//                group of 4 columns, the two columns the first-pass mask selects; bf16
+//                [M x N/2]
+//   kEpiPartial  fp32 partial sums of one K-split into workspace[split][M][N]
+// =====================================================================================
+constexpr int kEpiStore = 0, kEpiMasked = 1, kEpiPartial = 2;
+
+struct DenseGemmParams {
+    int M, N, K;
+    int k_splits;
+    void* out;
+    const uint8_t* mask;          // kEpiMasked: [M x N/8]
+};
+
+template <int BLOCK_N, int STAGES>
+struct DenseCfg {
+    static constexpr int kABytes = kBlockM * 128;                // 128 x 64 bf16
+    static constexpr int kBBytes = BLOCK_N * 128;                // BLOCK_N x 64 bf16
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kSmemBytes = STAGES * kStageBytes + 256 + 1024;
+    static constexpr int kTmemCols = 2 * BLOCK_N <= 32 ? 32 : (2 * BLOCK_N <= 64 ? 64 : (2 * BLOCK_N <= 128 ? 128 : (2 * BLOCK_N <= 256 ? 256 : 512)));
+    static_assert(BLOCK_N % 64 == 0 && BLOCK_N <= 256, "BLOCK_N must be 64, 128, 192 or 256");
+};
+
+template <bool A_MN, bool B_MN, int BLOCK_N, int EPI, int STAGES>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const DenseGemmParams p) {
+    using Cfg = DenseCfg<BLOCK_N, STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * Cfg::kStageBytes);
+    uint64_t* empty_bar = full_bar + STAGES;
+    uint64_t* tfull_bar = empty_bar + STAGES;
+    uint64_t* tempty_bar = tfull_bar + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_m = (p.M + kBlockM - 1) / kBlockM;
+    const int num_n = (p.N + BLOCK_N - 1) / BLOCK_N;
+    const int num_kb_total = (p.K + 63) / 64;
+    const int kb_per_split = (num_kb_total + p.k_splits - 1) / p.k_splits;
+    const int num_tiles = num_m * num_n * p.k_splits;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], 128); }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, Cfg::kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // tile -> (m block, n block, split): m fastest so that concurrently running CTAs share B
+    auto decode = [&](int tile, int& m_blk, int& n_blk, int& kb0, int& kb1) {
+        m_blk = tile % num_m;
+        const int rest = tile / num_m;
+        n_blk = rest % num_n;
+        const int split = rest / num_n;
+        kb0 = split * kb_per_split;
+        kb1 = min(num_kb_total, kb0 + kb_per_split);
+        return split;
+    };
+
+    if (warp == 0) {
+        if (elect_one()) {
+            tma_prefetch_desc(&tmA);
+            tma_prefetch_desc(&tmB);
+            PipeState ps;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                int m_blk, n_blk, kb0, kb1;
+                decode(tile, m_blk, n_blk, kb0, kb1);
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    if (!mbar_wait(&empty_bar[ps.stage], ps.phase ^ 1u, abort_flag)) { ok = false; break; }
+                    uint8_t* sA = smem + ps.stage * Cfg::kStageBytes;
+                    uint8_t* sB = sA + Cfg::kABytes;
+                    uint64_t* bar = &full_bar[ps.stage];
+                    mbar_expect_tx(bar, Cfg::kStageBytes);
+                    if (A_MN) {
+                        tma_load_2d(sA, &tmA, bar, m_blk * kBlockM, kb * 64);
+                        tma_load_2d(sA + 8192, &tmA, bar, m_blk * kBlockM + 64, kb * 64);
+                    } else {
+                        tma_load_2d(sA, &tmA, bar, kb * 64, m_blk * kBlockM);
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int h = 0; h < BLOCK_N / 64; ++h)
+                            tma_load_2d(sB + h * 8192, &tmB, bar, n_blk * BLOCK_N + h * 64, kb * 64);
+                    } else {
+                        tma_load_2d(sB, &tmB, bar, kb * 64, n_blk * BLOCK_N);
+                    }
+                    ps.advance(STAGES);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (elect_one()) {
+            constexpr uint32_t idesc = make_idesc_bf16(kBlockM, BLOCK_N, A_MN, B_MN, false);
+            PipeState ps;
+            bool ok = true;
+            int it = 0;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
+                int m_blk, n_blk, kb0, kb1;
+                decode(tile, m_blk, n_blk, kb0, kb1);
+                const int acc = it & 1;
+                const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
+                if (!mbar_wait(&tempty_bar[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * BLOCK_N;
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    if (!mbar_wait(&full_bar[ps.stage], ps.phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t sA = smem_u32(smem + ps.stage * Cfg::kStageBytes);
+                    const uint32_t sB = sA + Cfg::kABytes;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint64_t ad = A_MN ? make_smem_desc(sA + j * 2048, 8192, 1024, kSwizzle128B)
+                                                 : make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
+                        const uint64_t bd = B_MN ? make_smem_desc(sB + j * 2048, 8192, 1024, kSwizzle128B)
+                                                 : make_smem_desc(sB + j * 32, 16, 1024, kSwizzle128B);
+                        umma_bf16(d_tmem, ad, bd, idesc, (kb > kb0 || j > 0) ? 1u : 0u);
+                    }
+                    umma_commit(&empty_bar[ps.stage]);
+                    ps.advance(STAGES);
+                }
+                if (ok) umma_commit(&tfull_bar[acc]);
+            }
+        }
+    } else {
+        const int q = warp & 3;
+        bool ok = true;
+        int it = 0;
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
+            int m_blk, n_blk, kb0, kb1;
+            const int split = decode(tile, m_blk, n_blk, kb0, kb1);
+            const int acc = it & 1;
+            const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
+            if (!mbar_wait(&tfull_bar[acc], acc_phase, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t t_row = tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
+            const int m = m_blk * kBlockM + q * 32 + lane;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BLOCK_N; c0 += 16) {
+                uint32_t v[16];
+                tmem_ld_16(t_row + c0, v);
+                tmem_ld_wait();
+                const int n0 = n_blk * BLOCK_N + c0;
+                if (m >= p.M || n0 >= p.N) continue;
+                if (EPI == kEpiStore) {
+                    uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + static_cast<size_t>(m) * p.N + n0);
+                    uint32_t w[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) w[c] = pack_bf16x2(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1]));
+                    dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                    dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                } else if (EPI == kEpiMasked) {
+                    const uint32_t mbits =
+                        *reinterpret_cast<const uint16_t*>(p.mask + static_cast<size_t>(m) * (p.N >> 3) + (n0 >> 3));
+                    uint32_t w[4];
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        const uint32_t mb = (mbits >> (4 * g)) & 0xFu;
+                        // kept positions in ascending order: lowest set bit, highest set bit
+                        const int p0 = __ffs(mb) - 1, p1 = 31 - __clz(mb);
+                        const float e0 = __uint_as_float(v[4 * g]), e1 = __uint_as_float(v[4 * g + 1]),
+                                    e2 = __uint_as_float(v[4 * g + 2]), e3 = __uint_as_float(v[4 * g + 3]);
+                        const float lo = p0 == 0 ? e0 : (p0 == 1 ? e1 : e2);
+                        const float hi = p1 == 1 ? e1 : (p1 == 2 ? e2 : e3);
+                        w[g] = pack_bf16x2(lo, hi);
+                    }
+                    *reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + static_cast<size_t>(m) * (p.N >> 1) + (n0 >> 1)) =
+                        make_uint4(w[0], w[1], w[2], w[3]);
+                } else {
+                    float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.out) +
+                                                            (static_cast<size_t>(split) * p.M + m) * p.N + n0);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        dst[c] = make_float4(__uint_as_float(v[4 * c]), __uint_as_float(v[4 * c + 1]),
+                                             __uint_as_float(v[4 * c + 2]), __uint_as_float(v[4 * c + 3]));
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&tempty_bar[acc]);
+        }
+    }
+
+    __syncwarp();
+    if (*abort_flag) drain_after_abort();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    }
+}
+
+// Fixed-order reduction of K-split partial sums: out = bf16( sum_s ws[s][m][n] ), written
+// row-major [M x N] or transposed [N x M].
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float* __restrict__ ws, int M, int N, int splits, int transpose, uint16_t* __restrict__ out) {
+    const size_t total = static_cast<size_t>(M) * N;
+    for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
+         idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        float acc = 0.0f;
+        for (int s = 0; s < splits; ++s) acc += ws[static_cast<size_t>(s) * total + idx];
+        const size_t m = idx / N, n = idx % N;
+        out[transpose ? n * static_cast<size_t>(M) + m : idx] = to_bf16(acc);
+    }
+}
+
+}  // namespace slope

@@ -1,0 +1,336 @@
+// C ABI of the SLoPe 2:4-sparse linear layer for B200 (sm_100a): argument checks,
+// TMA descriptor construction and kernel launches.  No device memory is allocated here.
+#include "../../include/slope.h"
+
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+#include "gemm_kernels.cuh"
+#include "prune_kernels.cuh"
+
+namespace slope {
+
+static std::atomic<unsigned long long> g_launches{0};
+
+// ------------------------------------------------------------------ device / driver set-up
+struct DeviceInfo {
+    bool ok = false;
+    int sm_count = 0;
+    int cc_major = 0;
+};
+
+static DeviceInfo device_info() {
+    static std::mutex mu;
+    static DeviceInfo cache[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DeviceInfo{};
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cache[dev].ok) {
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return DeviceInfo{};
+        cache[dev].sm_count = prop.multiProcessorCount;
+        cache[dev].cc_major = prop.major;
+        cache[dev].ok = true;
+    }
+    return cache[dev];
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    });
+    return fn;
+}
+
+// 2-D bf16 tensor map over a row-major [rows x cols] matrix, 128-byte swizzle,
+// box = box_cols (<= 64) x box_rows, out-of-bounds elements read as zero.
+static bool make_tmap(CUtensorMap* tm, const void* base, int rows, int cols, int box_rows, int box_cols) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(cols) * 2};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static slope_status_t check_arch(DeviceInfo& info) {
+    info = device_info();
+    if (!info.ok) return SLOPE_ERR_CUDA;
+    if (info.cc_major != 10) return SLOPE_ERR_UNSUPPORTED_ARCH;
+    return SLOPE_OK;
+}
+
+static slope_status_t launch_result() {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? SLOPE_OK : SLOPE_ERR_CUDA;
+}
+
+template <typename Kernel>
+static bool set_smem(Kernel k, int bytes) {
+    return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+
+// ------------------------------------------------------------------ sparse GEMM launch
+constexpr int kSpBlockN = 240;
+constexpr int kSpStages = 2;
+
+static slope_status_t launch_sparse(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
+                                    const void* act2, const void* fac2, int r, bool a2_mn, void* out,
+                                    cudaStream_t stream, const DeviceInfo& info) {
+    using Cfg = SparseCfg<kSpBlockN, kSpStages>;
+    CUtensorMap tmA, tmB, tmA2, tmB2;
+    if (!make_tmap(&tmA, vals, M, K / 2, kBlockM, 64)) return SLOPE_ERR_CUDA;
+    if (!make_tmap(&tmB, act, ntok, K, kSpBlockN, 64)) return SLOPE_ERR_CUDA;
+    if (r > 0) {
+        const bool ok2 = a2_mn ? make_tmap(&tmA2, fac2, r, M, 64, 64) : make_tmap(&tmA2, fac2, M, r, kBlockM, 64);
+        if (!ok2 || !make_tmap(&tmB2, act2, ntok, r, kSpBlockN, 64)) return SLOPE_ERR_CUDA;
+    } else {
+        tmA2 = tmA;
+        tmB2 = tmB;
+    }
+    SparseGemmParams p;
+    p.M = M; p.K = K; p.Ntok = ntok; p.r = r; p.a2_mn_major = a2_mn ? 1 : 0;
+    p.meta = static_cast<const uint8_t*>(meta);
+    p.out = static_cast<uint16_t*>(out);
+    auto kern = sparse_gemm_kernel<kSpBlockN, kSpStages>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
+        attr_set = true;
+    }
+    const int tiles = (M / kBlockM) * ((ntok + kSpBlockN - 1) / kSpBlockN);
+    const int grid = tiles < info.sm_count ? tiles : info.sm_count;
+    kern<<<grid, kGemmThreads, Cfg::kSmemBytes, stream>>>(tmA, tmB, tmA2, tmB2, p);
+    return launch_result();
+}
+
+// ------------------------------------------------------------------ dense GEMM launch
+template <bool A_MN, bool B_MN, int BLOCK_N, int EPI, int STAGES>
+static slope_status_t launch_dense(const void* A, const void* B, int M, int N, int K, int k_splits, void* out,
+                                   const void* mask, cudaStream_t stream, const DeviceInfo& info) {
+    using Cfg = DenseCfg<BLOCK_N, STAGES>;
+    CUtensorMap tmA, tmB;
+    const bool okA = A_MN ? make_tmap(&tmA, A, K, M, 64, 64) : make_tmap(&tmA, A, M, K, kBlockM, 64);
+    const bool okB = B_MN ? make_tmap(&tmB, B, K, N, 64, 64) : make_tmap(&tmB, B, N, K, BLOCK_N, 64);
+    if (!okA || !okB) return SLOPE_ERR_CUDA;
+    DenseGemmParams p;
+    p.M = M; p.N = N; p.K = K; p.k_splits = k_splits; p.out = out;
+    p.mask = static_cast<const uint8_t*>(mask);
+    auto kern = dense_gemm_kernel<A_MN, B_MN, BLOCK_N, EPI, STAGES>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
+        attr_set = true;
+    }
+    const int tiles = ((M + kBlockM - 1) / kBlockM) * ((N + BLOCK_N - 1) / BLOCK_N) * k_splits;
+    const int grid = tiles < info.sm_count ? tiles : info.sm_count;
+    kern<<<grid, kGemmThreads, Cfg::kSmemBytes, stream>>>(tmA, tmB, p);
+    return launch_result();
+}
+
+static int adapter_splits(int b, int rows) {
+    // enough K-splits that (row tiles x splits) covers the machine, each split >= 512 tokens
+    const int tiles = (rows + kBlockM - 1) / kBlockM;
+    int s = (148 + tiles - 1) / tiles;
+    const int max_s = b / 512 > 0 ? b / 512 : 1;
+    if (s > max_s) s = max_s;
+    if (s > 16) s = 16;
+    return s < 1 ? 1 : s;
+}
+
+static bool dims_ok(int d_out, int d_in) {
+    return d_out > 0 && d_in > 0 && d_out % 128 == 0 && d_in % 128 == 0;
+}
+static bool rank_ok(int r) { return r >= 0 && r <= 128 && r % 16 == 0; }
+
+}  // namespace slope
+
+using namespace slope;
+
+extern "C" {
+
+size_t slope_values_bytes(int rows, int cols) { return static_cast<size_t>(rows) * cols; }
+size_t slope_meta_bytes(int rows, int cols) { return static_cast<size_t>(rows) * cols / 8; }
+size_t slope_mask_bytes(int rows, int cols) { return static_cast<size_t>(rows) * cols / 8; }
+
+unsigned long long slope_launch_count(void) { return g_launches.load(); }
+
+const char* slope_status_string(slope_status_t s) {
+    switch (s) {
+        case SLOPE_OK: return "ok";
+        case SLOPE_ERR_INVALID_ARG: return "invalid argument";
+        case SLOPE_ERR_SHAPE: return "unsupported shape";
+        case SLOPE_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case SLOPE_ERR_UNSUPPORTED_ARCH: return "device is not sm_100";
+        case SLOPE_ERR_CUDA: return "CUDA call failed";
+        case SLOPE_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+slope_status_t slope_poll_status(void* stream) {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return SLOPE_ERR_CUDA;
+    int st = 0;
+    if (cudaMemcpyFromSymbol(&st, g_device_status, sizeof(int)) != cudaSuccess) return SLOPE_ERR_CUDA;
+    if (st != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return SLOPE_ERR_CUDA;
+    }
+    return static_cast<slope_status_t>(st);
+}
+
+slope_status_t slope_prune_24(const void* W, int d_out, int d_in, void* Wc_vals, void* Wc_meta, void* mask1_bits,
+                              void* stream) {
+    if (!W || !Wc_vals || !Wc_meta) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(d_out, d_in)) return SLOPE_ERR_SHAPE;
+    if (!aligned16(W) || !aligned16(Wc_vals) || !aligned16(Wc_meta) || !aligned16(mask1_bits)) return SLOPE_ERR_ALIGNMENT;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    dim3 grid(d_in / 128, d_out / 128);
+    prune24_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4*>(W), d_out, d_in, static_cast<uint2*>(Wc_vals), static_cast<uint4*>(Wc_meta),
+        static_cast<uint4*>(mask1_bits));
+    return launch_result();
+}
+
+slope_status_t slope_double_prune(const void* W, const void* mask1_bits, int d_out, int d_in, void* WTc_vals,
+                                  void* WTc_meta, void* mask2_bits, void* stream) {
+    if (!W || !mask1_bits || !WTc_vals || !WTc_meta) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(d_out, d_in)) return SLOPE_ERR_SHAPE;
+    if (!aligned16(W) || !aligned16(mask1_bits) || !aligned16(WTc_vals) || !aligned16(WTc_meta) ||
+        !aligned16(mask2_bits))
+        return SLOPE_ERR_ALIGNMENT;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (!set_smem(double_prune_kernel, kDpSmemBytes)) return SLOPE_ERR_CUDA;
+        attr_set = true;
+    }
+    dim3 grid(d_in / 128, d_out / 128);
+    double_prune_kernel<<<grid, 256, kDpSmemBytes, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4*>(W), static_cast<const uint8_t*>(mask1_bits), d_out, d_in,
+        static_cast<uint4*>(WTc_vals), static_cast<uint4*>(WTc_meta), static_cast<uint4*>(mask2_bits));
+    return launch_result();
+}
+
+slope_status_t slope_linear_fwd(const void* X, int b, const void* Wc_vals, const void* Wc_meta, int d_out, int d_in,
+                                const void* T, const void* R, int r, void* Y, void* stream) {
+    if (!X || !Wc_vals || !Wc_meta || !Y) return SLOPE_ERR_INVALID_ARG;
+    if (r != 0 && (!T || !R)) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(d_out, d_in) || b < 8 || b % 8 != 0 || !rank_ok(r)) return SLOPE_ERR_SHAPE;
+    if (!aligned16(X) || !aligned16(Wc_vals) || !aligned16(Wc_meta) || !aligned16(Y) ||
+        (r != 0 && (!aligned16(T) || !aligned16(R))))
+        return SLOPE_ERR_ALIGNMENT;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    return launch_sparse(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R, r, /*a2_mn=*/true, Y,
+                         static_cast<cudaStream_t>(stream), info);
+}
+
+slope_status_t slope_linear_bwd_dx(const void* dY, int b, const void* WTc_vals, const void* WTc_meta, int d_out,
+                                   int d_in, const void* dT, const void* L, int r, void* dX, void* stream) {
+    if (!dY || !WTc_vals || !WTc_meta || !dX) return SLOPE_ERR_INVALID_ARG;
+    if (r != 0 && (!dT || !L)) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(d_out, d_in) || b < 8 || b % 8 != 0 || !rank_ok(r)) return SLOPE_ERR_SHAPE;
+    if (!aligned16(dY) || !aligned16(WTc_vals) || !aligned16(WTc_meta) || !aligned16(dX) ||
+        (r != 0 && (!aligned16(dT) || !aligned16(L))))
+        return SLOPE_ERR_ALIGNMENT;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    return launch_sparse(dY, b, WTc_vals, WTc_meta, d_in, d_out, dT, L, r, /*a2_mn=*/false, dX,
+                         static_cast<cudaStream_t>(stream), info);
+}
+
+slope_status_t slope_linear_bwd_dw_masked(const void* dY, const void* X, int b, int d_out, int d_in,
+                                          const void* mask1_bits, void* dWc_vals, void* stream) {
+    if (!dY || !X || !mask1_bits || !dWc_vals) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(d_out, d_in) || b < 8 || b % 8 != 0) return SLOPE_ERR_SHAPE;
+    if (!aligned16(dY) || !aligned16(X) || !aligned16(mask1_bits) || !aligned16(dWc_vals)) return SLOPE_ERR_ALIGNMENT;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    return launch_dense<true, true, 256, kEpiMasked, 4>(dY, X, d_out, d_in, b, 1, dWc_vals, mask1_bits,
+                                                        static_cast<cudaStream_t>(stream), info);
+}
+
+size_t slope_adapter_workspace_bytes(int b, int d_out, int d_in, int r) {
+    if (b <= 0 || d_out <= 0 || d_in <= 0 || r <= 0) return 0;
+    const int bn = r <= 64 ? 64 : 128;
+    const size_t wl = static_cast<size_t>(adapter_splits(b, d_in)) * d_in * bn * sizeof(float);
+    const size_t wr = static_cast<size_t>(adapter_splits(b, d_out)) * d_out * bn * sizeof(float);
+    return wl > wr ? wl : wr;
+}
+
+slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY, const void* L, const void* R, int b,
+                                     int d_out, int d_in, int r, void* T, void* dT, void* dL, void* dR,
+                                     void* workspace, size_t workspace_bytes, void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (phase != 0 && phase != 1) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(d_out, d_in) || b < 8 || b % 8 != 0 || !rank_ok(r) || r == 0) return SLOPE_ERR_SHAPE;
+    DeviceInfo info;
+    if (phase == 0) {
+        if (!X || !L || !T) return SLOPE_ERR_INVALID_ARG;
+        if (!aligned16(X) || !aligned16(L) || !aligned16(T)) return SLOPE_ERR_ALIGNMENT;
+        if (slope_status_t st = check_arch(info)) return st;
+        // T[b x r] = X[b x d_in] * L[d_in x r]   (A = X, K contiguous; B = L^T stored [K x N])
+        return r <= 64 ? launch_dense<false, true, 64, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info)
+                       : launch_dense<false, true, 128, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info);
+    }
+    if (!X || !dY || !R || !T || !dT || !dL || !dR || !workspace) return SLOPE_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(dY) || !aligned16(R) || !aligned16(T) || !aligned16(dT) || !aligned16(dL) ||
+        !aligned16(dR) || !aligned16(workspace))
+        return SLOPE_ERR_ALIGNMENT;
+    if (workspace_bytes < slope_adapter_workspace_bytes(b, d_out, d_in, r)) return SLOPE_ERR_INVALID_ARG;
+    if (slope_status_t st = check_arch(info)) return st;
+    slope_status_t st;
+    // dT[b x r] = dY[b x d_out] * R[r x d_out]^T   (both K contiguous)
+    st = r <= 64 ? launch_dense<false, false, 64, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info)
+                 : launch_dense<false, false, 128, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info);
+    if (st) return st;
+    // dL[d_in x r] = X^T dT: A = X stored [K x M], B = dT stored [K x N]; K = tokens, split in fixed slices
+    const int sl = adapter_splits(b, d_in);
+    st = r <= 64 ? launch_dense<true, true, 64, kEpiPartial, 6>(X, dT, d_in, r, b, sl, workspace, nullptr, stream, info)
+                 : launch_dense<true, true, 128, kEpiPartial, 6>(X, dT, d_in, r, b, sl, workspace, nullptr, stream, info);
+    if (st) return st;
+    splitk_reduce_kernel<<<info.sm_count * 4, 256, 0, stream>>>(static_cast<const float*>(workspace), d_in, r, sl, 0,
+                                                               static_cast<uint16_t*>(dL));
+    if ((st = launch_result())) return st;
+    // dR^T[d_out x r] = dY^T T, reduced and written transposed into dR[r x d_out]
+    const int sr = adapter_splits(b, d_out);
+    st = r <= 64 ? launch_dense<true, true, 64, kEpiPartial, 6>(dY, T, d_out, r, b, sr, workspace, nullptr, stream, info)
+                 : launch_dense<true, true, 128, kEpiPartial, 6>(dY, T, d_out, r, b, sr, workspace, nullptr, stream, info);
+    if (st) return st;
+    splitk_reduce_kernel<<<info.sm_count * 4, 256, 0, stream>>>(static_cast<const float*>(workspace), d_out, r, sr, 1,
+                                                               static_cast<uint16_t*>(dR));
+    return launch_result();
+}
+
+slope_status_t slope_meta_to_canonical(const void* meta_hw, int rows, int cols, void* meta_canon, void* stream) {
+    if (!meta_hw || !meta_canon) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(rows, cols)) return SLOPE_ERR_SHAPE;
+    if (!aligned16(meta_hw) || !aligned16(meta_canon)) return SLOPE_ERR_ALIGNMENT;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    meta_to_canonical_kernel<<<info.sm_count * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint16_t*>(meta_hw), rows, cols, static_cast<uint16_t*>(meta_canon));
+    return launch_result();
+}
+
+}  // extern "C"

@@ -1,0 +1,62 @@
+"""CPU-only checks of the boundary: the library builds for sm_100a, loads, and exports every
+symbol ``include/slope.h`` declares; pure host logic (sizes, argument checks) behaves."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2608_24070_b200 import build, binding
+
+    build.build()
+    return binding.lib()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "slope.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(slope_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported(lib):
+    from paper_2608_24070_b200 import binding
+
+    names = declared_symbols()
+    assert len(names) >= 14
+    for name in names:
+        assert hasattr(lib, name), name
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_size_helpers(lib):
+    assert lib.slope_values_bytes(4096, 4096) == 4096 * 4096
+    assert lib.slope_meta_bytes(4096, 11008) == 4096 * 11008 // 8
+    assert lib.slope_mask_bytes(512, 512) == 512 * 512 // 8
+    assert lib.slope_adapter_workspace_bytes(16384, 4096, 4096, 64) > 0
+    assert lib.slope_adapter_workspace_bytes(16384, 4096, 4096, 0) == 0
+
+
+def test_host_side_argument_checks_need_no_gpu(lib):
+    null = None
+    assert lib.slope_prune_24(null, 128, 128, null, null, null, null) == 1            # invalid arg
+    buf = ctypes.create_string_buffer(64)
+    p = ctypes.cast(buf, ctypes.c_void_p)
+    assert lib.slope_prune_24(p, 100, 128, p, p, null, null) == 2                      # shape
+    assert lib.slope_linear_fwd(p, 12, p, p, 128, 128, null, null, 0, p, null) == 2    # tokens % 8
+    assert lib.slope_linear_fwd(p, 16, p, p, 128, 128, null, null, 24, p, null) == 1   # rank without factors
+    assert lib.slope_adapter_fwd_bwd(7, p, p, p, p, 16, 128, 128, 16, p, p, p, p, p, 0, null) == 1
+    assert lib.slope_status_string(6) == b"device-side wait timed out"
+
+
+def test_binding_refuses_to_run_without_the_library(monkeypatch, tmp_path):
+    from paper_2608_24070_b200 import binding
+
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "_LIB_PATH", tmp_path / "libslope.so")
+    with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
+        binding.lib()

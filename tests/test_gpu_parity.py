@@ -1,0 +1,171 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on the same
+seeded inputs.  Integer / byte outputs bit-exact; GEMM outputs within 5e-3 relative
+Frobenius error (bf16 in, fp32 accumulate, one rounding to bf16)."""
+import itertools
+
+import numpy as np
+import pytest
+
+from paper_2608_24070_b200 import inputs as si
+from helpers import REL_TOL, GpuLayer, check_selection, rel_fro, to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2608_24070_b200 import binding
+
+    binding.lib()
+    return binding
+
+
+def dev(B, bits):
+    return B.bf16_from_bits(bits)
+
+
+# ------------------------------------------------------------------ selection / compression
+@pytest.mark.parametrize("d_out,d_in,seed", [(512, 512, 1), (384, 640, 2), (128, 1152, 3), (1280, 128, 4)])
+def test_prune_and_double_prune_bit_exact(B, oracle, d_out, d_in, seed):
+    W = si.gaussian_bf16((d_out, d_in), 0.02, seed)
+    layer = GpuLayer(W)
+    check_selection(oracle, layer, W)
+
+
+def test_prune_ties_zeros_and_specials(B, oracle):
+    """All 4-tuples over {+0,-0,+-1,+-2} (ties everywhere), plus inf / nan / denormal patterns."""
+    alphabet = si.f32_to_bf16_bits(np.array([0.0, -0.0, 1.0, -1.0, 2.0, -2.0], np.float32))
+    groups = np.array(list(itertools.product(alphabet, repeat=4)), np.uint16).reshape(-1)
+    W = np.zeros((256, 256), np.uint16)
+    W.reshape(-1)[: groups.size] = groups
+    special = np.array([0x7F80, 0xFF80, 0x7FC0, 0x0001, 0x8001, 0x7F7F, 0x0080, 0xFFFF], np.uint16)
+    rng = np.random.Generator(np.random.PCG64(5))
+    W[128:, :] = rng.choice(special, size=(128, 256))
+    layer = GpuLayer(W)
+    check_selection(oracle, layer, W)
+
+
+# ------------------------------------------------------------------ exact special cases through the MMAs
+def _nibble_pattern_weight(d_out, d_in, seed):
+    """Integer-valued weights whose kept pair cycles through all six patterns."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    pats = [(0, 1), (0, 2), (0, 3), (1, 2), (1, 3), (2, 3)]
+    Wf = np.zeros((d_out, d_in), np.float32)
+    for i in range(d_out):
+        for g in range(d_in // 4):
+            p = pats[(i * 7 + g * 5 + (i // 128) + (g // 32)) % 6]
+            small = rng.integers(1, 4, size=4).astype(np.float32) * rng.choice([-1, 1], size=4)
+            big = rng.integers(8, 64, size=2).astype(np.float32) * rng.choice([-1, 1], size=2)
+            grp = small.copy()
+            grp[p[0]], grp[p[1]] = big[0], big[1]
+            Wf[i, 4 * g:4 * g + 4] = grp
+    return si.f32_to_bf16_bits(Wf)
+
+
+def test_identity_activations_return_the_pruned_weight_exactly(B, oracle):
+    """X = I  =>  Y = (W^R)^T bit for bit;  dY = I  =>  dX = W^{R,C};  dY = I  =>  dWc = gather(X)."""
+    import torch
+
+    d_out, d_in = 256, 384
+    W = _nibble_pattern_weight(d_out, d_in, 6)
+    layer = GpuLayer(W)
+    mask1, mask2 = check_selection(oracle, layer, W)
+    m1, m2 = oracle.mask_to_bool(mask1, d_in), oracle.mask_to_bool(mask2, d_in)
+    Wf = to_f64(W)
+
+    eye_in = torch.eye(d_in, dtype=torch.bfloat16, device="cuda")
+    Y = layer.fwd(eye_in)
+    layer.poll()
+    assert np.array_equal(to_f64(B.bits_from_bf16(Y)), np.where(m1, Wf, 0.0).T)
+
+    eye_out = torch.eye(d_out, dtype=torch.bfloat16, device="cuda")
+    dX = layer.dx(eye_out)
+    layer.poll()
+    assert np.array_equal(to_f64(B.bits_from_bf16(dX)), np.where(m2, Wf, 0.0))
+
+    Xb = si.gaussian_bf16((d_out, d_in), 1.0, 8)
+    dWc = layer.dw(eye_out, dev(B, Xb))
+    layer.poll()
+    assert np.array_equal(B.bits_from_bf16(dWc), Xb[m1].reshape(d_out, d_in // 2))
+
+
+# ------------------------------------------------------------------ GEMM parity, full outputs
+CASES = [
+    # d_in, d_out, tokens, rank, seed
+    (512, 512, 256, 0, 11),          # config 1
+    (512, 512, 256, 64, 12),
+    (384, 640, 776, 32, 13),         # ragged token tail, several tiles in every dimension
+    (768, 256, 1000, 128, 14),
+    (128, 128, 8, 16, 15),           # smallest legal problem
+]
+
+
+@pytest.mark.parametrize("d_in,d_out,b,r,seed", CASES)
+def test_layer_against_oracle(B, oracle, d_in, d_out, b, r, seed):
+    W = si.gaussian_bf16((d_out, d_in), 0.02, seed)
+    X = si.gaussian_bf16((b, d_in), 1.0, seed + 100)
+    dY = si.gaussian_bf16((b, d_out), 1.0, seed + 200)
+    L = si.gaussian_bf16((d_in, r), 0.01, seed + 300) if r else None
+    R = si.gaussian_bf16((r, d_out), 0.01, seed + 400) if r else None
+    layer = GpuLayer(W)
+    mask1, mask2 = check_selection(oracle, layer, W)
+    Xd, dYd = dev(B, X), dev(B, dY)
+    rows = np.arange(b)
+    if r:
+        Ld, Rd = dev(B, L), dev(B, R)
+        T = layer.adapter_T(Xd, Ld)
+        Y = layer.fwd(Xd, T, Rd)
+        dT, dL, dR = layer.adapter_bwd(Xd, dYd, Ld, Rd, T)
+        dX = layer.dx(dYd, dT, Ld)
+    else:
+        Y = layer.fwd(Xd)
+        dX = layer.dx(dYd)
+    dWc = layer.dw(dYd, Xd)
+    layer.poll()
+    g = lambda t: to_f64(B.bits_from_bf16(t))
+    errs = {
+        "Y": rel_fro(g(Y), oracle.fwd_rows(X, W, mask1, rows, L, R)),
+        "dX": rel_fro(g(dX), oracle.dx_rows(dY, W, mask2, rows, L, R)),
+        "dWc": rel_fro(g(dWc), oracle.dw_rows(dY, X, mask1, np.arange(d_out))),
+    }
+    if r:
+        errs["T"] = rel_fro(g(T), oracle.adapter_T_rows(X, L, rows))
+        errs["dT"] = rel_fro(g(dT), oracle.adapter_dT_rows(dY, R, rows))
+        errs["dL"] = rel_fro(g(dL), oracle.adapter_dL_rows(X, dY, R, np.arange(d_in)))
+        errs["dR"] = rel_fro(g(dR), oracle.adapter_dR_cols(X, L, dY, np.arange(d_out)))
+    print(errs)
+    for k, v in errs.items():
+        assert v <= REL_TOL, (k, v, errs)
+
+
+def test_no_adapter_path_is_bitwise_the_rank0_path_and_deterministic(B, oracle):
+    W = si.gaussian_bf16((256, 256), 0.02, 31)
+    X = si.gaussian_bf16((512, 256), 1.0, 32)
+    layer = GpuLayer(W)
+    Xd = dev(B, X)
+    a = B.bits_from_bf16(layer.fwd(Xd))
+    b = B.bits_from_bf16(layer.fwd(Xd))
+    layer.poll()
+    assert np.array_equal(a, b)
+
+
+def test_argument_errors_are_reported_before_launch(B):
+    import torch
+
+    W = torch.zeros((100, 128), dtype=torch.bfloat16, device="cuda")
+    vals = torch.zeros((100, 64), dtype=torch.bfloat16, device="cuda")
+    meta = torch.zeros(100 * 16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.SlopeError) as e:
+        B.slope_prune_24(W, vals, meta)
+    assert e.value.status == 2
+    W = torch.zeros((128, 128), dtype=torch.bfloat16, device="cuda")
+    vals = torch.zeros((128, 64 + 4), dtype=torch.bfloat16, device="cuda").view(-1)[1:1 + 128 * 64]
+    with pytest.raises(B.SlopeError) as e:
+        B.slope_prune_24(W, vals, torch.zeros(2048, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 3
+    assert B.lib().slope_prune_24(None, 128, 128, None, None, None, None) == 1
+    assert B.slope_poll_status() == 0
