@@ -1,0 +1,499 @@
+#!/usr/bin/env python
+"""Benchmark of the SLoPe 2:4-sparse linear-layer path on B200.
+
+A step = one pass of the whole hot path over one batch of synthetic input, for every
+linear layer of the workload: first-pass prune + compress, double prune, [adapter T = X L],
+forward, [adapter backward], input gradient, masked weight gradient -- every stage a
+hand-written kernel behind the C ABI.  Prints ONE JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload KEY] [--impl reference]
+
+N > 1 (under torchrun) runs N independent replicas (the path has no exchange step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2608_24070_b200 import inputs as si  # noqa: E402
+
+METRIC = "SLoPe linear fwd+bwd TFLOP/s (dense-equivalent)"
+UNIT = "TFLOP/s"
+DEFAULT_WORKLOAD = "c4_llama7b_adapter"
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16": p["bf16_tflops"], "bf16_sustained": p["bf16_tflops_sustained"],
+                "src": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16": 1590.0, "bf16_sustained": 1400.0, "src": "fallback"}
+
+
+# ------------------------------------------------------------------------------ flop accounting
+def layer_flops(b, d_in, d_out, r):
+    """Dense-equivalent and executed FLOPs of one layer's fwd + dX + dW (+ adapter GEMMs)."""
+    main = 2.0 * b * d_in * d_out
+    adapter = 6.0 * b * r * (d_in + d_out)         # T, +T R, dT, dL, dR, +dT L^T
+    return 3 * main + adapter, 2 * main + adapter
+
+
+def workload_flops(wl, b):
+    de = ex = 0.0
+    for lay in wl.layers:
+        a, c = layer_flops(b, lay.d_in, lay.d_out, wl.rank)
+        de += a
+        ex += c
+    return de, ex
+
+
+# ------------------------------------------------------------------------------ clocks sampler
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for row in self.rows:
+            f = [x.strip() for x in row.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        # "under load": samples in the upper half of the observed power range
+        if power:
+            thr = 0.5 * (max(power) + min(power))
+            load = [s for s, p in zip(sm, power) if p >= thr] or sm
+        else:
+            load = sm
+        return {"sm_mhz": statistics.median(load) if load else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------ the CUDA arm
+class LayerState:
+    def __init__(self, B, torch, wl, idx, b, dev):
+        lay = wl.layers[idx]
+        self.name, self.d_in, self.d_out, self.r, self.b = lay.name, lay.d_in, lay.d_out, wl.rank, b
+        t = si.layer_tensors(wl, idx, tokens=b)
+        self.W = B.bf16_from_bits(t["W"], dev)
+        self.X = B.bf16_from_bits(t["X"], dev)
+        self.dY = B.bf16_from_bits(t["dY"], dev)
+        self.L = B.bf16_from_bits(t["L"], dev) if self.r else None
+        self.R = B.bf16_from_bits(t["R"], dev) if self.r else None
+        self.Wc_vals, self.Wc_meta, self.mask1 = B.alloc_compressed(self.d_out, self.d_in, dev)
+        self.WTc_vals, self.WTc_meta, _ = B.alloc_compressed(self.d_in, self.d_out, dev)
+        self.mask2 = torch.empty_like(self.mask1)
+        bf = torch.bfloat16
+        self.Y = torch.empty((b, self.d_out), dtype=bf, device=dev)
+        self.dX = torch.empty((b, self.d_in), dtype=bf, device=dev)
+        self.dWc = torch.empty((self.d_out, self.d_in // 2), dtype=bf, device=dev)
+        if self.r:
+            self.T = torch.empty((b, self.r), dtype=bf, device=dev)
+            self.dT = torch.empty((b, self.r), dtype=bf, device=dev)
+            self.dL = torch.empty((self.d_in, self.r), dtype=bf, device=dev)
+            self.dR = torch.empty((self.r, self.d_out), dtype=bf, device=dev)
+            self.ws = torch.empty(B.slope_adapter_workspace_bytes(b, self.d_out, self.d_in, self.r),
+                                  dtype=torch.uint8, device=dev)
+
+
+OPS = ("prune_24", "double_prune", "adapter_T", "linear_fwd", "adapter_bwd", "linear_bwd_dx", "linear_bwd_dw_masked")
+
+
+def run_layer(B, s: LayerState, rec=None):
+    """All stages of one layer; `rec(op)` brackets a stage with CUDA events when timing per stage."""
+    def stage(op, fn):
+        if rec is None:
+            fn()
+        else:
+            rec(op, s, fn)
+
+    stage("prune_24", lambda: B.slope_prune_24(s.W, s.Wc_vals, s.Wc_meta, s.mask1))
+    stage("double_prune", lambda: B.slope_double_prune(s.W, s.mask1, s.WTc_vals, s.WTc_meta, s.mask2))
+    if s.r:
+        stage("adapter_T", lambda: B.slope_adapter_fwd_bwd(0, s.X, None, s.L, None, s.b, s.d_out, s.d_in, s.r, T=s.T))
+        stage("linear_fwd", lambda: B.slope_linear_fwd(s.X, s.Wc_vals, s.Wc_meta, s.d_out, s.Y, s.T, s.R))
+        stage("adapter_bwd", lambda: B.slope_adapter_fwd_bwd(1, s.X, s.dY, s.L, s.R, s.b, s.d_out, s.d_in, s.r,
+                                                             T=s.T, dT=s.dT, dL=s.dL, dR=s.dR, workspace=s.ws))
+        stage("linear_bwd_dx", lambda: B.slope_linear_bwd_dx(s.dY, s.WTc_vals, s.WTc_meta, s.d_in, s.dX, s.dT, s.L))
+    else:
+        stage("linear_fwd", lambda: B.slope_linear_fwd(s.X, s.Wc_vals, s.Wc_meta, s.d_out, s.Y))
+        stage("linear_bwd_dx", lambda: B.slope_linear_bwd_dx(s.dY, s.WTc_vals, s.WTc_meta, s.d_in, s.dX))
+    stage("linear_bwd_dw_masked", lambda: B.slope_linear_bwd_dw_masked(s.dY, s.X, s.mask1, s.dWc))
+
+
+def cpu_baseline_sample(wl, seconds_hint=15.0):
+    """Time the oracle, as it stands, on a bounded sample of the workload's first layer."""
+    import oracle
+
+    oracle.build()
+    lay = wl.layers[0]
+    b = wl.tokens
+    t = si.layer_tensors(wl, 0, tokens=b)
+    _, _, mask1 = oracle.prune24(t["W"])
+    _, _, mask2 = oracle.double_prune(t["W"], mask1)
+    n_rows = 1024
+    rows = si.sample_indices(b, n_rows, 1)
+    orows = si.sample_indices(lay.d_out, n_rows, 2)
+    t0 = time.perf_counter()
+    oracle.fwd_rows(t["X"], t["W"], mask1, rows, t.get("L"), t.get("R"))
+    oracle.dx_rows(t["dY"], t["W"], mask2, rows, t.get("L"), t.get("R"))
+    oracle.dw_rows(t["dY"], t["X"], mask1, orows)
+    dt = time.perf_counter() - t0
+    r = wl.rank
+    flops = (2 * len(rows) * (2.0 * lay.d_in * lay.d_out + 2.0 * r * (lay.d_in + lay.d_out))
+             + len(orows) * 2.0 * b * lay.d_in)
+    return {"value": flops / dt / 1e12, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
+            "seconds": round(dt, 2),
+            "sample": f"layer '{lay.name}' {lay.d_in}->{lay.d_out}, b={b}: fwd+dX on {len(rows)} token rows, "
+                      f"masked dW on {len(orows)} d_out rows (dense-equivalent FLOPs of the sample / wall time)"}
+
+
+def run_reference(args, rank):
+    """The reference arm: the fp64 CPU oracle on the machine's host cores (there is no other
+    implementation of the paper to run)."""
+    if rank != 0:
+        return
+    wl = si.WORKLOADS[args.workload]
+    import oracle
+
+    oracle.build()
+    lay = wl.layers[0]
+    b = wl.tokens
+    t = si.layer_tensors(wl, 0, tokens=b)
+    _, _, mask1 = oracle.prune24(t["W"])
+    _, _, mask2 = oracle.double_prune(t["W"], mask1)
+    n_rows = 128
+    rows = si.sample_indices(b, n_rows, 1)
+    orows = si.sample_indices(lay.d_out, n_rows, 2)
+    r = wl.rank
+    flops = (2 * len(rows) * (2.0 * lay.d_in * lay.d_out + 2.0 * r * (lay.d_in + lay.d_out))
+             + len(orows) * 2.0 * b * lay.d_in)
+
+    def step():
+        oracle.fwd_rows(t["X"], t["W"], mask1, rows, t.get("L"), t.get("R"))
+        oracle.dx_rows(t["dY"], t["W"], mask2, rows, t.get("L"), t.get("R"))
+        oracle.dw_rows(t["dY"], t["X"], mask1, orows)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    val = flops * args.steps / dt / 1e12
+    sample = (f"each step: layer '{lay.name}' {lay.d_in}->{lay.d_out}, b={b}: fwd+dX on {len(rows)} token rows, "
+              f"masked dW on {len(orows)} d_out rows")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.key, "tokens": b, "rank": r, "note": "bounded sample of the workload per step"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }), flush=True)
+
+
+def replica_max_ms(torch, dist, ms_local, device):
+    """Replicas only: the job's time is the slowest rank's device time."""
+    if dist is None:
+        return float(ms_local)
+    tt = torch.tensor([ms_local], device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def replica_throughput(world, flops_per_replica, ms_step):
+    """Whole-job dense-equivalent TFLOP/s of `world` independent replicas."""
+    return world * flops_per_replica / (ms_step * 1e-3) / 1e12
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(si.WORKLOADS))
+    ap.add_argument("--impl", default="slope", choices=["slope", "reference"])
+    ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling only)")
+    ap.add_argument("--no-extras", action="store_true", help="skip dense comparison, e2e and CPU baseline")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "slope" and not args.tokens else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    from paper_2608_24070_b200 import binding as B
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the SLoPe path has no CPU fallback")
+    B.lib()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    pk = peaks()
+    wl = si.WORKLOADS[args.workload]
+    b = args.tokens or wl.tokens
+    layers = [LayerState(B, torch, wl, i, b, dev) for i in range(len(wl.layers))]
+    de_flops, ex_flops = workload_flops(wl, b)
+    stream = torch.cuda.current_stream()
+
+    def step(rec=None):
+        for s in layers:
+            run_layer(B, s, rec)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    st = B.slope_poll_status()
+    if st != 0:
+        raise SystemExit(f"device status after warm-up: {B.slope_status_string(st)}")
+
+    # ---------------- timed region: exactly K steps, device time, max over ranks
+    events = []
+
+    def rec(op, s, fn):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        fn()
+        e1.record(stream)
+        events.append((op, s, e0, e1))
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = B.slope_launch_count()
+    barrier()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step(rec)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    launches = B.slope_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = replica_max_ms(torch, dist, ev0.elapsed_time(ev1), dev)
+    st = B.slope_poll_status()
+    if st != 0:
+        raise SystemExit(f"device status after the timed region: {B.slope_status_string(st)}")
+    ms_step = ms_total / args.steps
+    value = replica_throughput(world, de_flops, ms_step)
+
+    # ---------------- per-stage times from the same timed region
+    per_op = {op: 0.0 for op in OPS}
+    per_layer_op = {}
+    for op, s, e0, e1 in events:
+        ms = e0.elapsed_time(e1)
+        per_op[op] += ms
+        per_layer_op.setdefault((s.name, s.d_in, s.d_out, op), []).append(ms)
+    per_op_ms_step = {op: v / args.steps for op, v in per_op.items() if v > 0}
+
+    def op_flops(op, s):
+        m = 2.0 * s.b * s.d_in * s.d_out
+        return {"linear_fwd": m + 2.0 * s.b * s.r * s.d_out, "linear_bwd_dx": m + 2.0 * s.b * s.r * s.d_in,
+                "linear_bwd_dw_masked": m}.get(op, 0.0)
+
+    sparse_peak = 2.0 * pk["bf16_sustained"]
+    stage_rows = []
+    tot = {"linear_fwd": [0.0, 0.0], "linear_bwd_dx": [0.0, 0.0], "linear_bwd_dw_masked": [0.0, 0.0]}
+    seen = set()
+    for (name, d_in, d_out, op), lst in per_layer_op.items():
+        ms = statistics.mean(lst)
+        s = next(x for x in layers if x.name == name)
+        fl = op_flops(op, s)
+        if fl:
+            tot[op][0] += fl
+            tot[op][1] += ms * 1e-3
+            stage_rows.append({"layer": name, "d_in": d_in, "d_out": d_out, "op": op, "ms": round(ms, 4),
+                               "tflops_dense_eq": round(fl / (ms * 1e-3) / 1e12, 1)})
+        elif op in ("prune_24", "double_prune") and (d_in, d_out, op) not in seen:
+            seen.add((d_in, d_out, op))
+            bytes_ = d_in * d_out * (3.25 if op == "prune_24" else 3.375)
+            stage_rows.append({"layer": name, "d_in": d_in, "d_out": d_out, "op": op, "ms": round(ms, 4),
+                               "gbs": round(bytes_ / (ms * 1e-3) / 1e9, 1)})
+
+    # dominant kernel by time inside the step: the dense tcgen05 GEMM of the masked weight gradient
+    dw_fl, dw_s = tot["linear_bwd_dw_masked"]
+    dw_tflops = dw_fl / dw_s / 1e12 if dw_s else 0.0
+    roofline = {"kernel": "dense_gemm_kernel<A_MN,B_MN,256,masked> (slope_linear_bwd_dw_masked)",
+                "bound": "tensor", "achieved": round(dw_tflops, 1), "peak": pk["bf16_sustained"], "unit": "TFLOP/s",
+                "frac": round(dw_tflops / pk["bf16_sustained"], 4), "traffic": None,
+                "peak_source": f"{pk['src']} sustained dense bf16"}
+    sp_fl = tot["linear_fwd"][0] + tot["linear_bwd_dx"][0]
+    sp_s = tot["linear_fwd"][1] + tot["linear_bwd_dx"][1]
+    sp_tflops = sp_fl / sp_s / 1e12 if sp_s else 0.0
+    roofline_sparse = {"kernel": "sparse_gemm_kernel (slope_linear_fwd, slope_linear_bwd_dx)", "bound": "tensor",
+                       "achieved": round(sp_tflops, 1), "peak": round(sparse_peak, 1), "unit": "TFLOP/s dense-equivalent",
+                       "frac": round(sp_tflops / sparse_peak, 4),
+                       "frac_of_datasheet_4500": round(sp_tflops / 4500.0, 4),
+                       "peak_source": f"2 x {pk['src']} sustained dense bf16"}
+
+    out = {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.key, "tokens": b, "rank": wl.rank, "layers": [f"{l.name}:{l.d_in}->{l.d_out}" for l in wl.layers],
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": "inputs larger than L2 (each layer streams > 126 MB of activations)",
+                   "step": "prune_24 + double_prune + adapter + fwd + dX + masked dW for every layer"},
+        "executed_tflops": round(world * ex_flops / (ms_step * 1e-3) / 1e12, 2),
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roofline,
+        "roofline_sparse": roofline_sparse,
+        "stage_ms_per_step": {k: round(v, 4) for k, v in per_op_ms_step.items()},
+        "stages": stage_rows,
+    }
+
+    if rank == 0 and not args.no_extras and world == 1:
+        out["dense_layer"] = dense_comparison(torch, B, layers, stream)
+        out["e2e"] = e2e_run(torch, B, layers, de_flops, max(2, min(args.steps, 5)))
+        out["cpu_baseline"] = cpu_baseline_sample(wl)
+    elif rank == 0:
+        out["e2e"] = None
+        out["cpu_baseline"] = None
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def dense_comparison(torch, B, layers, stream, reps=5):
+    """fwd+bwd of the same layers as dense bf16 GEMMs (torch.matmul -> cuBLAS), interleaved with the
+    SLoPe stages fwd/dX/dW (no pruning, no adapter) in the same process."""
+    t_dense = t_slope = 0.0
+    rows = []
+    for s in layers:
+        Wd = s.W
+        ed = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        es = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        md, ms_ = [], []
+        for _ in range(reps + 1):
+            ed[0].record(stream)
+            Y = torch.matmul(s.X, Wd.t())
+            dX = torch.matmul(s.dY, Wd)
+            dW = torch.matmul(s.dY.t(), s.X)
+            ed[1].record(stream)
+            es[0].record(stream)
+            B.slope_linear_fwd(s.X, s.Wc_vals, s.Wc_meta, s.d_out, s.Y)
+            B.slope_linear_bwd_dx(s.dY, s.WTc_vals, s.WTc_meta, s.d_in, s.dX)
+            B.slope_linear_bwd_dw_masked(s.dY, s.X, s.mask1, s.dWc)
+            es[1].record(stream)
+            torch.cuda.synchronize()
+            md.append(ed[0].elapsed_time(ed[1]))
+            ms_.append(es[0].elapsed_time(es[1]))
+            del Y, dX, dW
+        d, sl = statistics.median(md[1:]), statistics.median(ms_[1:])
+        t_dense += d
+        t_slope += sl
+        rows.append({"layer": s.name, "dense_ms": round(d, 4), "slope_ms": round(sl, 4), "speedup": round(d / sl, 3)})
+    return {"what": "torch.matmul (cuBLAS) Y=XW^T, dX=dY W, dW=dY^T X vs slope fwd+dX+masked dW, same shapes, interleaved",
+            "dense_ms": round(t_dense, 4), "slope_ms": round(t_slope, 4), "speedup": round(t_dense / t_slope, 3),
+            "layers": rows}
+
+
+def e2e_run(torch, B, layers, de_flops, steps):
+    """Same step with HOST buffers: every step copies each layer's X and dY from pinned host
+    memory, runs the path through the C ABI, and reads the compressed weight gradient back."""
+    stream = torch.cuda.current_stream()
+    host = {}
+    for s in layers:
+        for nm, t in (("X", s.X), ("dY", s.dY)):
+            key = (nm, tuple(t.shape))
+            if key not in host:
+                host[key] = t.cpu().pin_memory()
+        key = ("dWc", tuple(s.dWc.shape))
+        if key not in host:
+            host[key] = torch.empty(s.dWc.shape, dtype=s.dWc.dtype).pin_memory()
+    h2d = sum(2 * (s.X.numel() + s.dY.numel()) for s in layers)
+    d2h = sum(2 * s.dWc.numel() for s in layers)
+
+    def step():
+        for s in layers:
+            s.X.copy_(host[("X", tuple(s.X.shape))], non_blocking=True)
+            s.dY.copy_(host[("dY", tuple(s.dY.shape))], non_blocking=True)
+            run_layer(B, s)
+            host[("dWc", tuple(s.dWc.shape))].copy_(s.dWc, non_blocking=True)
+
+    step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    return {"value": round(de_flops / (ms * 1e-3) / 1e12, 2), "unit": UNIT, "ms_per_step": round(ms, 3),
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": steps}
+
+
+if __name__ == "__main__":
+    main()
