@@ -146,13 +146,17 @@ static slope_status_t launch_dense(const void* A, const void* B, int M, int N, i
 }
 
 static int adapter_splits(int b, int rows) {
-    // enough K-splits that (row tiles x splits) covers the machine, each split >= 512 tokens
+    // enough K-splits that (row tiles x splits) covers the machine, each split >= 512 tokens,
+    // and no split without a k-block (an empty split would leave its accumulator unwritten)
     const int tiles = (rows + kBlockM - 1) / kBlockM;
     int s = (148 + tiles - 1) / tiles;
     const int max_s = b / 512 > 0 ? b / 512 : 1;
     if (s > max_s) s = max_s;
     if (s > 16) s = 16;
-    return s < 1 ? 1 : s;
+    if (s < 1) s = 1;
+    const int num_kb = (b + 63) / 64;
+    const int per = (num_kb + s - 1) / s;
+    return (num_kb + per - 1) / per;
 }
 
 static bool dims_ok(int d_out, int d_in) {
