@@ -130,6 +130,29 @@ slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY,
                                      void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * dL[d_in x r] = X[b x d_in]^T dT[b x r] without any allocation, for callers that cannot
+ * call cudaMalloc or hand over a workspace (code running inside a host application whose
+ * memory pool is closed to it, or in a section where allocation is forbidden).
+ * The thesis has no counterpart of this call; it computes the same dL as phase 1 of
+ * slope_adapter_fwd_bwd from the same bf16 dT.
+ *  - The split-K partial sums live in a fixed 16 MiB array inside the library image
+ *    (slope_adapter_dl_noalloc_max_scratch_bytes()); every GPU that loads the library
+ *    holds that array until the process exits.
+ *  - Sizes whose partial sums do not fit (splits * d_in * r * 4 bytes, with at most 16
+ *    splits) are rejected with SLOPE_ERR_SHAPE before anything is launched; use
+ *    slope_adapter_fwd_bwd with a workspace for those.
+ *  - The first call on a device looks up the array's device address (once per device,
+ *    with that device current); make that first call before any stream capture.
+ *  - All calls on a device share the one array.  Nothing in it needs clearing between
+ *    calls, but two calls whose kernels overlap on the GPU (different streams) race on
+ *    it: serialise them.
+ * Calls no cudaMalloc / cudaFree and no allocating library routine.
+ */
+size_t slope_adapter_dl_noalloc_max_scratch_bytes(void);
+slope_status_t slope_adapter_dl_noalloc(const void* X, const void* dT, int b, int d_in, int r,
+                                        void* dL, void* stream);
+
+/*
  * Diagnostic: rewrite tensor-core-order metadata as canonical metadata
  * (uint16 [rows x cols/16], group g of a row at bits 4*(g%4) of unit g/4).
  * Paper counterpart: none (the index storage of Eq. (index_bits) in a

@@ -27,6 +27,7 @@ EXPORTS = (
     "slope_prune_24", "slope_double_prune", "slope_linear_fwd", "slope_linear_bwd_dx",
     "slope_linear_bwd_dw_masked", "slope_adapter_workspace_bytes", "slope_adapter_fwd_bwd",
     "slope_meta_to_canonical", "slope_poll_status", "slope_launch_count", "slope_status_string",
+    "slope_adapter_dl_noalloc", "slope_adapter_dl_noalloc_max_scratch_bytes",
 )
 
 
@@ -57,6 +58,10 @@ def lib() -> ctypes.CDLL:
         L.slope_adapter_workspace_bytes.argtypes = [ci, ci, ci, ci]
         L.slope_adapter_fwd_bwd.argtypes = [ci, vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, vp, sz, vp]
         L.slope_meta_to_canonical.argtypes = [vp, ci, ci, vp, vp]
+        L.slope_adapter_dl_noalloc.argtypes = [vp, vp, ci, ci, ci, vp, vp]
+        L.slope_adapter_dl_noalloc.restype = ci
+        L.slope_adapter_dl_noalloc_max_scratch_bytes.restype = sz
+        L.slope_adapter_dl_noalloc_max_scratch_bytes.argtypes = []
         L.slope_poll_status.argtypes = [vp]
         L.slope_launch_count.restype = ctypes.c_ulonglong
         L.slope_status_string.restype = ctypes.c_char_p
@@ -139,6 +144,19 @@ def slope_adapter_fwd_bwd(phase, X, dY, L, R, b, d_out, d_in, r, T=None, dT=None
     _check("slope_adapter_fwd_bwd", lib().slope_adapter_fwd_bwd(
         phase, _ptr(X), _ptr(dY), _ptr(L), _ptr(R), b, d_out, d_in, r, _ptr(T), _ptr(dT), _ptr(dL), _ptr(dR),
         _ptr(workspace), ws_bytes, _stream()))
+
+
+def slope_adapter_dl_noalloc(X, dT, dL):
+    """dL = X^T dT with the split-K scratch in the library's fixed device array (no allocation,
+    no workspace argument).  For callers that are not allowed to allocate GPU memory."""
+    b, d_in = X.shape
+    r = dT.shape[1]
+    _check("slope_adapter_dl_noalloc", lib().slope_adapter_dl_noalloc(_ptr(X), _ptr(dT), b, d_in, r, _ptr(dL),
+                                                                      _stream()))
+
+
+def slope_adapter_dl_noalloc_max_scratch_bytes() -> int:
+    return int(lib().slope_adapter_dl_noalloc_max_scratch_bytes())
 
 
 def slope_meta_to_canonical(meta_hw, rows, cols, meta_canon):

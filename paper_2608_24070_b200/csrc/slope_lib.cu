@@ -338,3 +338,62 @@ slope_status_t slope_meta_to_canonical(const void* meta_hw, int rows, int cols, 
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------ allocation-free adapter-gradient entry
+// Some callers may not allocate device memory at all: a plug-in running inside a host
+// application whose memory pool is closed to it, or code that runs where cudaMalloc is
+// forbidden (a latency-critical section, a process that has handed its whole GPU memory
+// budget to a framework allocator).  For them the split-K scratch of the dL gradient lives
+// in this fixed array instead of a caller workspace.  The array belongs to the loaded
+// library image: every GPU that loads the library keeps these 16 MiB until the process
+// exits, and every call on a device shares it.
+namespace slope {
+constexpr size_t kStaticScratchBytes = size_t(16) << 20;
+static __device__ __align__(256) float g_static_scratch[kStaticScratchBytes / sizeof(float)];
+
+// In host code `g_static_scratch` is only a handle; the address kernels can use comes from
+// cudaGetSymbolAddress, asked once per device with that device current.
+static slope_status_t static_scratch_address(float** out) {
+    static std::mutex mu;
+    static float* cache[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SLOPE_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cache[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return SLOPE_ERR_CUDA;
+        cache[dev] = static_cast<float*>(p);
+    }
+    *out = cache[dev];
+    return SLOPE_OK;
+}
+}  // namespace slope
+
+extern "C" {
+
+size_t slope_adapter_dl_noalloc_max_scratch_bytes(void) { return kStaticScratchBytes; }
+
+slope_status_t slope_adapter_dl_noalloc(const void* X, const void* dT, int b, int d_in, int r, void* dL,
+                                        void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!X || !dT || !dL) return SLOPE_ERR_INVALID_ARG;
+    if (d_in <= 0 || d_in % 128 != 0 || b < 8 || b % 8 != 0 || !rank_ok(r) || r == 0) return SLOPE_ERR_SHAPE;
+    if (!aligned16(X) || !aligned16(dT) || !aligned16(dL)) return SLOPE_ERR_ALIGNMENT;
+    const int splits = adapter_splits(b, d_in);
+    const size_t need = static_cast<size_t>(splits) * d_in * r * sizeof(float);
+    if (need > kStaticScratchBytes) return SLOPE_ERR_SHAPE;      // beyond the fixed scratch: use the workspace call
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    float* scratch = nullptr;
+    if (slope_status_t st = static_scratch_address(&scratch)) return st;
+    // Nothing has to start at zero: every partial sum the reduction reads is written by the
+    // GEMM of this same call, so what an earlier call left in the array is never observed.
+    slope_status_t st =
+        r <= 64 ? launch_dense<true, true, 64, kEpiPartial, 6>(X, dT, d_in, r, b, splits, scratch, nullptr, stream, info)
+                : launch_dense<true, true, 128, kEpiPartial, 6>(X, dT, d_in, r, b, splits, scratch, nullptr, stream, info);
+    if (st) return st;
+    splitk_reduce_kernel<<<info.sm_count * 4, 256, 0, stream>>>(scratch, d_in, r, splits, 0, static_cast<uint16_t*>(dL));
+    return launch_result();
+}
+
+}  // extern "C"
