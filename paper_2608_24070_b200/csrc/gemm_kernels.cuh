@@ -445,4 +445,378 @@ splitk_reduce_kernel(const float* __restrict__ ws, int M, int N, int splits, int
     }
 }
 
+
+// =====================================================================================
+// CTA-pair versions (cluster of 2, tcgen05 cta_group::2).  One MMA spans both SMs: the pair
+// owns a 256-row tile of the A operand (128 rows per CTA) and each CTA stages only HALF of
+// the B tile, which halves the activation bytes every SM pulls from L2 per MMA and leaves
+// room for twice as many pipeline stages.  The leader CTA (rank 0) issues all MMAs; both
+// CTAs run their own TMA producer (completion bytes are counted on the leader's barrier)
+// and their own epilogue (each drains its 128 accumulator rows).  tcgen05.commit arrives on
+// the barriers of both CTAs; the epilogues release an accumulator stage by arriving on the
+// leader's barrier through the cluster shared-memory window.
+// =====================================================================================
+template <int BLOCK_N, int STAGES>
+struct SparsePairCfg {
+    static constexpr int kHalfN = BLOCK_N / 2;
+    static constexpr int kABytes = kBlockM * 128;
+    static constexpr int kBBytes = kHalfN * 256;
+    static constexpr int kEBytes = 2048;
+    static constexpr int kStageBytes = kABytes + kBBytes + kEBytes;
+    static constexpr int kSmemBytes = STAGES * kStageBytes + 256 + 1024;
+    static constexpr int kECol = 2 * BLOCK_N;
+    static_assert(BLOCK_N % 16 == 0 && kHalfN % 8 == 0 && 2 * BLOCK_N + 8 <= 512, "tile does not fit tensor memory");
+    static_assert(kStageBytes % 1024 == 0, "stage must keep 1024-byte alignment");
+};
+
+template <int BLOCK_N, int STAGES>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                        const __grid_constant__ CUtensorMap tmE, const __grid_constant__ CUtensorMap tmA2,
+                        const __grid_constant__ CUtensorMap tmB2, const SparseGemmParams p) {
+    using Cfg = SparsePairCfg<BLOCK_N, STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * Cfg::kStageBytes);
+    uint64_t* empty_bar = full_bar + STAGES;
+    uint64_t* tfull_bar = empty_bar + STAGES;
+    uint64_t* tempty_bar = tfull_bar + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cta = cluster_ctarank();                  // 0 = leader
+    const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int num_mb = p.M / kBlockM;                        // 128-row blocks of A
+    const int num_m = (num_mb + 1) / 2;                      // 256-row pair tiles
+    const int num_n = (p.Ntok + BLOCK_N - 1) / BLOCK_N;
+    const int num_tiles = num_m * num_n;
+    const int num_kb = p.K / 128;
+    const int num_ab = (p.r + 63) / 64;
+    const int total_kb = num_kb + num_ab;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], 8); }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(tmem_slot, 512);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();                                      // peer barriers are initialised
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (both CTAs)
+        if (elect_one()) {
+            tma_prefetch_desc(&tmA);
+            tma_prefetch_desc(&tmB);
+            tma_prefetch_desc(&tmE);
+            PipeState ps;
+            bool ok = true;
+            for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
+                const int m_pair = tile % num_m, n_blk = tile / num_m;
+                const int mb = m_pair * 2 + static_cast<int>(cta);           // this CTA's 128-row block
+                const int mb_e = mb < num_mb ? mb : num_mb - 1;              // rows past M: any valid metadata block
+                const int n_row0 = n_blk * BLOCK_N + static_cast<int>(cta) * Cfg::kHalfN;
+                for (int kb = 0; kb < total_kb; ++kb) {
+                    if (!mbar_wait(&empty_bar[ps.stage], ps.phase ^ 1u, abort_flag)) { ok = false; break; }
+                    uint8_t* sA = smem + ps.stage * Cfg::kStageBytes;
+                    uint8_t* sB = sA + Cfg::kABytes;
+                    uint8_t* sE = sB + Cfg::kBBytes;
+                    const uint32_t bar = mapa_shared(smem_u32(&full_bar[ps.stage]), 0);
+                    if (kb < num_kb) {
+                        if (cta == 0) mbar_expect_tx(&full_bar[ps.stage], 2 * Cfg::kStageBytes);
+                        tma_load_2d_pair(sA, &tmA, bar, kb * 64, mb * kBlockM);
+                        tma_load_2d_pair(sB, &tmB, bar, kb * 128, n_row0);
+                        tma_load_2d_pair(sB + Cfg::kHalfN * 128, &tmB, bar, kb * 128 + 64, n_row0);
+                        tma_load_2d_pair(sE, &tmE, bar, 0, (mb_e * num_kb + kb) * 128);
+                    } else {
+                        const int ab = kb - num_kb;
+                        if (cta == 0) mbar_expect_tx(&full_bar[ps.stage], 2 * (Cfg::kABytes + Cfg::kHalfN * 128));
+                        if (p.a2_mn_major) {
+                            tma_load_2d_pair(sA, &tmA2, bar, mb * kBlockM, ab * 64);
+                            tma_load_2d_pair(sA + 8192, &tmA2, bar, mb * kBlockM + 64, ab * 64);
+                        } else {
+                            tma_load_2d_pair(sA, &tmA2, bar, ab * 64, mb * kBlockM);
+                        }
+                        tma_load_2d_pair(sB, &tmB2, bar, ab * 64, n_row0);
+                    }
+                    ps.advance(STAGES);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (cta == 0 && elect_one()) {
+            constexpr uint32_t idesc_sp = make_idesc_bf16(2 * kBlockM, BLOCK_N, false, false, true);
+            const uint32_t idesc_ad = make_idesc_bf16(2 * kBlockM, BLOCK_N, p.a2_mn_major != 0, false, false);
+            PipeState ps;
+            bool ok = true;
+            int it = 0;
+            for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
+                const int acc = it & 1;
+                const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
+                if (!mbar_wait(&tempty_bar[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * BLOCK_N;
+                for (int kb = 0; kb < total_kb; ++kb) {
+                    if (!mbar_wait(&full_bar[ps.stage], ps.phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t sA = smem_u32(smem + ps.stage * Cfg::kStageBytes);
+                    const uint32_t sB = sA + Cfg::kABytes;
+                    const uint32_t sE = sB + Cfg::kBBytes;
+                    if (kb < num_kb) {
+                        const uint32_t e_tmem = tmem_base + Cfg::kECol + (kb & 1) * 4;
+                        tmem_cp_128x128b_pair(e_tmem, make_smem_desc(sE, 128, 128, kSwizzleNone));
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint64_t ad = make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
+                            const uint64_t bd = make_smem_desc(sB + (j >> 1) * (Cfg::kHalfN * 128) + (j & 1) * 64, 16,
+                                                               1024, kSwizzle128B);
+                            umma_bf16_sp_pair(d_tmem, ad, bd, e_tmem + (j & 2), idesc_sp | (j & 1),
+                                              (kb | j) != 0 ? 1u : 0u);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint64_t ad = p.a2_mn_major
+                                                    ? make_smem_desc(sA + j * 2048, 8192, 1024, kSwizzle128B)
+                                                    : make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
+                            const uint64_t bd = make_smem_desc(sB + j * 32, 16, 1024, kSwizzle128B);
+                            umma_bf16_pair(d_tmem, ad, bd, idesc_ad, 1u);
+                        }
+                    }
+                    umma_commit_pair(&empty_bar[ps.stage], 3);
+                    ps.advance(STAGES);
+                }
+                if (ok) umma_commit_pair(&tfull_bar[acc], 3);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+        const int q = warp & 3;
+        bool ok = true;
+        int it = 0;
+        for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
+            const int m_pair = tile % num_m, n_blk = tile / num_m;
+            const int acc = it & 1;
+            const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
+            if (!mbar_wait(&tfull_bar[acc], acc_phase, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t t_row = tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
+            const int m = (m_pair * 2 + static_cast<int>(cta)) * kBlockM + q * 32 + lane;
+            uint16_t* out_col = p.out + m;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BLOCK_N; c0 += 16) {
+                uint32_t v[16];
+                tmem_ld_16(t_row + c0, v);
+                tmem_ld_wait();
+                const int n0 = n_blk * BLOCK_N + c0;
+                if (m < p.M) {
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const int n = n0 + c;
+                        if (n < p.Ntok) out_col[static_cast<size_t>(n) * p.M] = to_bf16(__uint_as_float(v[c]));
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&tempty_bar[acc]), 0));
+        }
+    }
+
+    __syncwarp();
+    if (*abort_flag) drain_after_abort();
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();                                      // nobody signals or reads the peer after this
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, 512);
+    }
+}
+
+// Dense CTA-pair GEMM: D[M x N] = A[M x K] * B[N x K]^T with a 256 x BLOCK_N tile per pair
+// (each CTA: 128 rows of A, BLOCK_N/2 rows of B, 128 x BLOCK_N accumulator rows).
+template <int BLOCK_N, int STAGES>
+struct DensePairCfg {
+    static constexpr int kHalfN = BLOCK_N / 2;
+    static constexpr int kABytes = kBlockM * 128;
+    static constexpr int kBBytes = kHalfN * 128;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kSmemBytes = STAGES * kStageBytes + 256 + 1024;
+    static_assert(BLOCK_N % 128 == 0 && BLOCK_N <= 256, "BLOCK_N must be 128 or 256");
+};
+
+template <bool A_MN, bool B_MN, int BLOCK_N, int EPI, int STAGES>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+dense_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                       const DenseGemmParams p) {
+    using Cfg = DensePairCfg<BLOCK_N, STAGES>;
+    constexpr int kTmemCols = 2 * BLOCK_N;                       // 256 or 512
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * Cfg::kStageBytes);
+    uint64_t* empty_bar = full_bar + STAGES;
+    uint64_t* tfull_bar = empty_bar + STAGES;
+    uint64_t* tempty_bar = tfull_bar + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cta = cluster_ctarank();
+    const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int num_m = (p.M + 2 * kBlockM - 1) / (2 * kBlockM);
+    const int num_n = (p.N + BLOCK_N - 1) / BLOCK_N;
+    const int num_kb = (p.K + 63) / 64;
+    const int num_tiles = num_m * num_n;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], 8); }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(tmem_slot, kTmemCols);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (elect_one()) {
+            tma_prefetch_desc(&tmA);
+            tma_prefetch_desc(&tmB);
+            PipeState ps;
+            bool ok = true;
+            for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
+                const int m_pair = tile % num_m, n_blk = tile / num_m;
+                const int m0 = (m_pair * 2 + static_cast<int>(cta)) * kBlockM;
+                const int n0 = n_blk * BLOCK_N + static_cast<int>(cta) * Cfg::kHalfN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&empty_bar[ps.stage], ps.phase ^ 1u, abort_flag)) { ok = false; break; }
+                    uint8_t* sA = smem + ps.stage * Cfg::kStageBytes;
+                    uint8_t* sB = sA + Cfg::kABytes;
+                    const uint32_t bar = mapa_shared(smem_u32(&full_bar[ps.stage]), 0);
+                    if (cta == 0) mbar_expect_tx(&full_bar[ps.stage], 2 * Cfg::kStageBytes);
+                    if (A_MN) {
+                        tma_load_2d_pair(sA, &tmA, bar, m0, kb * 64);
+                        tma_load_2d_pair(sA + 8192, &tmA, bar, m0 + 64, kb * 64);
+                    } else {
+                        tma_load_2d_pair(sA, &tmA, bar, kb * 64, m0);
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int h = 0; h < Cfg::kHalfN / 64; ++h)
+                            tma_load_2d_pair(sB + h * 8192, &tmB, bar, n0 + h * 64, kb * 64);
+                    } else {
+                        tma_load_2d_pair(sB, &tmB, bar, kb * 64, n0);
+                    }
+                    ps.advance(STAGES);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (cta == 0 && elect_one()) {
+            constexpr uint32_t idesc = make_idesc_bf16(2 * kBlockM, BLOCK_N, A_MN, B_MN, false);
+            PipeState ps;
+            bool ok = true;
+            int it = 0;
+            for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
+                const int acc = it & 1;
+                const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
+                if (!mbar_wait(&tempty_bar[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * BLOCK_N;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&full_bar[ps.stage], ps.phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t sA = smem_u32(smem + ps.stage * Cfg::kStageBytes);
+                    const uint32_t sB = sA + Cfg::kABytes;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint64_t ad = A_MN ? make_smem_desc(sA + j * 2048, 8192, 1024, kSwizzle128B)
+                                                 : make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
+                        const uint64_t bd = B_MN ? make_smem_desc(sB + j * 2048, 8192, 1024, kSwizzle128B)
+                                                 : make_smem_desc(sB + j * 32, 16, 1024, kSwizzle128B);
+                        umma_bf16_pair(d_tmem, ad, bd, idesc, (kb | j) != 0 ? 1u : 0u);
+                    }
+                    umma_commit_pair(&empty_bar[ps.stage], 3);
+                    ps.advance(STAGES);
+                }
+                if (ok) umma_commit_pair(&tfull_bar[acc], 3);
+            }
+        }
+    } else {
+        const int q = warp & 3;
+        bool ok = true;
+        int it = 0;
+        for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
+            const int m_pair = tile % num_m, n_blk = tile / num_m;
+            const int acc = it & 1;
+            const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
+            if (!mbar_wait(&tfull_bar[acc], acc_phase, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t t_row = tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
+            const int m = (m_pair * 2 + static_cast<int>(cta)) * kBlockM + q * 32 + lane;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BLOCK_N; c0 += 16) {
+                uint32_t v[16];
+                tmem_ld_16(t_row + c0, v);
+                tmem_ld_wait();
+                const int n0 = n_blk * BLOCK_N + c0;
+                if (m >= p.M || n0 >= p.N) continue;
+                if (EPI == kEpiStore) {
+                    uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + static_cast<size_t>(m) * p.N + n0);
+                    uint32_t w[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) w[c] = pack_bf16x2(__uint_as_float(v[2 * c]), __uint_as_float(v[2 * c + 1]));
+                    dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                    dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                } else {
+                    const uint32_t mbits =
+                        *reinterpret_cast<const uint16_t*>(p.mask + static_cast<size_t>(m) * (p.N >> 3) + (n0 >> 3));
+                    uint32_t w[4];
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        const uint32_t mb = (mbits >> (4 * g)) & 0xFu;
+                        const int p0 = __ffs(mb) - 1, p1 = 31 - __clz(mb);
+                        const float e0 = __uint_as_float(v[4 * g]), e1 = __uint_as_float(v[4 * g + 1]),
+                                    e2 = __uint_as_float(v[4 * g + 2]), e3 = __uint_as_float(v[4 * g + 3]);
+                        const float lo = p0 == 0 ? e0 : (p0 == 1 ? e1 : e2);
+                        const float hi = p1 == 1 ? e1 : (p1 == 2 ? e2 : e3);
+                        w[g] = pack_bf16x2(lo, hi);
+                    }
+                    *reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + static_cast<size_t>(m) * (p.N >> 1) + (n0 >> 1)) =
+                        make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&tempty_bar[acc]), 0));
+        }
+    }
+
+    __syncwarp();
+    if (*abort_flag) drain_after_abort();
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+}
+
 }  // namespace slope

@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstring>
 #include <mutex>
+#include <utility>
 
 #include "gemm_kernels.cuh"
 #include "prune_kernels.cuh"
@@ -66,6 +67,40 @@ static bool make_tmap(CUtensorMap* tm, const void* base, int rows, int cols, int
     return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Metadata as a 2-D byte tensor [bytes/16 x 16]: one 2 KB block = a 16 x 128 box, no swizzle.
+static bool make_tmap_meta(CUtensorMap* tm, const void* base, size_t total_bytes) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t gdim[2] = {16, static_cast<cuuint64_t>(total_bytes / 16)};
+    const cuuint64_t gstride[1] = {16};
+    const cuuint32_t box[2] = {16, 128};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Launch on clusters of two CTAs (cta_group::2 kernels).
+template <typename... KArgs, typename... Args>
+static slope_status_t launch_pairs(void (*kern)(KArgs...), int grid, int smem_bytes, cudaStream_t stream,
+                                   Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(kGemmThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? SLOPE_OK : SLOPE_ERR_CUDA;
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -143,6 +178,64 @@ static slope_status_t launch_dense(const void* A, const void* B, int M, int N, i
     const int grid = tiles < info.sm_count ? tiles : info.sm_count;
     kern<<<grid, kGemmThreads, Cfg::kSmemBytes, stream>>>(tmA, tmB, p);
     return launch_result();
+}
+
+// ------------------------------------------------------------------ CTA-pair launches (main GEMMs)
+constexpr int kPairBlockN = 240;
+constexpr int kPairStages = 4;
+
+static slope_status_t launch_sparse_pair(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
+                                         const void* act2, const void* fac2, int r, bool a2_mn, void* out,
+                                         cudaStream_t stream, const DeviceInfo& info) {
+    using Cfg = SparsePairCfg<kPairBlockN, kPairStages>;
+    CUtensorMap tmA, tmB, tmE, tmA2, tmB2;
+    if (!make_tmap(&tmA, vals, M, K / 2, kBlockM, 64)) return SLOPE_ERR_CUDA;
+    if (!make_tmap(&tmB, act, ntok, K, Cfg::kHalfN, 64)) return SLOPE_ERR_CUDA;
+    if (!make_tmap_meta(&tmE, meta, static_cast<size_t>(M) * K / 8)) return SLOPE_ERR_CUDA;
+    if (r > 0) {
+        const bool ok2 = a2_mn ? make_tmap(&tmA2, fac2, r, M, 64, 64) : make_tmap(&tmA2, fac2, M, r, kBlockM, 64);
+        if (!ok2 || !make_tmap(&tmB2, act2, ntok, r, Cfg::kHalfN, 64)) return SLOPE_ERR_CUDA;
+    } else {
+        tmA2 = tmA;
+        tmB2 = tmB;
+    }
+    SparseGemmParams p;
+    p.M = M; p.K = K; p.Ntok = ntok; p.r = r; p.a2_mn_major = a2_mn ? 1 : 0;
+    p.meta = static_cast<const uint8_t*>(meta);
+    p.out = static_cast<uint16_t*>(out);
+    auto kern = sparse_gemm_pair_kernel<kPairBlockN, kPairStages>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
+        attr_set = true;
+    }
+    const int tiles = ((M / kBlockM + 1) / 2) * ((ntok + kPairBlockN - 1) / kPairBlockN);
+    const int max_pairs = info.sm_count / 2;
+    const int pairs = tiles < max_pairs ? tiles : max_pairs;
+    return launch_pairs(kern, 2 * pairs, Cfg::kSmemBytes, stream, tmA, tmB, tmE, tmA2, tmB2, p);
+}
+
+template <bool A_MN, bool B_MN, int BLOCK_N, int EPI, int STAGES>
+static slope_status_t launch_dense_pair(const void* A, const void* B, int M, int N, int K, void* out,
+                                        const void* mask, cudaStream_t stream, const DeviceInfo& info) {
+    using Cfg = DensePairCfg<BLOCK_N, STAGES>;
+    CUtensorMap tmA, tmB;
+    const bool okA = A_MN ? make_tmap(&tmA, A, K, M, 64, 64) : make_tmap(&tmA, A, M, K, kBlockM, 64);
+    const bool okB = B_MN ? make_tmap(&tmB, B, K, N, 64, 64) : make_tmap(&tmB, B, N, K, Cfg::kHalfN, 64);
+    if (!okA || !okB) return SLOPE_ERR_CUDA;
+    DenseGemmParams p;
+    p.M = M; p.N = N; p.K = K; p.k_splits = 1; p.out = out;
+    p.mask = static_cast<const uint8_t*>(mask);
+    auto kern = dense_gemm_pair_kernel<A_MN, B_MN, BLOCK_N, EPI, STAGES>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
+        attr_set = true;
+    }
+    const int tiles = ((M + 2 * kBlockM - 1) / (2 * kBlockM)) * ((N + BLOCK_N - 1) / BLOCK_N);
+    const int max_pairs = info.sm_count / 2;
+    const int pairs = tiles < max_pairs ? tiles : max_pairs;
+    return launch_pairs(kern, 2 * pairs, Cfg::kSmemBytes, stream, tmA, tmB, p);
 }
 
 static int adapter_splits(int b, int rows) {
@@ -245,8 +338,8 @@ slope_status_t slope_linear_fwd(const void* X, int b, const void* Wc_vals, const
         return SLOPE_ERR_ALIGNMENT;
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
-    return launch_sparse(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R, r, /*a2_mn=*/true, Y,
-                         static_cast<cudaStream_t>(stream), info);
+    return launch_sparse_pair(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R, r, /*a2_mn=*/true, Y,
+                              static_cast<cudaStream_t>(stream), info);
 }
 
 slope_status_t slope_linear_bwd_dx(const void* dY, int b, const void* WTc_vals, const void* WTc_meta, int d_out,
@@ -259,8 +352,8 @@ slope_status_t slope_linear_bwd_dx(const void* dY, int b, const void* WTc_vals, 
         return SLOPE_ERR_ALIGNMENT;
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
-    return launch_sparse(dY, b, WTc_vals, WTc_meta, d_in, d_out, dT, L, r, /*a2_mn=*/false, dX,
-                         static_cast<cudaStream_t>(stream), info);
+    return launch_sparse_pair(dY, b, WTc_vals, WTc_meta, d_in, d_out, dT, L, r, /*a2_mn=*/false, dX,
+                              static_cast<cudaStream_t>(stream), info);
 }
 
 slope_status_t slope_linear_bwd_dw_masked(const void* dY, const void* X, int b, int d_out, int d_in,
@@ -270,8 +363,8 @@ slope_status_t slope_linear_bwd_dw_masked(const void* dY, const void* X, int b, 
     if (!aligned16(dY) || !aligned16(X) || !aligned16(mask1_bits) || !aligned16(dWc_vals)) return SLOPE_ERR_ALIGNMENT;
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
-    return launch_dense<true, true, 256, kEpiMasked, 4>(dY, X, d_out, d_in, b, 1, dWc_vals, mask1_bits,
-                                                        static_cast<cudaStream_t>(stream), info);
+    return launch_dense_pair<true, true, 256, kEpiMasked, 6>(dY, X, d_out, d_in, b, dWc_vals, mask1_bits,
+                                                             static_cast<cudaStream_t>(stream), info);
 }
 
 size_t slope_adapter_workspace_bytes(int b, int d_out, int d_in, int r) {
