@@ -47,180 +47,6 @@ struct SparseGemmParams {
     uint16_t* out;                // [Ntok x M]
 };
 
-template <int BLOCK_N, int STAGES>
-struct SparseCfg {
-    static constexpr int kABytes = kBlockM * 128;                // 128 rows x 64 compressed bf16
-    static constexpr int kBBytes = BLOCK_N * 256;                // BLOCK_N rows x 128 bf16 (two 64-wide boxes)
-    static constexpr int kEBytes = 2048;
-    static constexpr int kStageBytes = kABytes + kBBytes + kEBytes;
-    static constexpr int kBarBytes = 256;
-    static constexpr int kSmemBytes = STAGES * kStageBytes + kBarBytes + 1024;   // + alignment slack
-    static constexpr int kECol = 2 * BLOCK_N;                    // metadata columns after both accumulators
-    static_assert(BLOCK_N % 16 == 0 && BLOCK_N >= 16 && 2 * BLOCK_N + 8 <= 512, "tile does not fit tensor memory");
-    static_assert(kStageBytes % 1024 == 0, "stage must keep 1024-byte alignment for the 128-byte swizzle");
-};
-
-template <int BLOCK_N, int STAGES>
-__global__ void __launch_bounds__(kGemmThreads, 1)
-sparse_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                   const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
-                   const SparseGemmParams p) {
-    using Cfg = SparseCfg<BLOCK_N, STAGES>;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * Cfg::kStageBytes);
-    uint64_t* empty_bar = full_bar + STAGES;
-    uint64_t* tfull_bar = empty_bar + STAGES;
-    uint64_t* tempty_bar = tfull_bar + 2;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_m = p.M / kBlockM;
-    const int num_n = (p.Ntok + BLOCK_N - 1) / BLOCK_N;
-    const int num_tiles = num_m * num_n;
-    const int num_kb = p.K / 128;
-    const int num_ab = (p.r + 63) / 64;
-    const int total_kb = num_kb + num_ab;
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], 128); }
-        *abort_flag = 0;
-        fence_mbar_init();
-    }
-    if (warp == 1) {
-        tmem_alloc(tmem_slot, 512);
-        tmem_relinquish();
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot;
-
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        if (elect_one()) {
-            tma_prefetch_desc(&tmA);
-            tma_prefetch_desc(&tmB);
-            PipeState ps;
-            bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                const int m_blk = tile % num_m, n_blk = tile / num_m;
-                for (int kb = 0; kb < total_kb; ++kb) {
-                    if (!mbar_wait(&empty_bar[ps.stage], ps.phase ^ 1u, abort_flag)) { ok = false; break; }
-                    uint8_t* sA = smem + ps.stage * Cfg::kStageBytes;
-                    uint8_t* sB = sA + Cfg::kABytes;
-                    uint8_t* sE = sB + Cfg::kBBytes;
-                    uint64_t* bar = &full_bar[ps.stage];
-                    if (kb < num_kb) {
-                        mbar_expect_tx(bar, Cfg::kABytes + Cfg::kBBytes + Cfg::kEBytes);
-                        tma_load_2d(sA, &tmA, bar, kb * 64, m_blk * kBlockM);
-                        tma_load_2d(sB, &tmB, bar, kb * 128, n_blk * BLOCK_N);
-                        tma_load_2d(sB + BLOCK_N * 128, &tmB, bar, kb * 128 + 64, n_blk * BLOCK_N);
-                        bulk_load_1d(sE, p.meta + (static_cast<size_t>(m_blk) * num_kb + kb) * 2048, 2048, bar);
-                    } else {
-                        const int ab = kb - num_kb;
-                        mbar_expect_tx(bar, Cfg::kABytes + BLOCK_N * 128);
-                        if (p.a2_mn_major) {
-                            tma_load_2d(sA, &tmA2, bar, m_blk * kBlockM, ab * 64);
-                            tma_load_2d(sA + 8192, &tmA2, bar, m_blk * kBlockM + 64, ab * 64);
-                        } else {
-                            tma_load_2d(sA, &tmA2, bar, ab * 64, m_blk * kBlockM);
-                        }
-                        tma_load_2d(sB, &tmB2, bar, ab * 64, n_blk * BLOCK_N);
-                    }
-                    ps.advance(STAGES);
-                }
-            }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (elect_one()) {
-            constexpr uint32_t idesc_sp = make_idesc_bf16(kBlockM, BLOCK_N, false, false, true);
-            const uint32_t idesc_ad = make_idesc_bf16(kBlockM, BLOCK_N, p.a2_mn_major != 0, false, false);
-            PipeState ps;
-            bool ok = true;
-            int it = 0;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
-                const int acc = it & 1;
-                const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
-                if (!mbar_wait(&tempty_bar[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
-                tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + acc * BLOCK_N;
-                for (int kb = 0; kb < total_kb; ++kb) {
-                    if (!mbar_wait(&full_bar[ps.stage], ps.phase, abort_flag)) { ok = false; break; }
-                    tc_fence_after_sync();
-                    const uint32_t sA = smem_u32(smem + ps.stage * Cfg::kStageBytes);
-                    const uint32_t sB = sA + Cfg::kABytes;
-                    const uint32_t sE = sB + Cfg::kBBytes;
-                    if (kb < num_kb) {
-                        const uint32_t e_tmem = tmem_base + Cfg::kECol + (kb & 1) * 4;
-                        tmem_cp_128x128b(e_tmem, make_smem_desc(sE, 128, 128, kSwizzleNone));
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint64_t ad = make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
-                            const uint64_t bd =
-                                make_smem_desc(sB + (j >> 1) * (BLOCK_N * 128) + (j & 1) * 64, 16, 1024, kSwizzle128B);
-                            umma_bf16_sp(d_tmem, ad, bd, e_tmem + (j & 2), idesc_sp | (j & 1), (kb | j) != 0 ? 1u : 0u);
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint64_t ad = p.a2_mn_major
-                                                    ? make_smem_desc(sA + j * 2048, 8192, 1024, kSwizzle128B)
-                                                    : make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
-                            const uint64_t bd = make_smem_desc(sB + j * 32, 16, 1024, kSwizzle128B);
-                            umma_bf16(d_tmem, ad, bd, idesc_ad, 1u);
-                        }
-                    }
-                    umma_commit(&empty_bar[ps.stage]);
-                    ps.advance(STAGES);
-                }
-                if (ok) umma_commit(&tfull_bar[acc]);
-            }
-        }
-    } else {
-        // ------------------------------------------------------------ epilogue (warps 2..5)
-        const int q = warp & 3;                       // tensor-memory lane quadrant of this warp
-        bool ok = true;
-        int it = 0;
-        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
-            const int m_blk = tile % num_m, n_blk = tile / num_m;
-            const int acc = it & 1;
-            const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
-            if (!mbar_wait(&tfull_bar[acc], acc_phase, abort_flag)) { ok = false; break; }
-            tc_fence_after_sync();
-            const uint32_t t_row = tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
-            const int m = m_blk * kBlockM + q * 32 + lane;
-            uint16_t* out_col = p.out + m;
-#pragma unroll 1
-            for (int c0 = 0; c0 < BLOCK_N; c0 += 16) {
-                uint32_t v[16];
-                tmem_ld_16(t_row + c0, v);
-                tmem_ld_wait();
-                const int n0 = n_blk * BLOCK_N + c0;
-#pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    const int n = n0 + c;
-                    if (n < p.Ntok) out_col[static_cast<size_t>(n) * p.M] = to_bf16(__uint_as_float(v[c]));
-                }
-            }
-            tc_fence_before_sync();
-            mbar_arrive(&tempty_bar[acc]);
-        }
-    }
-
-    __syncwarp();
-    if (*abort_flag) drain_after_abort();
-    tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after_sync();
-        tmem_dealloc(tmem_base, 512);
-    }
-}
-
 // =====================================================================================
 // Dense GEMM:  D[M x N] = A[M x K] * B[N x K]^T, bf16 in, fp32 accumulate.
 //   A_MN / B_MN: the operand is stored with its M (resp. N) index contiguous, i.e. as
@@ -535,7 +361,7 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                         tma_load_2d_pair(sA, &tmA, bar, kb * 64, mb * kBlockM);
                         tma_load_2d_pair(sB, &tmB, bar, kb * 128, n_row0);
                         tma_load_2d_pair(sB + Cfg::kHalfN * 128, &tmB, bar, kb * 128 + 64, n_row0);
-                        tma_load_2d_pair(sE, &tmE, bar, 0, (mb_e * num_kb + kb) * 128);
+                        tma_load_2d_pair(sE, &tmE, bar, 0, mb_e * num_kb + kb);
                     } else {
                         const int ab = kb - num_kb;
                         if (cta == 0) mbar_expect_tx(&full_bar[ps.stage], 2 * (Cfg::kABytes + Cfg::kHalfN * 128));
@@ -816,6 +642,296 @@ dense_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     if (warp == 1) {
         tc_fence_after_sync();
         tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+}
+
+// =====================================================================================
+// Sparse CTA-pair GEMM with a 512-row tile: the pair runs TWO 256-row MMA sub-tiles against
+// ONE staged activation tile, so every activation byte pulled from L2 feeds twice as many
+// MMAs (L2 -> SM bytes per FLOP drop by 31 % against the 256-row tile; that fabric, not DRAM
+// or the tensor pipe, is what bounds these GEMMs).  Tensor memory then holds one accumulator
+// per sub-tile (2 x BLOCK_N columns) plus the metadata columns, so accumulators are single
+// buffered; the epilogue is made short instead: accumulator rows are transposed through
+// shared memory and leave as TMA stores of 32 tokens x 128 features.
+//   128-row block of A handled by CTA c for sub-tile s of tile mt:  4*mt + 2*s + c.
+// =====================================================================================
+constexpr int kPrefetchAhead = 8;          // k-blocks of L2 prefetch distance for activation boxes
+
+template <int BLOCK_N, int STAGES>
+struct SparseQuadCfg {
+    static constexpr int kHalfN = BLOCK_N / 2;
+    static constexpr int kABytes = kBlockM * 128;                 // per sub-tile
+    static constexpr int kBBytes = kHalfN * 256;
+    static constexpr int kEBytes = 2048;                          // per sub-tile
+    static constexpr int kOffB = 2 * kABytes;
+    static constexpr int kOffE = kOffB + kBBytes;
+    static constexpr int kStageBytes = kOffE + 2 * kEBytes;
+    static constexpr int kStoreRows = 32;                         // tokens per TMA store
+    static constexpr int kStoreCols = 32;                         // features per TMA store (one warp's lanes)
+    static constexpr int kStoreBytes = kStoreRows * kStoreCols * 2;   // 2 KB staging buffer
+    static constexpr int kEpiWarps = 8;                           // two warps per tensor-memory lane quadrant
+    static constexpr int kThreads = 64 + 32 * kEpiWarps;
+    static constexpr int kOffStore = STAGES * kStageBytes;
+    static constexpr int kOffBar = kOffStore + kEpiWarps * 2 * kStoreBytes;
+    static constexpr int kSmemBytes = kOffBar + 256 + 1024;
+    static constexpr int kECol = 2 * BLOCK_N;
+    static_assert(BLOCK_N % 32 == 0 && kHalfN % 8 == 0 && 2 * BLOCK_N + 16 <= 512, "tile does not fit tensor memory");
+    static_assert(kBBytes % 2048 == 0 && kStageBytes % 1024 == 0, "stage must keep 1024-byte alignment");
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
+};
+
+template <int BLOCK_N, int STAGES>
+__global__ void __launch_bounds__(SparseQuadCfg<BLOCK_N, STAGES>::kThreads, 1)
+sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                        const __grid_constant__ CUtensorMap tmE, const __grid_constant__ CUtensorMap tmA2,
+                        const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmO,
+                        const SparseGemmParams p) {
+    using Cfg = SparseQuadCfg<BLOCK_N, STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBar);
+    uint64_t* empty_bar = full_bar + STAGES;
+    uint64_t* tfull_bar = empty_bar + STAGES;                // [1]
+    uint64_t* tempty_bar = tfull_bar + 1;                    // [2], one per sub-tile accumulator
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cta = cluster_ctarank();
+    const int pair_id = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int num_mb = p.M / kBlockM;
+    const int num_m = (num_mb + 3) / 4;                      // 512-row tiles
+    const int num_n = (p.Ntok + BLOCK_N - 1) / BLOCK_N;
+    const int num_tiles = num_m * num_n;
+    const int num_kb = p.K / 128;
+    const int num_ab = (p.r + 63) / 64;
+    const int total_kb = num_kb + num_ab;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        mbar_init(&tfull_bar[0], 1);
+        mbar_init(&tempty_bar[0], 2 * Cfg::kEpiWarps);
+        mbar_init(&tempty_bar[1], 2 * Cfg::kEpiWarps);
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(tmem_slot, 512);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (both CTAs)
+        if (elect_one()) {
+            tma_prefetch_desc(&tmA);
+            tma_prefetch_desc(&tmB);
+            tma_prefetch_desc(&tmE);
+            PipeState ps;
+            bool ok = true;
+            for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
+                const int mt = tile % num_m, n_blk = tile / num_m;
+                const int nsub = (4 * mt + 2 < num_mb) ? 2 : 1;              // second sub-tile may lie past M
+                const int n_row0 = n_blk * BLOCK_N + static_cast<int>(cta) * Cfg::kHalfN;
+                // The pairs working on the same token block (same n_blk, different mt) run side by
+                // side and would all wait on the same first-touch DRAM fetch of an activation box.
+                // One of them (mt == 0) pulls the boxes into L2 kPrefetchAhead k-blocks early.
+                const int next_tile = tile + num_pairs;
+                const int next_row0 = (next_tile / num_m) * BLOCK_N + static_cast<int>(cta) * Cfg::kHalfN;
+                for (int kb = 0; kb < total_kb; ++kb) {
+                    if (kb < num_kb) {
+                        const int pk = kb + kPrefetchAhead;
+                        if (pk < num_kb) {
+                            if (mt == 0) {
+                                tma_prefetch_l2_2d(&tmB, pk * 128, n_row0);
+                                tma_prefetch_l2_2d(&tmB, pk * 128 + 64, n_row0);
+                            }
+                        } else if (next_tile < num_tiles && next_tile % num_m == 0 && pk - num_kb < num_kb) {
+                            tma_prefetch_l2_2d(&tmB, (pk - num_kb) * 128, next_row0);
+                            tma_prefetch_l2_2d(&tmB, (pk - num_kb) * 128 + 64, next_row0);
+                        }
+                    }
+                    if (!mbar_wait(&empty_bar[ps.stage], ps.phase ^ 1u, abort_flag)) { ok = false; break; }
+                    uint8_t* st = smem + ps.stage * Cfg::kStageBytes;
+                    uint8_t* sB = st + Cfg::kOffB;
+                    const uint32_t bar = mapa_shared(smem_u32(&full_bar[ps.stage]), 0);
+                    if (kb < num_kb) {
+                        if (cta == 0)
+                            mbar_expect_tx(&full_bar[ps.stage],
+                                           2 * (Cfg::kBBytes + nsub * (Cfg::kABytes + Cfg::kEBytes)));
+                        tma_load_2d_pair(sB, &tmB, bar, kb * 128, n_row0);
+                        tma_load_2d_pair(sB + Cfg::kHalfN * 128, &tmB, bar, kb * 128 + 64, n_row0);
+                        for (int s = 0; s < nsub; ++s) {
+                            const int mb = 4 * mt + 2 * s + static_cast<int>(cta);
+                            const int mb_e = mb < num_mb ? mb : num_mb - 1;
+                            tma_load_2d_pair(st + s * Cfg::kABytes, &tmA, bar, kb * 64, mb * kBlockM);
+                            tma_load_2d_pair(st + Cfg::kOffE + s * Cfg::kEBytes, &tmE, bar, 0, mb_e * num_kb + kb);
+                        }
+                    } else {
+                        const int ab = kb - num_kb;
+                        if (cta == 0)
+                            mbar_expect_tx(&full_bar[ps.stage], 2 * (Cfg::kHalfN * 128 + nsub * Cfg::kABytes));
+                        tma_load_2d_pair(sB, &tmB2, bar, ab * 64, n_row0);
+                        for (int s = 0; s < nsub; ++s) {
+                            const int m0 = (4 * mt + 2 * s + static_cast<int>(cta)) * kBlockM;
+                            uint8_t* sA = st + s * Cfg::kABytes;
+                            if (p.a2_mn_major) {
+                                tma_load_2d_pair(sA, &tmA2, bar, m0, ab * 64);
+                                tma_load_2d_pair(sA + 8192, &tmA2, bar, m0 + 64, ab * 64);
+                            } else {
+                                tma_load_2d_pair(sA, &tmA2, bar, ab * 64, m0);
+                            }
+                        }
+                    }
+                    ps.advance(STAGES);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (cta == 0 && elect_one()) {
+            constexpr uint32_t idesc_sp = make_idesc_bf16(2 * kBlockM, BLOCK_N, false, false, true);
+            const uint32_t idesc_ad = make_idesc_bf16(2 * kBlockM, BLOCK_N, p.a2_mn_major != 0, false, false);
+            PipeState ps;
+            bool ok = true;
+            int it = 0;
+            for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
+                const int mt = tile % num_m;
+                const int nsub = (4 * mt + 2 < num_mb) ? 2 : 1;
+                const uint32_t acc_phase = static_cast<uint32_t>(it) & 1u;
+                for (int kb = 0; ok && kb < total_kb; ++kb) {
+                    if (!mbar_wait(&full_bar[ps.stage], ps.phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t st = smem_u32(smem + ps.stage * Cfg::kStageBytes);
+                    const uint32_t sB = st + Cfg::kOffB;
+                    for (int s = 0; s < nsub; ++s) {
+                        if (kb == 0) {                        // accumulator s must have been drained
+                            if (!mbar_wait(&tempty_bar[s], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                            tc_fence_after_sync();
+                        }
+                        const uint32_t d_tmem = tmem_base + s * BLOCK_N;
+                        const uint32_t sA = st + s * Cfg::kABytes;
+                        if (kb < num_kb) {
+                            const uint32_t e_tmem = tmem_base + Cfg::kECol + (kb & 1) * 8 + s * 4;
+                            tmem_cp_128x128b_pair(e_tmem, make_smem_desc(st + Cfg::kOffE + s * Cfg::kEBytes, 128, 128,
+                                                                         kSwizzleNone));
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const uint64_t ad = make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
+                                const uint64_t bd = make_smem_desc(sB + (j >> 1) * (Cfg::kHalfN * 128) + (j & 1) * 64,
+                                                                   16, 1024, kSwizzle128B);
+                                umma_bf16_sp_pair(d_tmem, ad, bd, e_tmem + (j & 2), idesc_sp | (j & 1),
+                                                  (kb | j) != 0 ? 1u : 0u);
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const uint64_t ad = p.a2_mn_major
+                                                        ? make_smem_desc(sA + j * 2048, 8192, 1024, kSwizzle128B)
+                                                        : make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
+                                const uint64_t bd = make_smem_desc(sB + j * 32, 16, 1024, kSwizzle128B);
+                                umma_bf16_pair(d_tmem, ad, bd, idesc_ad, 1u);
+                            }
+                        }
+                    }
+                    if (!ok) break;
+                    umma_commit_pair(&empty_bar[ps.stage], 3);
+                    ps.advance(STAGES);
+                }
+                if (ok) umma_commit_pair(&tfull_bar[0], 3);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+        // Warp w drains lane quadrant w%4; the two warps of a quadrant take alternate 32-token
+        // blocks.  Phase 1 empties both accumulators into registers (packed bf16) and hands them
+        // back to the MMA issuer at once -- the accumulators are single buffered, so this is
+        // what the next tile waits for.  Phase 2 runs under the next tile's main loop: each warp
+        // transposes its 32 x 32 blocks through a private staging buffer and sends them with its
+        // own TMA stores; the warps never wait for one another.
+        constexpr int kBlocks = BLOCK_N / Cfg::kStoreRows;        // 32-token blocks per accumulator
+        constexpr int kMyBlocks = (kBlocks + 1) / 2;              // at most this many per warp
+        const int q = warp & 3;
+        const int ew = warp - 2;
+        const int half = ew >> 2;
+        uint8_t* my_buf = smem + Cfg::kOffStore + ew * 2 * Cfg::kStoreBytes;
+        bool ok = true;
+        int it = 0;
+        uint32_t buf = 0;
+        for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
+            const int mt = tile % num_m, n_blk = tile / num_m;
+            const int nsub = (4 * mt + 2 < num_mb) ? 2 : 1;
+            if (!mbar_wait(&tfull_bar[0], static_cast<uint32_t>(it) & 1u, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            uint32_t pk[2][kMyBlocks][16];
+#pragma unroll
+            for (int s = 0; s < 2; ++s) {
+                if (s < nsub) {
+                    const uint32_t t_row = tmem_base + s * BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
+#pragma unroll
+                    for (int j = 0; j < kMyBlocks; ++j) {
+                        const int c0 = (2 * j + half) * Cfg::kStoreRows;
+                        if (c0 < BLOCK_N) {
+                            uint32_t v0[16], v1[16];
+                            tmem_ld_16(t_row + c0, v0);
+                            tmem_ld_16(t_row + c0 + 16, v1);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                pk[s][j][i] = pack_bf16x2(__uint_as_float(v0[2 * i]), __uint_as_float(v0[2 * i + 1]));
+                                pk[s][j][8 + i] = pack_bf16x2(__uint_as_float(v1[2 * i]), __uint_as_float(v1[2 * i + 1]));
+                            }
+                        }
+                    }
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&tempty_bar[s]), 0));
+            }
+#pragma unroll
+            for (int s = 0; s < 2; ++s) {
+                if (s < nsub) {
+                    const int m0 = (4 * mt + 2 * s + static_cast<int>(cta)) * kBlockM + q * 32;
+#pragma unroll
+                    for (int j = 0; j < kMyBlocks; ++j) {
+                        const int c0 = (2 * j + half) * Cfg::kStoreRows;
+                        if (c0 < BLOCK_N) {
+                            // the staging buffer about to be overwritten must have been read by its TMA store
+                            if (lane == 0) tma_store_wait_read<1>();
+                            __syncwarp();
+                            uint16_t* sbuf = reinterpret_cast<uint16_t*>(my_buf + buf * Cfg::kStoreBytes) + lane;
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                sbuf[(2 * i) * Cfg::kStoreCols] = static_cast<uint16_t>(pk[s][j][i] & 0xFFFFu);
+                                sbuf[(2 * i + 1) * Cfg::kStoreCols] = static_cast<uint16_t>(pk[s][j][i] >> 16);
+                            }
+                            fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0 && m0 < p.M) {
+                                tma_store_2d(&tmO, my_buf + buf * Cfg::kStoreBytes, m0, n_blk * BLOCK_N + c0);
+                                tma_store_commit();
+                            }
+                            buf ^= 1u;
+                        }
+                    }
+                }
+            }
+        }
+        if (lane == 0) tma_store_wait_all<0>();
+    }
+
+    __syncwarp();
+    if (*abort_flag) drain_after_abort();
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, 512);
     }
 }
 

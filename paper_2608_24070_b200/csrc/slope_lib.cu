@@ -69,26 +69,40 @@ static bool make_tmap(CUtensorMap* tm, const void* base, int rows, int cols, int
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Metadata as a 2-D byte tensor [bytes/16 x 16]: one 2 KB block = a 16 x 128 box, no swizzle.
+// Metadata as a 2-D tensor of 8-byte words [blocks x 256]: one 2 KB block is ONE contiguous row,
+// so a block costs the TMA unit a single request (a 128 x 16-byte box costs 128).
 static bool make_tmap_meta(CUtensorMap* tm, const void* base, size_t total_bytes) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
-    const cuuint64_t gdim[2] = {16, static_cast<cuuint64_t>(total_bytes / 16)};
-    const cuuint64_t gstride[1] = {16};
-    const cuuint32_t box[2] = {16, 128};
+    const cuuint64_t gdim[2] = {256, static_cast<cuuint64_t>(total_bytes / 2048)};
+    const cuuint64_t gstride[1] = {2048};
+    const cuuint32_t box[2] = {256, 1};
     const cuuint32_t estr[2] = {1, 1};
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(base), gdim, gstride, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Plain (unswizzled) 2-D bf16 tensor map, used for TMA stores of output tiles.
+static bool make_tmap_plain(CUtensorMap* tm, const void* base, int rows, int cols, int box_rows, int box_cols) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(cols) * 2};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // Launch on clusters of two CTAs (cta_group::2 kernels).
 template <typename... KArgs, typename... Args>
-static slope_status_t launch_pairs(void (*kern)(KArgs...), int grid, int smem_bytes, cudaStream_t stream,
-                                   Args&&... args) {
+static slope_status_t launch_pairs(void (*kern)(KArgs...), int grid, int threads, int smem_bytes,
+                                   cudaStream_t stream, Args&&... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid, 1, 1);
-    cfg.blockDim = dim3(kGemmThreads, 1, 1);
+    cfg.blockDim = dim3(threads, 1, 1);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr;
@@ -120,40 +134,6 @@ static slope_status_t launch_result() {
 template <typename Kernel>
 static bool set_smem(Kernel k, int bytes) {
     return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
-}
-
-// ------------------------------------------------------------------ sparse GEMM launch
-constexpr int kSpBlockN = 240;
-constexpr int kSpStages = 2;
-
-static slope_status_t launch_sparse(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
-                                    const void* act2, const void* fac2, int r, bool a2_mn, void* out,
-                                    cudaStream_t stream, const DeviceInfo& info) {
-    using Cfg = SparseCfg<kSpBlockN, kSpStages>;
-    CUtensorMap tmA, tmB, tmA2, tmB2;
-    if (!make_tmap(&tmA, vals, M, K / 2, kBlockM, 64)) return SLOPE_ERR_CUDA;
-    if (!make_tmap(&tmB, act, ntok, K, kSpBlockN, 64)) return SLOPE_ERR_CUDA;
-    if (r > 0) {
-        const bool ok2 = a2_mn ? make_tmap(&tmA2, fac2, r, M, 64, 64) : make_tmap(&tmA2, fac2, M, r, kBlockM, 64);
-        if (!ok2 || !make_tmap(&tmB2, act2, ntok, r, kSpBlockN, 64)) return SLOPE_ERR_CUDA;
-    } else {
-        tmA2 = tmA;
-        tmB2 = tmB;
-    }
-    SparseGemmParams p;
-    p.M = M; p.K = K; p.Ntok = ntok; p.r = r; p.a2_mn_major = a2_mn ? 1 : 0;
-    p.meta = static_cast<const uint8_t*>(meta);
-    p.out = static_cast<uint16_t*>(out);
-    auto kern = sparse_gemm_kernel<kSpBlockN, kSpStages>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
-        attr_set = true;
-    }
-    const int tiles = (M / kBlockM) * ((ntok + kSpBlockN - 1) / kSpBlockN);
-    const int grid = tiles < info.sm_count ? tiles : info.sm_count;
-    kern<<<grid, kGemmThreads, Cfg::kSmemBytes, stream>>>(tmA, tmB, tmA2, tmB2, p);
-    return launch_result();
 }
 
 // ------------------------------------------------------------------ dense GEMM launch
@@ -212,7 +192,53 @@ static slope_status_t launch_sparse_pair(const void* act, int ntok, const void* 
     const int tiles = ((M / kBlockM + 1) / 2) * ((ntok + kPairBlockN - 1) / kPairBlockN);
     const int max_pairs = info.sm_count / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
-    return launch_pairs(kern, 2 * pairs, Cfg::kSmemBytes, stream, tmA, tmB, tmE, tmA2, tmB2, p);
+    return launch_pairs(kern, 2 * pairs, kGemmThreads, Cfg::kSmemBytes, stream, tmA, tmB, tmE, tmA2, tmB2, p);
+}
+
+constexpr int kQuadBlockN = 224;
+constexpr int kQuadStages = 3;
+
+static slope_status_t launch_sparse_quad(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
+                                         const void* act2, const void* fac2, int r, bool a2_mn, void* out,
+                                         cudaStream_t stream, const DeviceInfo& info) {
+    using Cfg = SparseQuadCfg<kQuadBlockN, kQuadStages>;
+    CUtensorMap tmA, tmB, tmE, tmA2, tmB2, tmO;
+    if (!make_tmap(&tmA, vals, M, K / 2, kBlockM, 64)) return SLOPE_ERR_CUDA;
+    if (!make_tmap(&tmB, act, ntok, K, Cfg::kHalfN, 64)) return SLOPE_ERR_CUDA;
+    if (!make_tmap_meta(&tmE, meta, static_cast<size_t>(M) * K / 8)) return SLOPE_ERR_CUDA;
+    if (!make_tmap_plain(&tmO, out, ntok, M, Cfg::kStoreRows, Cfg::kStoreCols)) return SLOPE_ERR_CUDA;
+    if (r > 0) {
+        const bool ok2 = a2_mn ? make_tmap(&tmA2, fac2, r, M, 64, 64) : make_tmap(&tmA2, fac2, M, r, kBlockM, 64);
+        if (!ok2 || !make_tmap(&tmB2, act2, ntok, r, Cfg::kHalfN, 64)) return SLOPE_ERR_CUDA;
+    } else {
+        tmA2 = tmA;
+        tmB2 = tmB;
+    }
+    SparseGemmParams p;
+    p.M = M; p.K = K; p.Ntok = ntok; p.r = r; p.a2_mn_major = a2_mn ? 1 : 0;
+    p.meta = static_cast<const uint8_t*>(meta);
+    p.out = static_cast<uint16_t*>(out);
+    auto kern = sparse_gemm_quad_kernel<kQuadBlockN, kQuadStages>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
+        attr_set = true;
+    }
+    const int tiles = ((M / kBlockM + 3) / 4) * ((ntok + kQuadBlockN - 1) / kQuadBlockN);
+    const int max_pairs = info.sm_count / 2;
+    const int pairs = tiles < max_pairs ? tiles : max_pairs;
+    return launch_pairs(kern, 2 * pairs, Cfg::kThreads, Cfg::kSmemBytes, stream, tmA, tmB, tmE, tmA2, tmB2, tmO, p);
+}
+
+// Tile choice for the sparse GEMMs.  The 512-row tile moves 31 % fewer L2 bytes per FLOP but
+// cannot overlap its epilogue with the next tile (tensor memory holds only one accumulator
+// set); that pays off once the reduction is long.  Short reductions keep the 256-row tile
+// with double-buffered accumulators.
+static slope_status_t launch_sparse_gemm(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
+                                         const void* act2, const void* fac2, int r, bool a2_mn, void* out,
+                                         cudaStream_t stream, const DeviceInfo& info) {
+    return K >= 6144 ? launch_sparse_quad(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info)
+                     : launch_sparse_pair(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
 }
 
 template <bool A_MN, bool B_MN, int BLOCK_N, int EPI, int STAGES>
@@ -235,7 +261,7 @@ static slope_status_t launch_dense_pair(const void* A, const void* B, int M, int
     const int tiles = ((M + 2 * kBlockM - 1) / (2 * kBlockM)) * ((N + BLOCK_N - 1) / BLOCK_N);
     const int max_pairs = info.sm_count / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
-    return launch_pairs(kern, 2 * pairs, Cfg::kSmemBytes, stream, tmA, tmB, p);
+    return launch_pairs(kern, 2 * pairs, kGemmThreads, Cfg::kSmemBytes, stream, tmA, tmB, p);
 }
 
 static int adapter_splits(int b, int rows) {
@@ -338,7 +364,7 @@ slope_status_t slope_linear_fwd(const void* X, int b, const void* Wc_vals, const
         return SLOPE_ERR_ALIGNMENT;
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
-    return launch_sparse_pair(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R, r, /*a2_mn=*/true, Y,
+    return launch_sparse_gemm(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R, r, /*a2_mn=*/true, Y,
                               static_cast<cudaStream_t>(stream), info);
 }
 
@@ -352,7 +378,7 @@ slope_status_t slope_linear_bwd_dx(const void* dY, int b, const void* WTc_vals, 
         return SLOPE_ERR_ALIGNMENT;
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
-    return launch_sparse_pair(dY, b, WTc_vals, WTc_meta, d_in, d_out, dT, L, r, /*a2_mn=*/false, dX,
+    return launch_sparse_gemm(dY, b, WTc_vals, WTc_meta, d_in, d_out, dT, L, r, /*a2_mn=*/false, dX,
                               static_cast<cudaStream_t>(stream), info);
 }
 

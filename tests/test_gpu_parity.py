@@ -53,24 +53,27 @@ def test_prune_ties_zeros_and_specials(B, oracle):
 def _nibble_pattern_weight(d_out, d_in, seed):
     """Integer-valued weights whose kept pair cycles through all six patterns."""
     rng = np.random.Generator(np.random.PCG64(seed))
-    pats = [(0, 1), (0, 2), (0, 3), (1, 2), (1, 3), (2, 3)]
-    Wf = np.zeros((d_out, d_in), np.float32)
-    for i in range(d_out):
-        for g in range(d_in // 4):
-            p = pats[(i * 7 + g * 5 + (i // 128) + (g // 32)) % 6]
-            small = rng.integers(1, 4, size=4).astype(np.float32) * rng.choice([-1, 1], size=4)
-            big = rng.integers(8, 64, size=2).astype(np.float32) * rng.choice([-1, 1], size=2)
-            grp = small.copy()
-            grp[p[0]], grp[p[1]] = big[0], big[1]
-            Wf[i, 4 * g:4 * g + 4] = grp
-    return si.f32_to_bf16_bits(Wf)
+    pats = np.array([(0, 1), (0, 2), (0, 3), (1, 2), (1, 3), (2, 3)])
+    groups = d_in // 4
+    i = np.arange(d_out)[:, None]
+    g = np.arange(groups)[None, :]
+    which = (i * 7 + g * 5 + (i // 128) + (g // 32)) % 6
+    sign = lambda shape: rng.choice(np.array([-1.0, 1.0], np.float32), size=shape)
+    Wf = (rng.integers(1, 4, size=(d_out, groups, 4)).astype(np.float32) * sign((d_out, groups, 4)))
+    big = rng.integers(8, 64, size=(d_out, groups, 2)).astype(np.float32) * sign((d_out, groups, 2))
+    ii, gg = np.meshgrid(np.arange(d_out), np.arange(groups), indexing="ij")
+    Wf[ii, gg, pats[which][..., 0]] = big[..., 0]
+    Wf[ii, gg, pats[which][..., 1]] = big[..., 1]
+    return si.f32_to_bf16_bits(Wf.reshape(d_out, d_in))
 
 
-def test_identity_activations_return_the_pruned_weight_exactly(B, oracle):
-    """X = I  =>  Y = (W^R)^T bit for bit;  dY = I  =>  dX = W^{R,C};  dY = I  =>  dWc = gather(X)."""
+@pytest.mark.parametrize("d_out,d_in", [(256, 384), (640, 6144), (6144, 640)])
+def test_identity_activations_return_the_pruned_weight_exactly(B, oracle, d_out, d_in):
+    """X = I  =>  Y = (W^R)^T bit for bit;  dY = I  =>  dX = W^{R,C};  dY = I  =>  dWc = gather(X).
+    The long dimensions reach the 512-row-tile kernel (reduction >= 6144), the short ones the
+    256-row-tile kernel, both with partial last tiles."""
     import torch
 
-    d_out, d_in = 256, 384
     W = _nibble_pattern_weight(d_out, d_in, 6)
     layer = GpuLayer(W)
     mask1, mask2 = check_selection(oracle, layer, W)
@@ -101,6 +104,8 @@ CASES = [
     (384, 640, 776, 32, 13),         # ragged token tail, several tiles in every dimension
     (768, 256, 1000, 128, 14),
     (128, 128, 8, 16, 15),           # smallest legal problem
+    (6144, 640, 264, 32, 16),        # forward reduction long enough for the 512-row-tile kernel
+    (640, 6144, 264, 0, 17),         # same for the input-gradient GEMM
 ]
 
 
