@@ -343,6 +343,7 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             tma_prefetch_desc(&tmA);
             tma_prefetch_desc(&tmB);
             tma_prefetch_desc(&tmE);
+            const uint64_t keep = l2_policy_evict_last();
             PipeState ps;
             bool ok = true;
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
@@ -358,10 +359,10 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     const uint32_t bar = mapa_shared(smem_u32(&full_bar[ps.stage]), 0);
                     if (kb < num_kb) {
                         if (cta == 0) mbar_expect_tx(&full_bar[ps.stage], 2 * Cfg::kStageBytes);
-                        tma_load_2d_pair(sA, &tmA, bar, kb * 64, mb * kBlockM);
+                        tma_load_2d_pair_hint(sA, &tmA, bar, kb * 64, mb * kBlockM, keep);
                         tma_load_2d_pair(sB, &tmB, bar, kb * 128, n_row0);
                         tma_load_2d_pair(sB + Cfg::kHalfN * 128, &tmB, bar, kb * 128 + 64, n_row0);
-                        tma_load_2d_pair(sE, &tmE, bar, 0, mb_e * num_kb + kb);
+                        tma_load_2d_pair_hint(sE, &tmE, bar, 0, mb_e * num_kb + kb, keep);
                     } else {
                         const int ab = kb - num_kb;
                         if (cta == 0) mbar_expect_tx(&full_bar[ps.stage], 2 * (Cfg::kABytes + Cfg::kHalfN * 128));
@@ -426,6 +427,7 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+        const uint64_t stream_out = l2_policy_evict_first();
         const int q = warp & 3;
         bool ok = true;
         int it = 0;
@@ -448,7 +450,9 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 #pragma unroll
                     for (int c = 0; c < 16; ++c) {
                         const int n = n0 + c;
-                        if (n < p.Ntok) out_col[static_cast<size_t>(n) * p.M] = to_bf16(__uint_as_float(v[c]));
+                        if (n < p.Ntok)
+                            st_global_evict_first_u16(out_col + static_cast<size_t>(n) * p.M,
+                                                      to_bf16(__uint_as_float(v[c])), stream_out);
                     }
                 }
             }
@@ -467,6 +471,21 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         tc_fence_after_sync();
         tmem_dealloc_pair(tmem_base, 512);
     }
+}
+
+// Tile order for GEMMs whose two operands are both streamed once per tile (dW: dY^T X with the
+// tokens as reduction).  The ~74 tiles in flight should form a near-square patch of the output:
+// a patch of gm x gn tiles reads (gm + gn) operand panels, a gm x 1 strip reads gm + 1 for 1/gn
+// of the work.  Tiles are numbered in groups of kRasterGroupM tile rows, column by column.
+constexpr int kRasterGroupM = 8;
+__device__ __forceinline__ void raster_tile(int tile, int num_m, int num_n, int& m, int& n) {
+    const int group_size = kRasterGroupM * num_n;
+    const int g = tile / group_size;
+    const int first_m = g * kRasterGroupM;
+    const int gm = min(num_m - first_m, kRasterGroupM);
+    const int local = tile - g * group_size;
+    m = first_m + local % gm;
+    n = local / gm;
 }
 
 // Dense CTA-pair GEMM: D[M x N] = A[M x K] * B[N x K]^T with a 256 x BLOCK_N tile per pair
@@ -527,7 +546,8 @@ dense_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
             PipeState ps;
             bool ok = true;
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
-                const int m_pair = tile % num_m, n_blk = tile / num_m;
+                int m_pair, n_blk;
+                raster_tile(tile, num_m, num_n, m_pair, n_blk);
                 const int m0 = (m_pair * 2 + static_cast<int>(cta)) * kBlockM;
                 const int n0 = n_blk * BLOCK_N + static_cast<int>(cta) * Cfg::kHalfN;
                 for (int kb = 0; kb < num_kb; ++kb) {
@@ -589,7 +609,8 @@ dense_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         bool ok = true;
         int it = 0;
         for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
-            const int m_pair = tile % num_m, n_blk = tile / num_m;
+            int m_pair, n_blk;
+            raster_tile(tile, num_m, num_n, m_pair, n_blk);
             const int acc = it & 1;
             const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
             if (!mbar_wait(&tfull_bar[acc], acc_phase, abort_flag)) { ok = false; break; }
@@ -731,6 +752,7 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             tma_prefetch_desc(&tmA);
             tma_prefetch_desc(&tmB);
             tma_prefetch_desc(&tmE);
+            const uint64_t keep = l2_policy_evict_last();
             PipeState ps;
             bool ok = true;
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
@@ -768,8 +790,9 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                         for (int s = 0; s < nsub; ++s) {
                             const int mb = 4 * mt + 2 * s + static_cast<int>(cta);
                             const int mb_e = mb < num_mb ? mb : num_mb - 1;
-                            tma_load_2d_pair(st + s * Cfg::kABytes, &tmA, bar, kb * 64, mb * kBlockM);
-                            tma_load_2d_pair(st + Cfg::kOffE + s * Cfg::kEBytes, &tmE, bar, 0, mb_e * num_kb + kb);
+                            tma_load_2d_pair_hint(st + s * Cfg::kABytes, &tmA, bar, kb * 64, mb * kBlockM, keep);
+                            tma_load_2d_pair_hint(st + Cfg::kOffE + s * Cfg::kEBytes, &tmE, bar, 0, mb_e * num_kb + kb,
+                                                  keep);
                         }
                     } else {
                         const int ab = kb - num_kb;
@@ -859,6 +882,7 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         const int ew = warp - 2;
         const int half = ew >> 2;
         uint8_t* my_buf = smem + Cfg::kOffStore + ew * 2 * Cfg::kStoreBytes;
+        const uint64_t stream_out = l2_policy_evict_first();
         bool ok = true;
         int it = 0;
         uint32_t buf = 0;
@@ -912,7 +936,8 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                             fence_proxy_async_smem();
                             __syncwarp();
                             if (lane == 0 && m0 < p.M) {
-                                tma_store_2d(&tmO, my_buf + buf * Cfg::kStoreBytes, m0, n_blk * BLOCK_N + c0);
+                                tma_store_2d_hint(&tmO, my_buf + buf * Cfg::kStoreBytes, m0, n_blk * BLOCK_N + c0,
+                                                  stream_out);
                                 tma_store_commit();
                             }
                             buf ^= 1u;
