@@ -398,6 +398,17 @@ def main():
                        "frac_of_2x_burst_3386": round(sp_tflops / (2.0 * pk["bf16"]), 4),
                        "frac_of_datasheet_4500": round(sp_tflops / 4500.0, 4),
                        "peak_source": f"2 x {pk['src']} sustained dense bf16 (sparse bf16 peak := 2 x dense)"}
+    # dram__bytes_read + write per launch from the 1-pass ncu capture at these sizes
+    # (profiles/dram_traffic_full_size_c3_llama7b.md), averaged over the launches of a step.
+    if wl.key in ("c3_llama7b", "c4_llama7b_adapter") and b == 16384:
+        sp_reads = 4 * (153.2 + 153.3) + 2 * (526.8 + 791.9) + (792.3 + 527.1)
+        sp_writes = 4 * (104.0 + 100.1) + 2 * (340.0 + 145.0) + (145.0 + 339.4)
+        roofline_sparse["traffic"] = round((sp_reads + sp_writes) / 14 * 1e6)
+        roofline_sparse["traffic_note"] = "mean DRAM bytes per launch over the 14 sparse GEMM launches of a step (ncu, no adapter operands)"
+        roofline_sparse["algorithmic_bytes"] = round((4 * 2 * (153.1 + 134.2) + 2 * (184.9 + 360.7 + 411.4 + 134.2) + (411.4 + 134.2 + 184.9 + 360.7)) / 14 * 1e6)
+        dw_traffic = 4 * (630.3 + 14.3) + 2 * (1820.0 + 43.3) + (1540.0 + 43.0)
+        roofline_dense["traffic"] = round(dw_traffic / 7 * 1e6)
+        roofline_dense["algorithmic_bytes"] = round((4 * (270.5 + 16.8) + 3 * (500.5 + 45.1)) / 7 * 1e6)
     sparse_dominant = sp_s >= dw_s
     roofline = roofline_sparse if sparse_dominant else roofline_dense
     roofline_other = roofline_dense if sparse_dominant else roofline_sparse
