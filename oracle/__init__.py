@@ -217,3 +217,26 @@ def adapter_dR_cols(X, L, dY, icols) -> np.ndarray:
     dR = np.empty((r, len(icols)), np.float64)
     _load().slope_oracle_adapter_dR_cols(_p(X), _p(L), _p(dY), b, d_out, d_in, r, _p(icols), len(icols), _p(dR))
     return dR
+
+
+def sparse_add(A_vals, B_vals, beta: float, gamma: float) -> np.ndarray:
+    """O7: beta*A + gamma*B on compressed value arrays of one pattern -> float64, same shape."""
+    A_vals, B_vals = _u16(A_vals), _u16(B_vals)
+    assert A_vals.shape == B_vals.shape
+    out = np.empty(A_vals.shape, np.float64)
+    lib = _load()
+    lib.slope_oracle_sparse_add.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_double, ctypes.c_double,
+                                            ctypes.c_long, ctypes.c_void_p]
+    lib.slope_oracle_sparse_add(_p(A_vals), _p(B_vals), float(beta), float(gamma), A_vals.size, _p(out))
+    return out
+
+
+def update_transposed(Wc_new, mask1, mask2, nibT) -> np.ndarray:
+    """O8: values of the compressed transposed double-pruned copy rebuilt from new forward values."""
+    Wc_new, mask1, mask2, nibT = _u16(Wc_new), _u8(mask1), _u8(mask2), _u8(nibT)
+    d_out, half = Wc_new.shape
+    d_in = half * 2
+    assert mask1.shape == (d_out, d_in // 8) and mask2.shape == mask1.shape and nibT.shape == (d_in, d_out // 4)
+    valsT = np.empty((d_in, d_out // 2), np.uint16)
+    _load().slope_oracle_update_transposed(_p(Wc_new), _p(mask1), _p(mask2), _p(nibT), d_out, d_in, _p(valsT))
+    return valsT

@@ -339,6 +339,42 @@ void slope_oracle_adapter_dR_cols(const uint16_t *X, const uint16_t *L, const ui
     free(T);
 }
 
+/* O7 -- Algorithm 1 "sparseAdd" (supplementary "Sparse matrix addition"): beta*A + gamma*B for
+ * two compressed value arrays sharing one sparsity pattern, e.g. (1/gamma_scale) * dW + alpha * W
+ * for weight decay under gradient scaling.  Element-wise, so the pattern never enters. */
+void slope_oracle_sparse_add(const uint16_t *A, const uint16_t *B, double beta, double gamma,
+                             long count, double *out)
+{
+    for (long e = 0; e < count; ++e) out[e] = beta * bf16_to_double(A[e]) + gamma * bf16_to_double(B[e]);
+}
+
+/* O8 -- Algorithm 1 "updateSparseMatrix" for the transposed copy: after the optimizer wrote new
+ * values Wc_new (same first-pass pattern, [d_out x d_in/2]), rebuild the values of the
+ * compressed (W^{R,C})^T under the static masks.  Slot t of group h of row j of the
+ * transposed copy holds W_new[4h + q_t][j] when that element survived both passes, else +0;
+ * W_new[i][j] sits in Wc_new at the rank of column j among the kept columns of its group. */
+void slope_oracle_update_transposed(const uint16_t *Wc_new, const uint8_t *mask1, const uint8_t *mask2,
+                                    const uint8_t *nibT, int d_out, int d_in, uint16_t *valsT)
+{
+    long mrow = d_in / 8;
+    for (long j = 0; j < d_in; ++j)
+        for (long h = 0; h < d_out / 4; ++h) {
+            int n = nibT[j * (d_out / 4) + h];
+            int q[2] = {n & 3, (n >> 2) & 3};
+            for (int t = 0; t < 2; ++t) {
+                long i = 4 * h + q[t];
+                uint16_t v = 0;
+                if (mask_get(mask2, mrow, i, j)) {
+                    long g = j / 4;
+                    int rank = 0;
+                    for (long c = 4 * g; c < j; ++c) rank += mask_get(mask1, mrow, i, c);
+                    v = Wc_new[i * (d_in / 2) + 2 * g + rank];
+                }
+                valsT[j * (d_out / 2) + 2 * h + t] = v;
+            }
+        }
+}
+
 int slope_oracle_max_threads(void)
 {
 #ifdef _OPENMP

@@ -265,16 +265,20 @@ static slope_status_t launch_dense_pair(const void* A, const void* B, int M, int
 }
 
 static int adapter_splits(int b, int rows) {
-    // enough K-splits that (row tiles x splits) covers the machine, each split >= 512 tokens,
-    // and no split without a k-block (an empty split would leave its accumulator unwritten)
+    // K-splits of the token reduction for the skinny adapter gradients (rows x r outputs).
+    // rounds(s) = ceil(tiles * s / SMs) passes over the machine, each 1/s of a tile long; take
+    // the s that minimises rounds(s) / s (with a small charge per split for the fp32 partials),
+    // keeping at least 4 k-blocks (256 tokens) per split and no split without a k-block.
     const int tiles = (rows + kBlockM - 1) / kBlockM;
-    int s = (148 + tiles - 1) / tiles;
-    const int max_s = b / 512 > 0 ? b / 512 : 1;
-    if (s > max_s) s = max_s;
-    if (s > 16) s = 16;
-    if (s < 1) s = 1;
     const int num_kb = (b + 63) / 64;
-    const int per = (num_kb + s - 1) / s;
+    int best_s = 1;
+    double best_cost = 1e30;
+    for (int s = 1; s <= 16 && s * 4 <= num_kb; ++s) {
+        const int rounds = (tiles * s + 147) / 148;
+        const double cost = static_cast<double>(rounds) / s + 0.004 * s;
+        if (cost < best_cost - 1e-12) { best_cost = cost; best_s = s; }
+    }
+    const int per = (num_kb + best_s - 1) / best_s;
     return (num_kb + per - 1) / per;
 }
 

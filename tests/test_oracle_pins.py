@@ -313,3 +313,37 @@ def test_p8_metadata_layout_spot_values(oracle):
 def test_pack_canonical(oracle):
     nib = np.array([[0x4, 0xD, 0x9, 0xE]], np.uint8)
     assert oracle.pack_canonical(nib).tolist() == [[0xE9D4]]
+
+
+# ----------------------------------------------------------------------------- optimizer tail (Algorithm 1)
+def test_sparse_add_equals_numpy(oracle):
+    A = si.gaussian_bf16((64, 96), 1.0, 41)
+    Bv = si.gaussian_bf16((64, 96), 0.02, 42)
+    beta, gamma = 1.0 / 1024.0, 0.01
+    got = oracle.sparse_add(A, Bv, beta, gamma)
+    assert np.array_equal(got, beta * f64(A) + gamma * f64(Bv))
+    assert np.array_equal(oracle.sparse_add(A, Bv, 1.0, 0.0), f64(A))
+
+
+def test_update_transposed_reproduces_double_prune(oracle):
+    """Feeding the forward copy's own values back must rebuild exactly what the second pruning
+    pass wrote; with the masks held fixed the map is linear in the values (scale by 2, negate)."""
+    W = si.gaussian_bf16((256, 384), 0.02, 43)
+    vals, nib, mask1 = oracle.prune24(W)
+    valsT, nibT, mask2 = oracle.double_prune(W, mask1)
+    assert np.array_equal(oracle.update_transposed(vals, mask1, mask2, nibT), valsT)
+    W2 = bf16(-2.0 * si.bf16_bits_to_f32(W))            # same magnitudes order -> same masks
+    vals2, nib2, mask1b = oracle.prune24(W2)
+    valsT2, nibT2, mask2b = oracle.double_prune(W2, mask1b)
+    assert np.array_equal(mask1b, mask1) and np.array_equal(mask2b, mask2) and np.array_equal(nibT2, nibT)
+    assert np.array_equal(oracle.update_transposed(vals2, mask1, mask2, nibT), valsT2)
+    # entries dropped by the second pass stay +0 whatever the new values are
+    junk = np.full_like(vals, 0x3F80)
+    out = oracle.update_transposed(junk, mask1, mask2, nibT)
+    m2T = oracle.mask_to_bool(mask2, 384).T
+    sel = np.zeros_like(out, bool)
+    for t in range(2):
+        q = (nibT >> (2 * t)) & 3
+        rows = 4 * np.arange(64)[None, :] + q
+        sel[:, t::2] = m2T[np.arange(384)[:, None], rows]
+    assert np.array_equal(out != 0, sel)
