@@ -130,6 +130,28 @@ slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY,
                                      void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Optimizer tail of Algorithm 1 ("sparseAdd", supplementary "Sparse matrix addition"):
+ *   out = beta * A + gamma * B
+ * element-wise on two compressed value arrays [rows x cols/2] bf16 that share one sparsity
+ * pattern, e.g. (1/gamma_scale) * dWc + alpha * Wc for weight decay under gradient scaling.
+ * fp32 arithmetic, one rounding to bf16.  out may alias A or B.
+ */
+slope_status_t slope_sparse_add(const void* A_vals, const void* B_vals, float beta, float gamma,
+                                int rows, int cols, void* out_vals, void* stream);
+
+/*
+ * Optimizer tail of Algorithm 1 ("updateSparseMatrix", supplementary "Update Sparse Matrix").
+ * The optimizer writes the new weights straight into the forward copy's values Wc_vals (the
+ * pattern is static, so that copy needs nothing else); this call refreshes the values of the
+ * transposed double-pruned copy from them: slot t of group h of row j of WTc_vals becomes
+ * W_new[4h + q_t][j] if that element survived both pruning passes, else +0 (q_t from
+ * WTc_meta; existence and position inside Wc_vals from mask1_bits).  Metadata and masks are
+ * not modified.
+ */
+slope_status_t slope_update_sparse_matrix(const void* Wc_vals, const void* mask1_bits, const void* WTc_meta,
+                                          int d_out, int d_in, void* WTc_vals, void* stream);
+
+/*
  * dL[d_in x r] = X[b x d_in]^T dT[b x r] without any allocation, for callers that cannot
  * call cudaMalloc or hand over a workspace (code running inside a host application whose
  * memory pool is closed to it, or in a section where allocation is forbidden).

@@ -28,6 +28,7 @@ EXPORTS = (
     "slope_linear_bwd_dw_masked", "slope_adapter_workspace_bytes", "slope_adapter_fwd_bwd",
     "slope_meta_to_canonical", "slope_poll_status", "slope_launch_count", "slope_status_string",
     "slope_adapter_dl_noalloc", "slope_adapter_dl_noalloc_max_scratch_bytes",
+    "slope_sparse_add", "slope_update_sparse_matrix",
 )
 
 
@@ -62,6 +63,10 @@ def lib() -> ctypes.CDLL:
         L.slope_adapter_dl_noalloc.restype = ci
         L.slope_adapter_dl_noalloc_max_scratch_bytes.restype = sz
         L.slope_adapter_dl_noalloc_max_scratch_bytes.argtypes = []
+        L.slope_sparse_add.argtypes = [vp, vp, ctypes.c_float, ctypes.c_float, ci, ci, vp, vp]
+        L.slope_sparse_add.restype = ci
+        L.slope_update_sparse_matrix.argtypes = [vp, vp, vp, ci, ci, vp, vp]
+        L.slope_update_sparse_matrix.restype = ci
         L.slope_poll_status.argtypes = [vp]
         L.slope_launch_count.restype = ctypes.c_ulonglong
         L.slope_status_string.restype = ctypes.c_char_p
@@ -157,6 +162,18 @@ def slope_adapter_dl_noalloc(X, dT, dL):
 
 def slope_adapter_dl_noalloc_max_scratch_bytes() -> int:
     return int(lib().slope_adapter_dl_noalloc_max_scratch_bytes())
+
+
+def slope_sparse_add(A_vals, B_vals, beta, gamma, out_vals):
+    rows, half = A_vals.shape
+    _check("slope_sparse_add", lib().slope_sparse_add(_ptr(A_vals), _ptr(B_vals), float(beta), float(gamma), rows,
+                                                      half * 2, _ptr(out_vals), _stream()))
+
+
+def slope_update_sparse_matrix(Wc_vals, mask1_bits, WTc_meta, WTc_vals):
+    d_out, half = Wc_vals.shape
+    _check("slope_update_sparse_matrix", lib().slope_update_sparse_matrix(
+        _ptr(Wc_vals), _ptr(mask1_bits), _ptr(WTc_meta), d_out, half * 2, _ptr(WTc_vals), _stream()))
 
 
 def slope_meta_to_canonical(meta_hw, rows, cols, meta_canon):

@@ -194,4 +194,96 @@ __global__ void __launch_bounds__(256) meta_to_canonical_kernel(const uint16_t* 
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Optimizer tail of Algorithm 1.
+// ---------------------------------------------------------------------------------------
+
+// "sparseAdd": out = beta * A + gamma * B on two compressed value arrays with one pattern
+// (fp32 arithmetic, one rounding to bf16).  Pure streaming: 16-byte vectors, grid-stride.
+__global__ void __launch_bounds__(256) sparse_add_kernel(const uint4* __restrict__ A, const uint4* __restrict__ B,
+                                                         float beta, float gamma, size_t n_vec,
+                                                         uint4* __restrict__ out) {
+    for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < n_vec;
+         idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        const uint4 a = __ldg(A + idx), b = __ldg(B + idx);
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+        uint32_t r[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const float a0 = __uint_as_float(aw[t] << 16), a1 = __uint_as_float(aw[t] & 0xFFFF0000u);
+            const float b0 = __uint_as_float(bw[t] << 16), b1 = __uint_as_float(bw[t] & 0xFFFF0000u);
+            r[t] = pack_bf16x2(__fmaf_rn(beta, a0, gamma * b0), __fmaf_rn(beta, a1, gamma * b1));
+        }
+        out[idx] = make_uint4(r[0], r[1], r[2], r[3]);
+    }
+}
+
+// "updateSparseMatrix" for the transposed copy: rebuild the values of the compressed
+// (W^{R,C})^T from new forward values Wc_new under the static masks.  Tile (rb, cb) of W
+// (128 x 128 elements = 128 x 64 compressed values) feeds tile (cb, rb) of the transposed copy:
+// its metadata block says which two rows of every 4-row group were kept by the second pass,
+// the first-pass mask says whether such an element exists at all and at which rank it sits
+// in its row's compressed group.
+constexpr int kUpdWcPitchW = 33;                 // 32-bit words per staged row of 64 bf16 (+1 pad)
+constexpr int kUpdSmemBytes = 128 * kUpdWcPitchW * 4 + 2048 + 2048 + 128 * kDpOutPitch;
+
+__global__ void __launch_bounds__(256) update_transposed_kernel(const uint4* __restrict__ Wc_new,
+                                                                const uint8_t* __restrict__ mask1,
+                                                                const uint4* __restrict__ metaT, int d_out, int d_in,
+                                                                uint4* __restrict__ valsT) {
+    extern __shared__ __align__(16) uint8_t up_smem[];
+    uint32_t* s_wc = reinterpret_cast<uint32_t*>(up_smem);
+    uint8_t* s_m1 = up_smem + 128 * kUpdWcPitchW * 4;
+    uint8_t* s_mt = s_m1 + 2048;
+    uint8_t* s_out = s_mt + 2048;
+
+    const int cb = blockIdx.x, rb = blockIdx.y;
+    const int tid = threadIdx.x;
+    const size_t wc_row_u4 = static_cast<size_t>(d_in) >> 4;        // uint4 per compressed row (d_in/2 bf16)
+#pragma unroll
+    for (int pass = 0; pass < 4; ++pass) {
+        const int rr = pass * 32 + (tid >> 3), seg = tid & 7;
+        const uint4 v = __ldg(Wc_new + (static_cast<size_t>(rb) * 128 + rr) * wc_row_u4 + cb * 8 + seg);
+        uint32_t* dst = s_wc + rr * kUpdWcPitchW + seg * 4;
+        dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+    }
+    if (tid < 128) {
+        const size_t row = static_cast<size_t>(rb) * 128 + tid;
+        reinterpret_cast<uint4*>(s_m1)[tid] = __ldg(reinterpret_cast<const uint4*>(mask1 + row * (d_in >> 3)) + cb);
+    } else {
+        const size_t blk = static_cast<size_t>(cb) * (d_out >> 7) + rb;
+        reinterpret_cast<uint4*>(s_mt)[tid - 128] = __ldg(metaT + blk * 128 + (tid - 128));
+    }
+    __syncthreads();
+
+    const int j = tid & 127;
+    const uint16_t* s_wc16 = reinterpret_cast<const uint16_t*>(s_wc);
+    auto fetch = [&](int i) -> uint32_t {
+        const uint32_t mbyte = s_m1[i * 16 + (j >> 3)];
+        const uint32_t kept = (mbyte >> (j & 7)) & 1u;
+        const uint32_t group = (mbyte >> (j & 4)) & 0xFu;
+        const int rank = __popc(group & ((1u << (j & 3)) - 1u));
+        return kept ? s_wc16[i * (kUpdWcPitchW * 2) + 2 * (j >> 2) + rank] : 0u;
+    };
+#pragma unroll 1
+    for (int it = 0; it < 8; ++it) {
+        const int ig = it * 2 + (tid >> 7);
+        const uint32_t code = s_mt[meta_byte_offset(j, ig)];
+        const int base = ig * 8;
+        uint2 out;
+        out.x = fetch(base + (code & 3)) | (fetch(base + ((code >> 2) & 3)) << 16);
+        out.y = fetch(base + 4 + ((code >> 4) & 3)) | (fetch(base + 4 + ((code >> 6) & 3)) << 16);
+        *reinterpret_cast<uint2*>(s_out + j * kDpOutPitch + ig * 8) = out;
+    }
+    __syncthreads();
+    const size_t vrow_u4 = static_cast<size_t>(d_out) >> 4;
+#pragma unroll
+    for (int pass = 0; pass < 4; ++pass) {
+        const int jr = pass * 32 + (tid >> 3), seg = tid & 7;
+        const uint2 a = *reinterpret_cast<const uint2*>(s_out + jr * kDpOutPitch + seg * 16);
+        const uint2 b = *reinterpret_cast<const uint2*>(s_out + jr * kDpOutPitch + seg * 16 + 8);
+        valsT[(static_cast<size_t>(cb) * 128 + jr) * vrow_u4 + rb * 8 + seg] = make_uint4(a.x, a.y, b.x, b.y);
+    }
+}
+
 }  // namespace slope

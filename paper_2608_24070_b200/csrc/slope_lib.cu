@@ -449,6 +449,40 @@ slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY, c
     return launch_result();
 }
 
+slope_status_t slope_sparse_add(const void* A_vals, const void* B_vals, float beta, float gamma, int rows, int cols,
+                                void* out_vals, void* stream) {
+    if (!A_vals || !B_vals || !out_vals) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(rows, cols)) return SLOPE_ERR_SHAPE;
+    if (!aligned16(A_vals) || !aligned16(B_vals) || !aligned16(out_vals)) return SLOPE_ERR_ALIGNMENT;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    const size_t n_vec = static_cast<size_t>(rows) * cols / 2 / 8;
+    sparse_add_kernel<<<info.sm_count * 8, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4*>(A_vals), static_cast<const uint4*>(B_vals), beta, gamma, n_vec,
+        static_cast<uint4*>(out_vals));
+    return launch_result();
+}
+
+slope_status_t slope_update_sparse_matrix(const void* Wc_vals, const void* mask1_bits, const void* WTc_meta,
+                                          int d_out, int d_in, void* WTc_vals, void* stream) {
+    if (!Wc_vals || !mask1_bits || !WTc_meta || !WTc_vals) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(d_out, d_in)) return SLOPE_ERR_SHAPE;
+    if (!aligned16(Wc_vals) || !aligned16(mask1_bits) || !aligned16(WTc_meta) || !aligned16(WTc_vals))
+        return SLOPE_ERR_ALIGNMENT;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (!set_smem(update_transposed_kernel, kUpdSmemBytes)) return SLOPE_ERR_CUDA;
+        attr_set = true;
+    }
+    dim3 grid(d_in / 128, d_out / 128);
+    update_transposed_kernel<<<grid, 256, kUpdSmemBytes, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4*>(Wc_vals), static_cast<const uint8_t*>(mask1_bits),
+        static_cast<const uint4*>(WTc_meta), d_out, d_in, static_cast<uint4*>(WTc_vals));
+    return launch_result();
+}
+
 slope_status_t slope_meta_to_canonical(const void* meta_hw, int rows, int cols, void* meta_canon, void* stream) {
     if (!meta_hw || !meta_canon) return SLOPE_ERR_INVALID_ARG;
     if (!dims_ok(rows, cols)) return SLOPE_ERR_SHAPE;
