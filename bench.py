@@ -158,7 +158,8 @@ def run_layer(B, s: LayerState, rec=None):
             rec(op, s, fn)
 
     stage("prune_24", lambda: B.slope_prune_24(s.W, s.Wc_vals, s.Wc_meta, s.mask1))
-    stage("double_prune", lambda: B.slope_double_prune(s.W, s.mask1, s.WTc_vals, s.WTc_meta, s.mask2))
+    # the second-pass mask is an optional diagnostic output (no kernel of the step reads it)
+    stage("double_prune", lambda: B.slope_double_prune(s.W, s.mask1, s.WTc_vals, s.WTc_meta, None))
     if s.r:
         stage("adapter_T", lambda: B.slope_adapter_fwd_bwd(0, s.X, None, s.L, None, s.b, s.d_out, s.d_in, s.r, T=s.T))
         stage("linear_fwd", lambda: B.slope_linear_fwd(s.X, s.Wc_vals, s.Wc_meta, s.d_out, s.Y, s.T, s.R))
@@ -375,7 +376,7 @@ def main():
                                "tflops_dense_eq": round(fl / (ms * 1e-3) / 1e12, 1)})
         elif op in ("prune_24", "double_prune") and (d_in, d_out, op) not in seen:
             seen.add((d_in, d_out, op))
-            bytes_ = d_in * d_out * (3.25 if op == "prune_24" else 3.375)
+            bytes_ = d_in * d_out * (3.25 if op == "prune_24" else 3.25)   # double prune: 2 + 0.125 in, 1 + 0.125 out
             stage_rows.append({"layer": name, "d_in": d_in, "d_out": d_out, "op": op, "ms": round(ms, 4),
                                "gbs": round(bytes_ / (ms * 1e-3) / 1e9, 1)})
 

@@ -4,40 +4,64 @@
 // Both pruning kernels work on 128 x 128 element tiles (one CTA of 256 threads per
 // tile) so that the 2 KB metadata block of a tile -- already in the order the sparse
 // tensor-core instruction reads it -- and the tile's mask rows leave the CTA as full
-// 16-byte stores.  Every global access is a 16-byte vector, rows are read 256 B at a
-// time per half-warp.
+// 16-byte stores.  Every global access is a 16-byte vector.  The selection itself is
+// done on packed half-words (two groups per 32-bit lane) because a scalar formulation
+// makes these kernels issue-bound long before they reach the HBM roof.
 #pragma once
 #include "ptx.cuh"
 
 namespace slope {
 
-// Two largest of four magnitudes, lower position wins ties.  Each candidate is folded
-// into one integer (magnitude << 2 | 3 - position) so that plain max/min decide.
-// Returns the kept positions p0 < p1.
-__device__ __forceinline__ void top2_of_4(uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3, int& p0, int& p1) {
-    const uint32_t c0 = (k0 << 2) | 3u, c1 = (k1 << 2) | 2u, c2 = (k2 << 2) | 1u, c3 = (k3 << 2);
-    const uint32_t hi01 = max(c0, c1), lo01 = min(c0, c1);
-    const uint32_t hi23 = max(c2, c3), lo23 = min(c2, c3);
-    const uint32_t first = max(hi01, hi23);
-    const uint32_t second = max(min(hi01, hi23), hi01 > hi23 ? lo01 : lo23);
-    const int i1 = 3 - static_cast<int>(first & 3u), i2 = 3 - static_cast<int>(second & 3u);
-    p0 = min(i1, i2);
-    p1 = max(i1, i2);
-}
+// ---------------------------------------------------------------------------------------
+// Packed selection.  Two groups of four bf16 are processed at once: word E[i] holds element
+// i of group 0 in its low half and element i of group 1 in its high half.  All arithmetic
+// stays in 32-bit integer / logic instructions on both halves simultaneously:
+//   - magnitudes are 15 bits, so (M[i] + 0x80008000) - M[j] never borrows across halves and
+//     leaves "M[i] >= M[j]" in bits 15 and 31 (for i < j that is exactly "i beats j", the
+//     lower position winning ties);
+//   - an element is kept when it beats at least two of the other three (majority of three
+//     comparison bits, one LOP3 each);
+//   - prmt's sign-replication mode turns the keep bits into half-word masks.
+// ---------------------------------------------------------------------------------------
+struct PackedPick {
+    uint32_t out0, out1;      // kept pair of group 0 / group 1: first kept in the low half
+    uint32_t mask_byte;       // 4 keep bits of group 0 | 4 keep bits of group 1 << 4
+    uint32_t meta_byte;       // code p0 | p1<<2 of group 0 | code of group 1 << 4
+};
 
-__device__ __forceinline__ uint32_t pick16(uint32_t e0, uint32_t e1, uint32_t e2, uint32_t e3, int p) {
-    return p == 0 ? e0 : (p == 1 ? e1 : (p == 2 ? e2 : e3));
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
 }
+__device__ __forceinline__ uint32_t maj3(uint32_t a, uint32_t b, uint32_t c) { return (a & b) | (a & c) | (b & c); }
+__device__ __forceinline__ uint32_t bitsel(uint32_t m, uint32_t a, uint32_t b) { return (m & a) | (~m & b); }
 
-// One group of four bf16 (two 32-bit words, element 0 in the low half of `lo`):
-// returns kept pair packed as bf16x2 (ascending position), 4-bit code and 4-bit mask.
-__device__ __forceinline__ uint32_t prune_group(uint32_t lo, uint32_t hi, uint32_t& code, uint32_t& mbits) {
-    const uint32_t e0 = lo & 0xFFFFu, e1 = lo >> 16, e2 = hi & 0xFFFFu, e3 = hi >> 16;
-    int p0, p1;
-    top2_of_4(e0 & 0x7FFFu, e1 & 0x7FFFu, e2 & 0x7FFFu, e3 & 0x7FFFu, p0, p1);
-    code = static_cast<uint32_t>(p0 | (p1 << 2));
-    mbits = (1u << p0) | (1u << p1);
-    return pick16(e0, e1, e2, e3, p0) | (pick16(e0, e1, e2, e3, p1) << 16);
+__device__ __forceinline__ PackedPick pick2of4_packed(uint32_t E0, uint32_t E1, uint32_t E2, uint32_t E3) {
+    constexpr uint32_t G = 0x80008000u;
+    const uint32_t M0 = E0 & 0x7FFF7FFFu, M1 = E1 & 0x7FFF7FFFu, M2 = E2 & 0x7FFF7FFFu, M3 = E3 & 0x7FFF7FFFu;
+    const uint32_t c01 = M0 + G - M1, c02 = M0 + G - M2, c03 = M0 + G - M3;
+    const uint32_t c12 = M1 + G - M2, c13 = M1 + G - M3, c23 = M2 + G - M3;
+    // keep flags in bits 15 / 31
+    const uint32_t k0 = maj3(c01, c02, c03);
+    const uint32_t k1 = maj3(~c01, c12, c13);
+    const uint32_t k2 = maj3(~c02, ~c12, c23);
+    const uint32_t k3 = maj3(~c03, ~c13, ~c23);
+    // half-word masks (0xFFFF where kept): bytes 0,1 <- sign of byte 1; bytes 2,3 <- sign of byte 3
+    const uint32_t m0 = prmt(k0, 0u, 0xBB99u), m1 = prmt(k1, 0u, 0xBB99u);
+    const uint32_t m2 = prmt(k2, 0u, 0xBB99u), m3 = prmt(k3, 0u, 0xBB99u);
+    const uint32_t first = bitsel(m0, E0, bitsel(m1, E1, E2));      // lowest kept position
+    const uint32_t second = bitsel(m3, E3, bitsel(m2, E2, E1));     // highest kept position
+    PackedPick r;
+    r.out0 = prmt(first, second, 0x5410u);
+    r.out1 = prmt(first, second, 0x7632u);
+    const uint32_t t = (m0 & 0x00010001u) | (m1 & 0x00020002u) | (m2 & 0x00040004u) | (m3 & 0x00080008u);
+    r.mask_byte = (t | (t >> 12)) & 0xFFu;
+    const uint32_t p0 = ~m0 & bitsel(m1, 0x00010001u, 0x00020002u);
+    const uint32_t p1 = bitsel(m3, 0x00030003u, bitsel(m2, 0x00020002u, 0x00010001u));
+    const uint32_t c = p0 | (p1 << 2);
+    r.meta_byte = (c | (c >> 12)) & 0xFFu;
+    return r;
 }
 
 // Byte offset, inside a 2 KB metadata block, of the byte holding the codes of local
@@ -48,33 +72,38 @@ __device__ __forceinline__ int meta_byte_offset(int rr, int c8) {
     return word * 4 + ((rr >> 3) & 1) * 2 + (c8 & 1);
 }
 
+// First pass.  A thread owns 16 consecutive elements of a row (two 16-byte loads): four groups
+// = one 16-bit metadata unit, 16 mask bits and eight kept values (one 16-byte store).
 __global__ void __launch_bounds__(256) prune24_kernel(const uint4* __restrict__ W, int d_out, int d_in,
-                                                      uint2* __restrict__ vals, uint4* __restrict__ meta,
+                                                      uint4* __restrict__ vals, uint4* __restrict__ meta,
                                                       uint4* __restrict__ mask /* may be null */) {
-    __shared__ __align__(16) uint8_t s_meta[2048];
-    __shared__ __align__(16) uint8_t s_mask[2048];
+    __shared__ __align__(16) uint16_t s_meta[1024];
+    __shared__ __align__(16) uint16_t s_mask[1024];
     const int cb = blockIdx.x, rb = blockIdx.y;
     const int tid = threadIdx.x;
-    const int c8 = tid & 15, r0 = tid >> 4;
+    const int u = tid & 7, r0 = tid >> 3;                 // 16-column slot, row within a pass of 32 rows
     const size_t row_u4 = static_cast<size_t>(d_in) >> 3;
 
-    uint4 w[8];
+    uint4 w[4][2];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const size_t row = static_cast<size_t>(rb) * 128 + i * 16 + r0;
-        w[i] = __ldg(W + row * row_u4 + cb * 16 + c8);
+    for (int i = 0; i < 4; ++i) {
+        const size_t row = static_cast<size_t>(rb) * 128 + i * 32 + r0;
+        const uint4* src = W + row * row_u4 + cb * 16 + 2 * u;
+        w[i][0] = __ldg(src);
+        w[i][1] = __ldg(src + 1);
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const int rr = i * 16 + r0;
+    for (int i = 0; i < 4; ++i) {
+        const int rr = i * 32 + r0;
         const size_t row = static_cast<size_t>(rb) * 128 + rr;
-        uint32_t code0, code1, m0, m1;
-        uint2 out;
-        out.x = prune_group(w[i].x, w[i].y, code0, m0);
-        out.y = prune_group(w[i].z, w[i].w, code1, m1);
-        vals[row * row_u4 + cb * 16 + c8] = out;                  // d_in/8 uint2 per compressed row
-        s_meta[meta_byte_offset(rr, c8)] = static_cast<uint8_t>(code0 | (code1 << 4));
-        s_mask[rr * 16 + c8] = static_cast<uint8_t>(m0 | (m1 << 4));
+        // groups 0,1 from the first vector, groups 2,3 from the second
+        const PackedPick a = pick2of4_packed(prmt(w[i][0].x, w[i][0].z, 0x5410u), prmt(w[i][0].x, w[i][0].z, 0x7632u),
+                                             prmt(w[i][0].y, w[i][0].w, 0x5410u), prmt(w[i][0].y, w[i][0].w, 0x7632u));
+        const PackedPick b = pick2of4_packed(prmt(w[i][1].x, w[i][1].z, 0x5410u), prmt(w[i][1].x, w[i][1].z, 0x7632u),
+                                             prmt(w[i][1].y, w[i][1].w, 0x5410u), prmt(w[i][1].y, w[i][1].w, 0x7632u));
+        vals[row * (row_u4 >> 1) + cb * 8 + u] = make_uint4(a.out0, a.out1, b.out0, b.out1);
+        s_meta[meta_byte_offset(rr, 2 * u) >> 1] = static_cast<uint16_t>(a.meta_byte | (b.meta_byte << 8));
+        s_mask[rr * 8 + u] = static_cast<uint16_t>(a.mask_byte | (b.mask_byte << 8));
     }
     __syncthreads();
     if (tid < 128) {
@@ -90,7 +119,9 @@ __global__ void __launch_bounds__(256) prune24_kernel(const uint4* __restrict__ 
 // Second pass.  Tile (rb, cb) of W (rows = d_out, cols = d_in) produces tile (cb, rb) of
 // the compressed transposed matrix.  Shared memory: the bf16 tile with a 260-byte row
 // pitch (column reads are then conflict free), the first-pass mask rows, and staging for
-// the three outputs.
+// the three outputs.  A thread owns one column j and eight rows (two groups, processed as
+// one packed pair); a warp owns 32 consecutive columns, so a row's 32 first-pass mask bits
+// are one broadcast word and the second mask leaves as warp ballots.
 constexpr int kDpTilePitchW = 65;            // 32-bit words per tile row (130 bf16)
 constexpr int kDpOutPitch = 136;             // bytes per staged output row (128 + 8)
 constexpr int kDpSmemBytes = 128 * kDpTilePitchW * 4 + 2048 + 128 * kDpOutPitch + 2048 + 2048;
@@ -131,31 +162,32 @@ __global__ void __launch_bounds__(256) double_prune_kernel(const uint4* __restri
 
     const int j = tid & 127;                         // local column of W = local row of W^T
     const int lane = tid & 31;
+    const int jw = j >> 5;                           // which 32-column word of a mask row
     const uint16_t* s_w16 = reinterpret_cast<const uint16_t*>(s_w);
+    const uint32_t* s_m1w = reinterpret_cast<const uint32_t*>(s_m1);
+    uint32_t* s_m2w = reinterpret_cast<uint32_t*>(s_m2);
 #pragma unroll 1
     for (int it = 0; it < 8; ++it) {
         const int ig = it * 2 + (tid >> 7);          // 8-row slot of the tile (0..15)
-        uint32_t e[8], kept = 0;
+        uint32_t e[8], mrow[8];
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
             const int i = ig * 8 + t;
-            const uint32_t k1 = (s_m1[i * 16 + (j >> 3)] >> (j & 7)) & 1u;
-            kept |= k1 << t;
-            e[t] = k1 ? s_w16[i * (kDpTilePitchW * 2) + j] : 0u;
+            mrow[t] = s_m1w[i * 4 + jw];                                     // same word for the whole warp
+            const uint32_t keep = static_cast<uint32_t>(static_cast<int32_t>(mrow[t] << (31 - lane)) >> 31);
+            e[t] = s_w16[i * (kDpTilePitchW * 2) + j] & keep;                // pruned in pass 1 -> +0
         }
-        int p0, p1, q0, q1;
-        top2_of_4(e[0] & 0x7FFFu, e[1] & 0x7FFFu, e[2] & 0x7FFFu, e[3] & 0x7FFFu, p0, p1);
-        top2_of_4(e[4] & 0x7FFFu, e[5] & 0x7FFFu, e[6] & 0x7FFFu, e[7] & 0x7FFFu, q0, q1);
-        uint2 out;
-        out.x = pick16(e[0], e[1], e[2], e[3], p0) | (pick16(e[0], e[1], e[2], e[3], p1) << 16);
-        out.y = pick16(e[4], e[5], e[6], e[7], q0) | (pick16(e[4], e[5], e[6], e[7], q1) << 16);
-        *reinterpret_cast<uint2*>(s_out + j * kDpOutPitch + ig * 8) = out;
-        s_meta[meta_byte_offset(j, ig)] = static_cast<uint8_t>(p0 | (p1 << 2) | (q0 << 4) | (q1 << 6));
-        const uint32_t sel = ((1u << p0) | (1u << p1) | (16u << q0) | (16u << q1)) & kept;
+        const PackedPick pk = pick2of4_packed(e[0] | (e[4] << 16), e[1] | (e[5] << 16), e[2] | (e[6] << 16),
+                                              e[3] | (e[7] << 16));
+        *reinterpret_cast<uint2*>(s_out + j * kDpOutPitch + ig * 8) = make_uint2(pk.out0, pk.out1);
+        s_meta[meta_byte_offset(j, ig)] = static_cast<uint8_t>(pk.meta_byte);
+        // second mask (optional output) = selected here AND kept by the first pass; one ballot per row
+        if (mask2 != nullptr) {
 #pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            const uint32_t word = __ballot_sync(0xFFFFFFFFu, (sel >> t) & 1u);
-            if (lane == 0) reinterpret_cast<uint32_t*>(s_m2)[(ig * 8 + t) * 4 + (j >> 5)] = word;
+            for (int t = 0; t < 8; ++t) {
+                const uint32_t word = __ballot_sync(0xFFFFFFFFu, (pk.mask_byte >> t) & 1u) & mrow[t];
+                if (lane == 0) s_m2w[(ig * 8 + t) * 4 + jw] = word;
+            }
         }
     }
     __syncthreads();

@@ -332,7 +332,7 @@ slope_status_t slope_prune_24(const void* W, int d_out, int d_in, void* Wc_vals,
     if (slope_status_t st = check_arch(info)) return st;
     dim3 grid(d_in / 128, d_out / 128);
     prune24_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const uint4*>(W), d_out, d_in, static_cast<uint2*>(Wc_vals), static_cast<uint4*>(Wc_meta),
+        static_cast<const uint4*>(W), d_out, d_in, static_cast<uint4*>(Wc_vals), static_cast<uint4*>(Wc_meta),
         static_cast<uint4*>(mask1_bits));
     return launch_result();
 }
