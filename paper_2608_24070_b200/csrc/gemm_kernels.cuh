@@ -289,21 +289,30 @@ struct SparsePairCfg {
     static constexpr int kBBytes = kHalfN * 256;
     static constexpr int kEBytes = 2048;
     static constexpr int kStageBytes = kABytes + kBBytes + kEBytes;
-    static constexpr int kSmemBytes = STAGES * kStageBytes + 256 + 1024;
+    static constexpr int kStoreRows = 32;                         // tokens per TMA store
+    static constexpr int kStoreCols = 32;                         // features per TMA store (one warp's lanes)
+    static constexpr int kStoreBytes = kStoreRows * kStoreCols * 2;
+    static constexpr int kEpiWarps = 8;                           // two warps per tensor-memory lane quadrant
+    static constexpr int kThreads = 64 + 32 * kEpiWarps;
+    static constexpr int kOffStore = STAGES * kStageBytes;
+    static constexpr int kOffBar = kOffStore + kEpiWarps * 2 * kStoreBytes;
+    static constexpr int kSmemBytes = kOffBar + 256 + 1024;
     static constexpr int kECol = 2 * BLOCK_N;
-    static_assert(BLOCK_N % 16 == 0 && kHalfN % 8 == 0 && 2 * BLOCK_N + 8 <= 512, "tile does not fit tensor memory");
+    static_assert(BLOCK_N % 32 == 0 && kHalfN % 8 == 0 && 2 * BLOCK_N + 8 <= 512, "tile does not fit tensor memory");
     static_assert(kStageBytes % 1024 == 0, "stage must keep 1024-byte alignment");
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
 };
 
 template <int BLOCK_N, int STAGES>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(SparsePairCfg<BLOCK_N, STAGES>::kThreads, 1)
 sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                         const __grid_constant__ CUtensorMap tmE, const __grid_constant__ CUtensorMap tmA2,
-                        const __grid_constant__ CUtensorMap tmB2, const SparseGemmParams p) {
+                        const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmO,
+                        const SparseGemmParams p) {
     using Cfg = SparsePairCfg<BLOCK_N, STAGES>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * Cfg::kStageBytes);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBar);
     uint64_t* empty_bar = full_bar + STAGES;
     uint64_t* tfull_bar = empty_bar + STAGES;
     uint64_t* tempty_bar = tfull_bar + 2;
@@ -323,7 +332,7 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], 8); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], 2 * Cfg::kEpiWarps); }
         *abort_flag = 0;
         fence_mbar_init();
     }
@@ -426,11 +435,19 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
-        const uint64_t stream_out = l2_policy_evict_first();
+        // ------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+        // Warp w drains lane quadrant w%4; the two warps of a quadrant take alternate 32-token
+        // blocks.  A block is transposed through the warp's private staging buffer (lane =
+        // feature writes one bf16 per token row) and leaves as a TMA store of 32 tokens x 32
+        // features, so no warp waits for another and the stores cost no LSU issue slots.
         const int q = warp & 3;
+        const int ew = warp - 2;
+        const int half = ew >> 2;
+        uint8_t* my_buf = smem + Cfg::kOffStore + ew * 2 * Cfg::kStoreBytes;
+        const uint64_t stream_out = l2_policy_evict_first();
         bool ok = true;
         int it = 0;
+        uint32_t buf = 0;
         for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
             const int m_pair = tile % num_m, n_blk = tile / num_m;
             const int acc = it & 1;
@@ -438,28 +455,35 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             if (!mbar_wait(&tfull_bar[acc], acc_phase, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t t_row = tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
-            const int m = (m_pair * 2 + static_cast<int>(cta)) * kBlockM + q * 32 + lane;
-            uint16_t* out_col = p.out + m;
+            const int m0 = (m_pair * 2 + static_cast<int>(cta)) * kBlockM + q * 32;
 #pragma unroll 1
-            for (int c0 = 0; c0 < BLOCK_N; c0 += 16) {
-                uint32_t v[16];
-                tmem_ld_16(t_row + c0, v);
+            for (int c0 = half * Cfg::kStoreRows; c0 < BLOCK_N; c0 += 2 * Cfg::kStoreRows) {
+                uint32_t v0[16], v1[16];
+                tmem_ld_16(t_row + c0, v0);
+                tmem_ld_16(t_row + c0 + 16, v1);
+                // the staging buffer about to be overwritten must have been read by its TMA store
+                if (lane == 0) tma_store_wait_read<1>();
+                __syncwarp();
                 tmem_ld_wait();
-                const int n0 = n_blk * BLOCK_N + c0;
-                if (m < p.M) {
+                uint16_t* sbuf = reinterpret_cast<uint16_t*>(my_buf + buf * Cfg::kStoreBytes) + lane;
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const int n = n0 + c;
-                        if (n < p.Ntok)
-                            st_global_evict_first_u16(out_col + static_cast<size_t>(n) * p.M,
-                                                      to_bf16(__uint_as_float(v[c])), stream_out);
-                    }
+                for (int c = 0; c < 16; ++c) {
+                    sbuf[c * Cfg::kStoreCols] = to_bf16(__uint_as_float(v0[c]));
+                    sbuf[(c + 16) * Cfg::kStoreCols] = to_bf16(__uint_as_float(v1[c]));
                 }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0 && m0 < p.M) {
+                    tma_store_2d_hint(&tmO, my_buf + buf * Cfg::kStoreBytes, m0, n_blk * BLOCK_N + c0, stream_out);
+                    tma_store_commit();
+                }
+                buf ^= 1u;
             }
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&tempty_bar[acc]), 0));
         }
+        if (lane == 0) tma_store_wait_all<0>();
     }
 
     __syncwarp();

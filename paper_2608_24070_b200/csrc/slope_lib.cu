@@ -161,17 +161,18 @@ static slope_status_t launch_dense(const void* A, const void* B, int M, int N, i
 }
 
 // ------------------------------------------------------------------ CTA-pair launches (main GEMMs)
-constexpr int kPairBlockN = 240;
+constexpr int kPairBlockN = 224;
 constexpr int kPairStages = 4;
 
 static slope_status_t launch_sparse_pair(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                          const void* act2, const void* fac2, int r, bool a2_mn, void* out,
                                          cudaStream_t stream, const DeviceInfo& info) {
     using Cfg = SparsePairCfg<kPairBlockN, kPairStages>;
-    CUtensorMap tmA, tmB, tmE, tmA2, tmB2;
+    CUtensorMap tmA, tmB, tmE, tmA2, tmB2, tmO;
     if (!make_tmap(&tmA, vals, M, K / 2, kBlockM, 64)) return SLOPE_ERR_CUDA;
     if (!make_tmap(&tmB, act, ntok, K, Cfg::kHalfN, 64)) return SLOPE_ERR_CUDA;
     if (!make_tmap_meta(&tmE, meta, static_cast<size_t>(M) * K / 8)) return SLOPE_ERR_CUDA;
+    if (!make_tmap_plain(&tmO, out, ntok, M, Cfg::kStoreRows, Cfg::kStoreCols)) return SLOPE_ERR_CUDA;
     if (r > 0) {
         const bool ok2 = a2_mn ? make_tmap(&tmA2, fac2, r, M, 64, 64) : make_tmap(&tmA2, fac2, M, r, kBlockM, 64);
         if (!ok2 || !make_tmap(&tmB2, act2, ntok, r, Cfg::kHalfN, 64)) return SLOPE_ERR_CUDA;
@@ -192,7 +193,7 @@ static slope_status_t launch_sparse_pair(const void* act, int ntok, const void* 
     const int tiles = ((M / kBlockM + 1) / 2) * ((ntok + kPairBlockN - 1) / kPairBlockN);
     const int max_pairs = info.sm_count / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
-    return launch_pairs(kern, 2 * pairs, kGemmThreads, Cfg::kSmemBytes, stream, tmA, tmB, tmE, tmA2, tmB2, p);
+    return launch_pairs(kern, 2 * pairs, Cfg::kThreads, Cfg::kSmemBytes, stream, tmA, tmB, tmE, tmA2, tmB2, tmO, p);
 }
 
 constexpr int kQuadBlockN = 224;
@@ -393,6 +394,12 @@ slope_status_t slope_linear_bwd_dw_masked(const void* dY, const void* X, int b, 
     if (!aligned16(dY) || !aligned16(X) || !aligned16(mask1_bits) || !aligned16(dWc_vals)) return SLOPE_ERR_ALIGNMENT;
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
+    // Small weight matrices do not have enough 256 x 256 tiles for the 74 CTA pairs; they run on
+    // 128 x 128 tiles, one CTA each, which fill the machine at the price of more L2 traffic per FLOP.
+    const int pair_tiles = ((d_out + 255) / 256) * ((d_in + 255) / 256);
+    if (pair_tiles * 2 <= info.sm_count)
+        return launch_dense<true, true, 128, kEpiMasked, 6>(dY, X, d_out, d_in, b, 1, dWc_vals, mask1_bits,
+                                                            static_cast<cudaStream_t>(stream), info);
     return launch_dense_pair<true, true, 256, kEpiMasked, 6>(dY, X, d_out, d_in, b, dWc_vals, mask1_bits,
                                                              static_cast<cudaStream_t>(stream), info);
 }
