@@ -183,6 +183,14 @@ slope_status_t slope_adapter_dl_noalloc(const void* X, const void* dT, int b, in
 slope_status_t slope_meta_to_canonical(const void* meta_hw, int rows, int cols,
                                        void* meta_canon, void* stream);
 
+/*
+ * Self-test of the bounded device-side waits (no counterpart in the paper): launches one warp
+ * that waits, for at most limit_us microseconds (1..100000), on a barrier nothing ever
+ * completes.  The kernel then returns normally, writes 1 to the device int *gave_up_flag and
+ * leaves SLOPE_ERR_TIMEOUT in the sticky status; the context stays usable.
+ */
+slope_status_t slope_selftest_wait_timeout(unsigned int limit_us, void* gave_up_flag, void* stream);
+
 /* Synchronises `stream`, returns and clears the sticky device status. */
 slope_status_t slope_poll_status(void* stream);
 

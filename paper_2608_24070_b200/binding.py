@@ -28,7 +28,7 @@ EXPORTS = (
     "slope_linear_bwd_dw_masked", "slope_adapter_workspace_bytes", "slope_adapter_fwd_bwd",
     "slope_meta_to_canonical", "slope_poll_status", "slope_launch_count", "slope_status_string",
     "slope_adapter_dl_noalloc", "slope_adapter_dl_noalloc_max_scratch_bytes",
-    "slope_sparse_add", "slope_update_sparse_matrix",
+    "slope_sparse_add", "slope_update_sparse_matrix", "slope_selftest_wait_timeout",
 )
 
 
@@ -67,6 +67,8 @@ def lib() -> ctypes.CDLL:
         L.slope_sparse_add.restype = ci
         L.slope_update_sparse_matrix.argtypes = [vp, vp, vp, ci, ci, vp, vp]
         L.slope_update_sparse_matrix.restype = ci
+        L.slope_selftest_wait_timeout.argtypes = [ctypes.c_uint, vp, vp]
+        L.slope_selftest_wait_timeout.restype = ci
         L.slope_poll_status.argtypes = [vp]
         L.slope_launch_count.restype = ctypes.c_ulonglong
         L.slope_status_string.restype = ctypes.c_char_p
@@ -179,6 +181,10 @@ def slope_update_sparse_matrix(Wc_vals, mask1_bits, WTc_meta, WTc_vals):
 def slope_meta_to_canonical(meta_hw, rows, cols, meta_canon):
     _check("slope_meta_to_canonical", lib().slope_meta_to_canonical(_ptr(meta_hw), rows, cols, _ptr(meta_canon),
                                                                     _stream()))
+
+
+def slope_selftest_wait_timeout(limit_us: int, gave_up_flag):
+    _check("slope_selftest_wait_timeout", lib().slope_selftest_wait_timeout(int(limit_us), _ptr(gave_up_flag), _stream()))
 
 
 def slope_poll_status() -> int:

@@ -318,4 +318,22 @@ __global__ void __launch_bounds__(256) update_transposed_kernel(const uint4* __r
     }
 }
 
+// Self-test of the bounded wait every pipeline role uses: one warp waits on an mbarrier phase
+// that nothing will ever complete.  The wait must give up after `limit_ns`, raise the device
+// status to "timeout" and let the kernel return normally.
+__global__ void __launch_bounds__(32) wait_timeout_probe_kernel(unsigned long long limit_ns, int* gave_up) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        fence_mbar_init();
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) {
+        const bool done = mbar_wait(&bar, 0u, &abort_flag, limit_ns);
+        *gave_up = done ? 0 : 1;
+    }
+}
+
 }  // namespace slope

@@ -490,6 +490,15 @@ slope_status_t slope_update_sparse_matrix(const void* Wc_vals, const void* mask1
     return launch_result();
 }
 
+slope_status_t slope_selftest_wait_timeout(unsigned int limit_us, void* gave_up_flag, void* stream) {
+    if (!gave_up_flag || limit_us == 0 || limit_us > 100000) return SLOPE_ERR_INVALID_ARG;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    wait_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<unsigned long long>(limit_us) * 1000ull, static_cast<int*>(gave_up_flag));
+    return launch_result();
+}
+
 slope_status_t slope_meta_to_canonical(const void* meta_hw, int rows, int cols, void* meta_canon, void* stream) {
     if (!meta_hw || !meta_canon) return SLOPE_ERR_INVALID_ARG;
     if (!dims_ok(rows, cols)) return SLOPE_ERR_SHAPE;

@@ -174,3 +174,24 @@ def test_argument_errors_are_reported_before_launch(B):
     assert e.value.status == 3
     assert B.lib().slope_prune_24(None, 128, 128, None, None, None, None) == 1
     assert B.slope_poll_status() == 0
+
+
+def test_bounded_wait_times_out_and_reports_status(B, oracle):
+    """A device-side wait that nothing satisfies gives up after its limit, the kernel returns,
+    the sticky status reads SLOPE_ERR_TIMEOUT once, and the library keeps working afterwards."""
+    import time
+
+    import torch
+
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    t0 = time.perf_counter()
+    B.slope_selftest_wait_timeout(2000, flag)                 # 2 ms
+    st = B.slope_poll_status()
+    dt = time.perf_counter() - t0
+    assert st == 6 and B.slope_status_string(st) == "device-side wait timed out"
+    assert int(flag.item()) == 1
+    assert dt < 1.0
+    assert B.slope_poll_status() == 0                          # cleared by the read
+    W = si.gaussian_bf16((128, 128), 0.02, 77)
+    layer = GpuLayer(W)
+    check_selection(oracle, layer, W)                          # context still healthy
