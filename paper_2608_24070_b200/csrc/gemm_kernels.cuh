@@ -1,11 +1,16 @@
 // tcgen05 GEMM kernels for sm_100a.
 //
-// Both kernels are persistent and warp-specialised: warp 0 feeds shared memory with TMA,
-// warp 1 owns tensor memory and issues the MMAs (one elected thread), warps 2..5 drain the
-// fp32 accumulators from tensor memory, convert to bf16 and store.  Two accumulator stages
-// in tensor memory let the epilogue of tile t overlap the main loop of tile t+1.  Every
-// mbarrier wait is bounded (ptx.cuh); a role that gives up sets a CTA-wide flag, all roles
-// leave their loops, tensor memory is released and the kernel returns.
+// All kernels are persistent and warp-specialised: warp 0 feeds shared memory with TMA,
+// warp 1 owns tensor memory and issues the MMAs (one elected thread), the remaining warps
+// drain the fp32 accumulators from tensor memory, convert to bf16 and store.  Every mbarrier
+// wait is bounded (ptx.cuh); a role that gives up sets a CTA-wide flag, all roles leave their
+// loops, tensor memory is released and the kernel returns.
+//
+//   dense_gemm_kernel          1 CTA per 128 x N tile; the skinny adapter GEMMs and small dW
+//   dense_gemm_pair_kernel     CTA pair per 256 x 256 tile (cta_group::2); dW
+//   sparse_gemm_pair_kernel    CTA pair per 256 x 224 tile, tcgen05.mma.sp; forward / dX
+//   sparse_gemm_quad_kernel    CTA pair per 512 x 224 tile (two MMA sub-tiles per activation
+//                              tile); forward / dX with long reductions
 #pragma once
 #include "ptx.cuh"
 
