@@ -84,8 +84,11 @@ struct DenseCfg {
 
 template <bool A_MN, bool B_MN, int BLOCK_N, int EPI, int STAGES>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                  const DenseGemmParams p) {
+dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+                  const DenseGemmParams p0, const __grid_constant__ CUtensorMap tmA1,
+                  const __grid_constant__ CUtensorMap tmB1, const DenseGemmParams p1) {
+    // Up to two independent problems of the same kind share one launch (p1.M == 0: only one):
+    // tiles [0, tiles0) belong to problem 0, the rest to problem 1.
     using Cfg = DenseCfg<BLOCK_N, STAGES>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -97,11 +100,11 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_m = (p.M + kBlockM - 1) / kBlockM;
-    const int num_n = (p.N + BLOCK_N - 1) / BLOCK_N;
-    const int num_kb_total = (p.K + 63) / 64;
-    const int kb_per_split = (num_kb_total + p.k_splits - 1) / p.k_splits;
-    const int num_tiles = num_m * num_n * p.k_splits;
+    auto tiles_of = [](const DenseGemmParams& q) {
+        return q.M == 0 ? 0 : ((q.M + kBlockM - 1) / kBlockM) * ((q.N + BLOCK_N - 1) / BLOCK_N) * q.k_splits;
+    };
+    const int tiles0 = tiles_of(p0);
+    const int num_tiles = tiles0 + tiles_of(p1);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
@@ -118,26 +121,35 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    // tile -> (m block, n block, split): m fastest so that concurrently running CTAs share B
+    // tile -> (problem, m block, n block, split): m fastest so that concurrently running CTAs share B
     auto decode = [&](int tile, int& m_blk, int& n_blk, int& kb0, int& kb1) {
+        const bool second = tile >= tiles0;
+        const DenseGemmParams& q = second ? p1 : p0;
+        if (second) tile -= tiles0;
+        const int num_m = (q.M + kBlockM - 1) / kBlockM;
+        const int num_n = (q.N + BLOCK_N - 1) / BLOCK_N;
+        const int num_kb_total = (q.K + 63) / 64;
+        const int kb_per_split = (num_kb_total + q.k_splits - 1) / q.k_splits;
         m_blk = tile % num_m;
         const int rest = tile / num_m;
         n_blk = rest % num_n;
         const int split = rest / num_n;
         kb0 = split * kb_per_split;
         kb1 = min(num_kb_total, kb0 + kb_per_split);
-        return split;
+        return split | (second ? 0x10000 : 0);
     };
 
     if (warp == 0) {
         if (elect_one()) {
-            tma_prefetch_desc(&tmA);
-            tma_prefetch_desc(&tmB);
+            tma_prefetch_desc(&tmA0);
+            tma_prefetch_desc(&tmB0);
             PipeState ps;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
                 int m_blk, n_blk, kb0, kb1;
-                decode(tile, m_blk, n_blk, kb0, kb1);
+                const bool second = (decode(tile, m_blk, n_blk, kb0, kb1) & 0x10000) != 0;
+                const CUtensorMap* tmA = second ? &tmA1 : &tmA0;
+                const CUtensorMap* tmB = second ? &tmB1 : &tmB0;
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (!mbar_wait(&empty_bar[ps.stage], ps.phase ^ 1u, abort_flag)) { ok = false; break; }
                     uint8_t* sA = smem + ps.stage * Cfg::kStageBytes;
@@ -145,17 +157,17 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     uint64_t* bar = &full_bar[ps.stage];
                     mbar_expect_tx(bar, Cfg::kStageBytes);
                     if (A_MN) {
-                        tma_load_2d(sA, &tmA, bar, m_blk * kBlockM, kb * 64);
-                        tma_load_2d(sA + 8192, &tmA, bar, m_blk * kBlockM + 64, kb * 64);
+                        tma_load_2d(sA, tmA, bar, m_blk * kBlockM, kb * 64);
+                        tma_load_2d(sA + 8192, tmA, bar, m_blk * kBlockM + 64, kb * 64);
                     } else {
-                        tma_load_2d(sA, &tmA, bar, kb * 64, m_blk * kBlockM);
+                        tma_load_2d(sA, tmA, bar, kb * 64, m_blk * kBlockM);
                     }
                     if (B_MN) {
 #pragma unroll
                         for (int h = 0; h < BLOCK_N / 64; ++h)
-                            tma_load_2d(sB + h * 8192, &tmB, bar, n_blk * BLOCK_N + h * 64, kb * 64);
+                            tma_load_2d(sB + h * 8192, tmB, bar, n_blk * BLOCK_N + h * 64, kb * 64);
                     } else {
-                        tma_load_2d(sB, &tmB, bar, kb * 64, n_blk * BLOCK_N);
+                        tma_load_2d(sB, tmB, bar, kb * 64, n_blk * BLOCK_N);
                     }
                     ps.advance(STAGES);
                 }
@@ -200,7 +212,9 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         int it = 0;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++it) {
             int m_blk, n_blk, kb0, kb1;
-            const int split = decode(tile, m_blk, n_blk, kb0, kb1);
+            const int code = decode(tile, m_blk, n_blk, kb0, kb1);
+            const int split = code & 0xFFFF;
+            const DenseGemmParams& p = (code & 0x10000) ? p1 : p0;
             const int acc = it & 1;
             const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
             if (!mbar_wait(&tfull_bar[acc], acc_phase, abort_flag)) { ok = false; break; }
@@ -263,19 +277,28 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 }
 
 // Fixed-order reduction of K-split partial sums: out = bf16( sum_s ws[s][m][n] ), written
-// row-major [M x N] or transposed [N x M].
-__global__ void __launch_bounds__(256)
-splitk_reduce_kernel(const float* __restrict__ ws, int M, int N, int splits, int transpose, uint16_t* __restrict__ out) {
-    const size_t total = static_cast<size_t>(M) * N;
-    for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < total;
-         idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
+// row-major [M x N] or transposed [N x M].  Up to two reductions per launch (second.M == 0: one).
+struct SplitKReduce {
+    const float* ws;
+    uint16_t* out;
+    int M, N, splits, transpose;
+};
+
+__global__ void __launch_bounds__(256) splitk_reduce_kernel(const SplitKReduce r0, const SplitKReduce r1) {
+    const size_t total0 = static_cast<size_t>(r0.M) * r0.N;
+    const size_t total1 = static_cast<size_t>(r1.M) * r1.N;
+    for (size_t gidx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; gidx < total0 + total1;
+         gidx += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        const bool second = gidx >= total0;
+        const SplitKReduce& r = second ? r1 : r0;
+        const size_t idx = second ? gidx - total0 : gidx;
+        const size_t total = second ? total1 : total0;
         float acc = 0.0f;
-        for (int s = 0; s < splits; ++s) acc += ws[static_cast<size_t>(s) * total + idx];
-        const size_t m = idx / N, n = idx % N;
-        out[transpose ? n * static_cast<size_t>(M) + m : idx] = to_bf16(acc);
+        for (int s = 0; s < r.splits; ++s) acc += r.ws[static_cast<size_t>(s) * total + idx];
+        const size_t m = idx / r.N, n = idx % r.N;
+        r.out[r.transpose ? n * static_cast<size_t>(r.M) + m : idx] = to_bf16(acc);
     }
 }
-
 
 // =====================================================================================
 // CTA-pair versions (cluster of 2, tcgen05 cta_group::2).  One MMA spans both SMs: the pair

@@ -131,33 +131,55 @@ static slope_status_t launch_result() {
     return cudaGetLastError() == cudaSuccess ? SLOPE_OK : SLOPE_ERR_CUDA;
 }
 
+// Opt in to more than 48 KB of dynamic shared memory.  Set on every launch: the attribute
+// belongs to the current device's context, and a cached "already done" flag would be wrong
+// for a second device or a second host thread.
 template <typename Kernel>
 static bool set_smem(Kernel k, int bytes) {
     return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
 }
 
 // ------------------------------------------------------------------ dense GEMM launch
+struct DenseProblem {
+    const void* A = nullptr;
+    const void* B = nullptr;
+    int M = 0, N = 0, K = 0, k_splits = 1;
+    void* out = nullptr;
+    const void* mask = nullptr;
+};
+
+// One launch of the 1-CTA dense kernel over one or two problems of the same kind.
+template <bool A_MN, bool B_MN, int BLOCK_N, int EPI, int STAGES>
+static slope_status_t launch_dense2(const DenseProblem& q0, const DenseProblem& q1, cudaStream_t stream,
+                                    const DeviceInfo& info) {
+    using Cfg = DenseCfg<BLOCK_N, STAGES>;
+    CUtensorMap tm[4];
+    DenseGemmParams p[2];
+    int tiles = 0;
+    for (int i = 0; i < 2; ++i) {
+        const DenseProblem& q = i == 0 ? q0 : (q1.M > 0 ? q1 : q0);          // unused slot mirrors problem 0
+        const bool okA = A_MN ? make_tmap(&tm[2 * i], q.A, q.K, q.M, 64, 64) : make_tmap(&tm[2 * i], q.A, q.M, q.K, kBlockM, 64);
+        const bool okB = B_MN ? make_tmap(&tm[2 * i + 1], q.B, q.K, q.N, 64, 64)
+                              : make_tmap(&tm[2 * i + 1], q.B, q.N, q.K, BLOCK_N, 64);
+        if (!okA || !okB) return SLOPE_ERR_CUDA;
+        const bool live = i == 0 || q1.M > 0;
+        p[i].M = live ? q.M : 0; p[i].N = q.N; p[i].K = q.K; p[i].k_splits = q.k_splits; p[i].out = q.out;
+        p[i].mask = static_cast<const uint8_t*>(q.mask);
+        if (live) tiles += ((q.M + kBlockM - 1) / kBlockM) * ((q.N + BLOCK_N - 1) / BLOCK_N) * q.k_splits;
+    }
+    auto kern = dense_gemm_kernel<A_MN, B_MN, BLOCK_N, EPI, STAGES>;
+    if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
+    const int grid = tiles < info.sm_count ? tiles : info.sm_count;
+    kern<<<grid, kGemmThreads, Cfg::kSmemBytes, stream>>>(tm[0], tm[1], p[0], tm[2], tm[3], p[1]);
+    return launch_result();
+}
+
 template <bool A_MN, bool B_MN, int BLOCK_N, int EPI, int STAGES>
 static slope_status_t launch_dense(const void* A, const void* B, int M, int N, int K, int k_splits, void* out,
                                    const void* mask, cudaStream_t stream, const DeviceInfo& info) {
-    using Cfg = DenseCfg<BLOCK_N, STAGES>;
-    CUtensorMap tmA, tmB;
-    const bool okA = A_MN ? make_tmap(&tmA, A, K, M, 64, 64) : make_tmap(&tmA, A, M, K, kBlockM, 64);
-    const bool okB = B_MN ? make_tmap(&tmB, B, K, N, 64, 64) : make_tmap(&tmB, B, N, K, BLOCK_N, 64);
-    if (!okA || !okB) return SLOPE_ERR_CUDA;
-    DenseGemmParams p;
-    p.M = M; p.N = N; p.K = K; p.k_splits = k_splits; p.out = out;
-    p.mask = static_cast<const uint8_t*>(mask);
-    auto kern = dense_gemm_kernel<A_MN, B_MN, BLOCK_N, EPI, STAGES>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
-        attr_set = true;
-    }
-    const int tiles = ((M + kBlockM - 1) / kBlockM) * ((N + BLOCK_N - 1) / BLOCK_N) * k_splits;
-    const int grid = tiles < info.sm_count ? tiles : info.sm_count;
-    kern<<<grid, kGemmThreads, Cfg::kSmemBytes, stream>>>(tmA, tmB, p);
-    return launch_result();
+    DenseProblem q;
+    q.A = A; q.B = B; q.M = M; q.N = N; q.K = K; q.k_splits = k_splits; q.out = out; q.mask = mask;
+    return launch_dense2<A_MN, B_MN, BLOCK_N, EPI, STAGES>(q, DenseProblem{}, stream, info);
 }
 
 // ------------------------------------------------------------------ CTA-pair launches (main GEMMs)
@@ -185,11 +207,7 @@ static slope_status_t launch_sparse_pair(const void* act, int ntok, const void* 
     p.meta = static_cast<const uint8_t*>(meta);
     p.out = static_cast<uint16_t*>(out);
     auto kern = sparse_gemm_pair_kernel<kPairBlockN, kPairStages>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
-        attr_set = true;
-    }
+    if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
     const int tiles = ((M / kBlockM + 1) / 2) * ((ntok + kPairBlockN - 1) / kPairBlockN);
     const int max_pairs = info.sm_count / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
@@ -220,11 +238,7 @@ static slope_status_t launch_sparse_quad(const void* act, int ntok, const void* 
     p.meta = static_cast<const uint8_t*>(meta);
     p.out = static_cast<uint16_t*>(out);
     auto kern = sparse_gemm_quad_kernel<kQuadBlockN, kQuadStages>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
-        attr_set = true;
-    }
+    if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
     const int tiles = ((M / kBlockM + 3) / 4) * ((ntok + kQuadBlockN - 1) / kQuadBlockN);
     const int max_pairs = info.sm_count / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
@@ -254,11 +268,7 @@ static slope_status_t launch_dense_pair(const void* A, const void* B, int M, int
     p.M = M; p.N = N; p.K = K; p.k_splits = 1; p.out = out;
     p.mask = static_cast<const uint8_t*>(mask);
     auto kern = dense_gemm_pair_kernel<A_MN, B_MN, BLOCK_N, EPI, STAGES>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
-        attr_set = true;
-    }
+    if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
     const int tiles = ((M + 2 * kBlockM - 1) / (2 * kBlockM)) * ((N + BLOCK_N - 1) / BLOCK_N);
     const int max_pairs = info.sm_count / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
@@ -347,11 +357,7 @@ slope_status_t slope_double_prune(const void* W, const void* mask1_bits, int d_o
         return SLOPE_ERR_ALIGNMENT;
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (!set_smem(double_prune_kernel, kDpSmemBytes)) return SLOPE_ERR_CUDA;
-        attr_set = true;
-    }
+    if (!set_smem(double_prune_kernel, kDpSmemBytes)) return SLOPE_ERR_CUDA;
     dim3 grid(d_in / 128, d_out / 128);
     double_prune_kernel<<<grid, 256, kDpSmemBytes, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint4*>(W), static_cast<const uint8_t*>(mask1_bits), d_out, d_in,
@@ -404,12 +410,13 @@ slope_status_t slope_linear_bwd_dw_masked(const void* dY, const void* X, int b, 
                                                              static_cast<cudaStream_t>(stream), info);
 }
 
+static size_t adapter_partial_bytes(int b, int rows, int r) {
+    return ((static_cast<size_t>(adapter_splits(b, rows)) * rows * r * sizeof(float)) + 255) & ~size_t(255);
+}
+
 size_t slope_adapter_workspace_bytes(int b, int d_out, int d_in, int r) {
     if (b <= 0 || d_out <= 0 || d_in <= 0 || r <= 0) return 0;
-    const int bn = r <= 64 ? 64 : 128;
-    const size_t wl = static_cast<size_t>(adapter_splits(b, d_in)) * d_in * bn * sizeof(float);
-    const size_t wr = static_cast<size_t>(adapter_splits(b, d_out)) * d_out * bn * sizeof(float);
-    return wl > wr ? wl : wr;
+    return adapter_partial_bytes(b, d_in, r) + adapter_partial_bytes(b, d_out, r);     // dL and dR partial sums
 }
 
 slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY, const void* L, const void* R, int b,
@@ -438,21 +445,20 @@ slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY, c
     st = r <= 64 ? launch_dense<false, false, 64, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info)
                  : launch_dense<false, false, 128, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info);
     if (st) return st;
-    // dL[d_in x r] = X^T dT: A = X stored [K x M], B = dT stored [K x N]; K = tokens, split in fixed slices
-    const int sl = adapter_splits(b, d_in);
-    st = r <= 64 ? launch_dense<true, true, 64, kEpiPartial, 6>(X, dT, d_in, r, b, sl, workspace, nullptr, stream, info)
-                 : launch_dense<true, true, 128, kEpiPartial, 6>(X, dT, d_in, r, b, sl, workspace, nullptr, stream, info);
+    // dL[d_in x r] = X^T dT and dR^T[d_out x r] = dY^T T: operands stored [K x M] / [K x N] with
+    // K = tokens, split into fixed slices; both problems share one launch, their fp32 partial
+    // sums are reduced in slice order by one more launch (dR written transposed).
+    float* ws_l = static_cast<float*>(workspace);
+    float* ws_r = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + adapter_partial_bytes(b, d_in, r));
+    DenseProblem ql, qr;
+    ql.A = X; ql.B = dT; ql.M = d_in; ql.N = r; ql.K = b; ql.k_splits = adapter_splits(b, d_in); ql.out = ws_l;
+    qr.A = dY; qr.B = T; qr.M = d_out; qr.N = r; qr.K = b; qr.k_splits = adapter_splits(b, d_out); qr.out = ws_r;
+    st = r <= 64 ? launch_dense2<true, true, 64, kEpiPartial, 6>(ql, qr, stream, info)
+                 : launch_dense2<true, true, 128, kEpiPartial, 6>(ql, qr, stream, info);
     if (st) return st;
-    splitk_reduce_kernel<<<info.sm_count * 4, 256, 0, stream>>>(static_cast<const float*>(workspace), d_in, r, sl, 0,
-                                                               static_cast<uint16_t*>(dL));
-    if ((st = launch_result())) return st;
-    // dR^T[d_out x r] = dY^T T, reduced and written transposed into dR[r x d_out]
-    const int sr = adapter_splits(b, d_out);
-    st = r <= 64 ? launch_dense<true, true, 64, kEpiPartial, 6>(dY, T, d_out, r, b, sr, workspace, nullptr, stream, info)
-                 : launch_dense<true, true, 128, kEpiPartial, 6>(dY, T, d_out, r, b, sr, workspace, nullptr, stream, info);
-    if (st) return st;
-    splitk_reduce_kernel<<<info.sm_count * 4, 256, 0, stream>>>(static_cast<const float*>(workspace), d_out, r, sr, 1,
-                                                               static_cast<uint16_t*>(dR));
+    const SplitKReduce rl{ws_l, static_cast<uint16_t*>(dL), d_in, r, ql.k_splits, 0};
+    const SplitKReduce rr{ws_r, static_cast<uint16_t*>(dR), d_out, r, qr.k_splits, 1};
+    splitk_reduce_kernel<<<info.sm_count * 4, 256, 0, stream>>>(rl, rr);
     return launch_result();
 }
 
@@ -478,11 +484,7 @@ slope_status_t slope_update_sparse_matrix(const void* Wc_vals, const void* mask1
         return SLOPE_ERR_ALIGNMENT;
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (!set_smem(update_transposed_kernel, kUpdSmemBytes)) return SLOPE_ERR_CUDA;
-        attr_set = true;
-    }
+    if (!set_smem(update_transposed_kernel, kUpdSmemBytes)) return SLOPE_ERR_CUDA;
     dim3 grid(d_in / 128, d_out / 128);
     update_transposed_kernel<<<grid, 256, kUpdSmemBytes, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint4*>(Wc_vals), static_cast<const uint8_t*>(mask1_bits),
@@ -565,7 +567,8 @@ slope_status_t slope_adapter_dl_noalloc(const void* X, const void* dT, int b, in
         r <= 64 ? launch_dense<true, true, 64, kEpiPartial, 6>(X, dT, d_in, r, b, splits, scratch, nullptr, stream, info)
                 : launch_dense<true, true, 128, kEpiPartial, 6>(X, dT, d_in, r, b, splits, scratch, nullptr, stream, info);
     if (st) return st;
-    splitk_reduce_kernel<<<info.sm_count * 4, 256, 0, stream>>>(scratch, d_in, r, splits, 0, static_cast<uint16_t*>(dL));
+    const SplitKReduce red{scratch, static_cast<uint16_t*>(dL), d_in, r, splits, 0};
+    splitk_reduce_kernel<<<info.sm_count * 4, 256, 0, stream>>>(red, SplitKReduce{nullptr, nullptr, 0, 0, 0, 0});
     return launch_result();
 }
 
