@@ -86,9 +86,10 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append(line.strip())
+            self.rows.append((time.time(), line.strip()))
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
+        """Summary of the samples taken between the two host timestamps (the timed region)."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -98,7 +99,10 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons, power = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for row in self.rows:
+        rows = [r for (t, r) in self.rows if (t_begin is None or t >= t_begin) and (t_end is None or t <= t_end)]
+        if len(rows) < 3:
+            rows = [r for (_, r) in self.rows]
+        for row in rows:
             f = [x.strip() for x in row.split(",")]
             if len(f) < 7:
                 continue
@@ -109,14 +113,9 @@ class ClockSampler:
             for n, v in zip(names, f[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
-        # "under load": samples in the upper half of the observed power range
-        if power:
-            thr = 0.5 * (max(power) + min(power))
-            load = [s for s, p in zip(sm, power) if p >= thr] or sm
-        else:
-            load = sm
-        return {"sm_mhz": statistics.median(load) if load else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_mhz_min": min(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "power_w_max": max(power) if power else None,
+                "samples": len(sm), "window": "samples taken inside the timed region", "reasons": sorted(reasons)}
 
 
 # ------------------------------------------------------------------------------ the CUDA arm
@@ -261,7 +260,7 @@ def replica_throughput(world, flops_per_replica, ms_step):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(si.WORKLOADS))
     ap.add_argument("--impl", default="slope", choices=["slope", "reference"])
@@ -279,9 +278,12 @@ def main():
 
     import torch
     from paper_2608_24070_b200 import binding as B
+    from paper_2608_24070_b200 import build as _build
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the SLoPe path has no CPU fallback")
+    if local_rank == 0:
+        _build.build()                # no-op when libslope.so is newer than its sources
     B.lib()
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
@@ -332,14 +334,18 @@ def main():
     barrier()
     torch.cuda.synchronize()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_begin = time.time()
     ev0.record(stream)
     for _ in range(args.steps):
         step(rec)
     ev1.record(stream)
     torch.cuda.synchronize()
+    t_end = time.time()
     barrier()
     launches = B.slope_launch_count() - launches0
-    clocks = sampler.stop() if rank == 0 else None
+    if rank == 0:
+        time.sleep(0.1)
+    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     ms_total = replica_max_ms(torch, dist, ev0.elapsed_time(ev1), dev)
     st = B.slope_poll_status()
     if st != 0:
@@ -383,7 +389,7 @@ def main():
     # roofline of the two tensor-core kernels; the dominant one (by time inside the step) is "roofline"
     dw_fl, dw_s = tot["linear_bwd_dw_masked"]
     dw_tflops = dw_fl / dw_s / 1e12 if dw_s else 0.0
-    roofline_dense = {"kernel": "dense_gemm_kernel<A_MN,B_MN,256,masked> (slope_linear_bwd_dw_masked)",
+    roofline_dense = {"kernel": "dense_gemm_pair_kernel<MN,MN,256,masked,6> (slope_linear_bwd_dw_masked)",
                       "bound": "tensor", "achieved": round(dw_tflops, 1), "peak": pk["bf16_sustained"],
                       "unit": "TFLOP/s", "frac": round(dw_tflops / pk["bf16_sustained"], 4), "traffic": None,
                       "ms_per_step": round(dw_s * 1e3, 4),
@@ -391,7 +397,7 @@ def main():
     sp_fl = tot["linear_fwd"][0] + tot["linear_bwd_dx"][0]
     sp_s = tot["linear_fwd"][1] + tot["linear_bwd_dx"][1]
     sp_tflops = sp_fl / sp_s / 1e12 if sp_s else 0.0
-    roofline_sparse = {"kernel": "sparse_gemm_kernel (slope_linear_fwd, slope_linear_bwd_dx)", "bound": "tensor",
+    roofline_sparse = {"kernel": "sparse_gemm_pair_kernel<224,4> + sparse_gemm_quad_kernel<224,3> (slope_linear_fwd, slope_linear_bwd_dx)", "bound": "tensor",
                        "achieved": round(sp_tflops, 1), "peak": round(sparse_peak, 1),
                        "unit": "TFLOP/s", "frac": round(sp_tflops / sparse_peak, 4), "traffic": None,
                        "ms_per_step": round(sp_s * 1e3, 4),

@@ -23,8 +23,9 @@ def B():
 
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
-    from paper_2608_24070_b200 import binding
+    from paper_2608_24070_b200 import binding, build
 
+    build.build()                     # no-op when libslope.so is newer than its sources
     binding.lib()
     return binding
 
