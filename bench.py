@@ -282,9 +282,6 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the SLoPe path has no CPU fallback")
-    if local_rank == 0:
-        _build.build()                # no-op when libslope.so is newer than its sources
-    B.lib()
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     dist = None
@@ -293,6 +290,11 @@ def main():
 
         dist = dist_mod
         dist.init_process_group("nccl", device_id=dev)
+    if local_rank == 0:
+        _build.build()                # no-op when libslope.so is newer than its sources
+    if dist is not None:
+        dist.barrier()
+    B.lib()
 
     pk = peaks()
     wl = si.WORKLOADS[args.workload]
