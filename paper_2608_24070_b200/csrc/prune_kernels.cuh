@@ -116,98 +116,90 @@ __global__ void __launch_bounds__(256) prune24_kernel(const uint4* __restrict__ 
     }
 }
 
-// Second pass.  Tile (rb, cb) of W (rows = d_out, cols = d_in) produces tile (cb, rb) of
-// the compressed transposed matrix.  Shared memory: the bf16 tile with a 260-byte row
-// pitch (column reads are then conflict free), the first-pass mask rows, and staging for
-// the three outputs.  A thread owns one column j and eight rows (two groups, processed as
-// one packed pair); a warp owns 32 consecutive columns, so a row's 32 first-pass mask bits
-// are one broadcast word and the second mask leaves as warp ballots.
-constexpr int kDpTilePitchW = 65;            // 32-bit words per tile row (130 bf16)
-constexpr int kDpOutPitch = 136;             // bytes per staged output row (128 + 8)
-constexpr int kDpSmemBytes = 128 * kDpTilePitchW * 4 + 2048 + 128 * kDpOutPitch + 2048 + 2048;
+// Second pass.  Tile (rb, cb) of W (rows = d_out, cols = d_in) produces tile (cb, rb) of the
+// compressed transposed matrix.  A thread owns 8 rows x 8 columns of the tile, read straight
+// from global memory (eight 16-byte loads, rows 256 B apart per half-warp).  Groups run down
+// the columns here, so a 32-bit word of a row (two adjacent columns) IS the packed pair the
+// selection works on: word w of rows 4g..4g+3 gives the groups of columns 2w and 2w+1 without
+// any transposition of the input.  Only the outputs (half the bytes) are transposed, through
+// an XOR-swizzled 16 KB staging tile whose 64-bit stores are conflict free.
+__device__ __forceinline__ uint32_t halfword_mask_from_bits(uint32_t mask_byte, int w) {
+    // bit 2w of the byte -> low half-word, bit 2w+1 -> high half-word (all ones where kept)
+    const uint32_t z = (mask_byte << (15 - 2 * w)) | (mask_byte << (30 - 2 * w));
+    return prmt(z, 0u, 0xBB99u);
+}
 
 __global__ void __launch_bounds__(256) double_prune_kernel(const uint4* __restrict__ W,
                                                            const uint8_t* __restrict__ mask1, int d_out, int d_in,
                                                            uint4* __restrict__ valsT, uint4* __restrict__ metaT,
-                                                           uint4* __restrict__ mask2 /* may be null */) {
-    extern __shared__ __align__(16) uint8_t dp_smem[];
-    uint32_t* s_w = reinterpret_cast<uint32_t*>(dp_smem);
-    uint8_t* s_m1 = dp_smem + 128 * kDpTilePitchW * 4;
-    uint8_t* s_out = s_m1 + 2048;
-    uint8_t* s_meta = s_out + 128 * kDpOutPitch;
-    uint8_t* s_m2 = s_meta + 2048;
+                                                           uint8_t* __restrict__ mask2 /* may be null */) {
+    __shared__ __align__(16) uint8_t s_out[128 * 128];       // [column j][16 slots of 8 B], slot index XOR (j >> 3)
+    __shared__ __align__(16) uint8_t s_meta[2048];
 
     const int cb = blockIdx.x, rb = blockIdx.y;
     const int tid = threadIdx.x;
-    const int c8 = tid & 15, r0 = tid >> 4;
+    const int c8 = tid & 15;                                 // 8-column slot of the tile
+    const int ig = tid >> 4;                                 // 8-row slot of the tile
     const size_t row_u4 = static_cast<size_t>(d_in) >> 3;
+    const size_t mrow = static_cast<size_t>(d_in) >> 3;      // mask bytes per row
 
     uint4 w[8];
+    uint32_t mb[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const size_t row = static_cast<size_t>(rb) * 128 + i * 16 + r0;
-        w[i] = __ldg(W + row * row_u4 + cb * 16 + c8);
+    for (int t = 0; t < 8; ++t) {
+        const size_t row = static_cast<size_t>(rb) * 128 + ig * 8 + t;
+        w[t] = __ldg(W + row * row_u4 + cb * 16 + c8);
+        mb[t] = __ldg(mask1 + row * mrow + cb * 16 + c8);
     }
-    if (tid < 128) {
-        const size_t row = static_cast<size_t>(rb) * 128 + tid;
-        reinterpret_cast<uint4*>(s_m1)[tid] =
-            __ldg(reinterpret_cast<const uint4*>(mask1 + row * (d_in >> 3)) + cb);
-    }
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        uint32_t* dst = s_w + (i * 16 + r0) * kDpTilePitchW + c8 * 4;
-        dst[0] = w[i].x; dst[1] = w[i].y; dst[2] = w[i].z; dst[3] = w[i].w;
-    }
-    __syncthreads();
 
-    const int j = tid & 127;                         // local column of W = local row of W^T
-    const int lane = tid & 31;
-    const int jw = j >> 5;                           // which 32-column word of a mask row
-    const uint16_t* s_w16 = reinterpret_cast<const uint16_t*>(s_w);
-    const uint32_t* s_m1w = reinterpret_cast<const uint32_t*>(s_m1);
-    uint32_t* s_m2w = reinterpret_cast<uint32_t*>(s_m2);
-#pragma unroll 1
-    for (int it = 0; it < 8; ++it) {
-        const int ig = it * 2 + (tid >> 7);          // 8-row slot of the tile (0..15)
-        uint32_t e[8], mrow[8];
+    uint32_t sel_bits[8] = {0, 0, 0, 0, 0, 0, 0, 0};         // per row: which of the 8 columns the second pass keeps
+    const int meta_base = meta_byte_offset(c8 * 8, ig);      // + 16 per column inside the 8-column slot
+#pragma unroll
+    for (int wi = 0; wi < 4; ++wi) {
+        uint32_t e[8];
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
-            const int i = ig * 8 + t;
-            mrow[t] = s_m1w[i * 4 + jw];                                     // same word for the whole warp
-            const uint32_t keep = static_cast<uint32_t>(static_cast<int32_t>(mrow[t] << (31 - lane)) >> 31);
-            e[t] = s_w16[i * (kDpTilePitchW * 2) + j] & keep;                // pruned in pass 1 -> +0
+            const uint32_t word = wi == 0 ? w[t].x : (wi == 1 ? w[t].y : (wi == 2 ? w[t].z : w[t].w));
+            e[t] = word & halfword_mask_from_bits(mb[t], wi);                 // pruned in pass 1 -> +0
         }
-        const PackedPick pk = pick2of4_packed(e[0] | (e[4] << 16), e[1] | (e[5] << 16), e[2] | (e[6] << 16),
-                                              e[3] | (e[7] << 16));
-        *reinterpret_cast<uint2*>(s_out + j * kDpOutPitch + ig * 8) = make_uint2(pk.out0, pk.out1);
-        s_meta[meta_byte_offset(j, ig)] = static_cast<uint8_t>(pk.meta_byte);
-        // second mask (optional output) = selected here AND kept by the first pass; one ballot per row
+        const PackedPick a = pick2of4_packed(e[0], e[1], e[2], e[3]);        // rows 0..3 of columns 2wi, 2wi+1
+        const PackedPick b = pick2of4_packed(e[4], e[5], e[6], e[7]);        // rows 4..7
+        const int j0 = c8 * 8 + 2 * wi;
+        const int slot = (ig ^ c8) * 8;                                        // (j >> 3) & 15 == c8 for both columns
+        *reinterpret_cast<uint2*>(s_out + j0 * 128 + slot) = make_uint2(a.out0, b.out0);
+        *reinterpret_cast<uint2*>(s_out + (j0 + 1) * 128 + slot) = make_uint2(a.out1, b.out1);
+        s_meta[meta_base + 16 * (2 * wi)] = static_cast<uint8_t>((a.meta_byte & 0xFu) | ((b.meta_byte & 0xFu) << 4));
+        s_meta[meta_base + 16 * (2 * wi + 1)] = static_cast<uint8_t>((a.meta_byte >> 4) | (b.meta_byte & 0xF0u));
         if (mask2 != nullptr) {
 #pragma unroll
-            for (int t = 0; t < 8; ++t) {
-                const uint32_t word = __ballot_sync(0xFFFFFFFFu, (pk.mask_byte >> t) & 1u) & mrow[t];
-                if (lane == 0) s_m2w[(ig * 8 + t) * 4 + jw] = word;
+            for (int i = 0; i < 4; ++i) {
+                sel_bits[i] |= (((a.mask_byte >> i) & 1u) << (2 * wi)) | (((a.mask_byte >> (4 + i)) & 1u) << (2 * wi + 1));
+                sel_bits[4 + i] |= (((b.mask_byte >> i) & 1u) << (2 * wi)) | (((b.mask_byte >> (4 + i)) & 1u) << (2 * wi + 1));
             }
         }
     }
+    if (mask2 != nullptr) {
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            const size_t row = static_cast<size_t>(rb) * 128 + ig * 8 + t;
+            mask2[row * mrow + cb * 16 + c8] = static_cast<uint8_t>(sel_bits[t] & mb[t]);
+        }
+    }
     __syncthreads();
 
-    // (W^T) tile (cb, rb): values rows of 128 B, metadata block, second mask rows.
+    // (W^T) tile (cb, rb): value rows of 128 B (undo the slot swizzle), then the metadata block.
     const size_t vrow_u4 = static_cast<size_t>(d_out) >> 4;        // uint4 per row of valsT (d_out/2 bf16)
 #pragma unroll
     for (int pass = 0; pass < 4; ++pass) {
-        const int jr = pass * 32 + (tid >> 3), seg = tid & 7;
-        const uint2 a = *reinterpret_cast<const uint2*>(s_out + jr * kDpOutPitch + seg * 16);
-        const uint2 b = *reinterpret_cast<const uint2*>(s_out + jr * kDpOutPitch + seg * 16 + 8);
-        valsT[(static_cast<size_t>(cb) * 128 + jr) * vrow_u4 + rb * 8 + seg] = make_uint4(a.x, a.y, b.x, b.y);
+        const int jr = pass * 32 + (tid >> 3), seg = tid & 7;      // logical slots 2*seg, 2*seg+1
+        const int x = (jr >> 3) & 15;
+        const uint4 v = *reinterpret_cast<const uint4*>(s_out + jr * 128 + (((2 * seg) ^ x) >> 1) * 16);
+        const uint4 o = (x & 1) ? make_uint4(v.z, v.w, v.x, v.y) : v;
+        valsT[(static_cast<size_t>(cb) * 128 + jr) * vrow_u4 + rb * 8 + seg] = o;
     }
     if (tid < 128) {
         const size_t blk = static_cast<size_t>(cb) * (d_out >> 7) + rb;
         metaT[blk * 128 + tid] = reinterpret_cast<const uint4*>(s_meta)[tid];
-    } else if (mask2 != nullptr) {
-        const int rr = tid - 128;
-        const size_t row = static_cast<size_t>(rb) * 128 + rr;
-        mask2[row * (d_in >> 7) + cb] = reinterpret_cast<const uint4*>(s_m2)[rr];
     }
 }
 
@@ -256,6 +248,7 @@ __global__ void __launch_bounds__(256) sparse_add_kernel(const uint4* __restrict
 // its metadata block says which two rows of every 4-row group were kept by the second pass,
 // the first-pass mask says whether such an element exists at all and at which rank it sits
 // in its row's compressed group.
+constexpr int kDpOutPitch = 136;                // bytes per staged output row (128 + 8)
 constexpr int kUpdWcPitchW = 33;                 // 32-bit words per staged row of 64 bf16 (+1 pad)
 constexpr int kUpdSmemBytes = 128 * kUpdWcPitchW * 4 + 2048 + 2048 + 128 * kDpOutPitch;
 

@@ -357,11 +357,10 @@ slope_status_t slope_double_prune(const void* W, const void* mask1_bits, int d_o
         return SLOPE_ERR_ALIGNMENT;
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
-    if (!set_smem(double_prune_kernel, kDpSmemBytes)) return SLOPE_ERR_CUDA;
     dim3 grid(d_in / 128, d_out / 128);
-    double_prune_kernel<<<grid, 256, kDpSmemBytes, static_cast<cudaStream_t>(stream)>>>(
+    double_prune_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint4*>(W), static_cast<const uint8_t*>(mask1_bits), d_out, d_in,
-        static_cast<uint4*>(WTc_vals), static_cast<uint4*>(WTc_meta), static_cast<uint4*>(mask2_bits));
+        static_cast<uint4*>(WTc_vals), static_cast<uint4*>(WTc_meta), static_cast<uint8_t*>(mask2_bits));
     return launch_result();
 }
 
