@@ -129,7 +129,7 @@ __device__ __forceinline__ uint32_t halfword_mask_from_bits(uint32_t mask_byte, 
     return prmt(z, 0u, 0xBB99u);
 }
 
-__global__ void __launch_bounds__(256) double_prune_kernel(const uint4* __restrict__ W,
+__global__ void __launch_bounds__(256, 4) double_prune_kernel(const uint4* __restrict__ W,
                                                            const uint8_t* __restrict__ mask1, int d_out, int d_in,
                                                            uint4* __restrict__ valsT, uint4* __restrict__ metaT,
                                                            uint8_t* __restrict__ mask2 /* may be null */) {
