@@ -196,3 +196,40 @@ def test_bounded_wait_times_out_and_reports_status(B, oracle):
     W = si.gaussian_bf16((128, 128), 0.02, 77)
     layer = GpuLayer(W)
     check_selection(oracle, layer, W)                          # context still healthy
+
+
+def test_optional_masks_and_run_to_run_determinism(B, oracle):
+    """The mask outputs are optional and do not change the other outputs; every GEMM is
+    bit-identical run to run (no floating-point atomics, split-K reduced in a fixed order)."""
+    import torch
+
+    d_out, d_in, b, r = 384, 512, 520, 32
+    W = si.gaussian_bf16((d_out, d_in), 0.02, 61)
+    layer = GpuLayer(W)
+    vals = torch.empty_like(layer.Wc_vals)
+    meta = torch.empty_like(layer.Wc_meta)
+    B.slope_prune_24(layer.W, vals, meta, None)
+    valsT = torch.empty_like(layer.WTc_vals)
+    metaT = torch.empty_like(layer.WTc_meta)
+    B.slope_double_prune(layer.W, layer.mask1, valsT, metaT, None)
+    layer.poll()
+    for a, ref in ((vals, layer.Wc_vals), (meta, layer.Wc_meta), (valsT, layer.WTc_vals), (metaT, layer.WTc_meta)):
+        assert torch.equal(a.view(torch.uint8), ref.view(torch.uint8))
+
+    X = dev(B, si.gaussian_bf16((b, d_in), 1.0, 62))
+    dY = dev(B, si.gaussian_bf16((b, d_out), 1.0, 63))
+    L = dev(B, si.gaussian_bf16((d_in, r), 0.01, 64))
+    R = dev(B, si.gaussian_bf16((r, d_out), 0.01, 65))
+
+    def run():
+        T = layer.adapter_T(X, L)
+        Y = layer.fwd(X, T, R)
+        dT, dL, dR = layer.adapter_bwd(X, dY, L, R, T)
+        dX = layer.dx(dY, dT, L)
+        dWc = layer.dw(dY, X)
+        layer.poll()
+        return [B.bits_from_bf16(t) for t in (T, Y, dT, dL, dR, dX, dWc)]
+
+    first, second = run(), run()
+    for a, c in zip(first, second):
+        assert np.array_equal(a, c)
