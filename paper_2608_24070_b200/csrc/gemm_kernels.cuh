@@ -11,6 +11,9 @@
 //   sparse_gemm_pair_kernel    CTA pair per 256 x 224 tile, tcgen05.mma.sp; forward / dX
 //   sparse_gemm_quad_kernel    CTA pair per 512 x 224 tile (two MMA sub-tiles per activation
 //                              tile); forward / dX with long reductions
+//   sparse_gemm_skinny_kernel  one CTA per 128-row weight slab and K-slice, cluster reduction
+//                              through distributed shared memory; forward / dX with at most
+//                              256 tokens (inference, decode), not persistent
 #pragma once
 #include "ptx.cuh"
 
@@ -1009,6 +1012,241 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     if (warp == 1) {
         tc_fence_after_sync();
         tmem_dealloc_pair(tmem_base, 512);
+    }
+}
+
+// =====================================================================================
+// Sparse GEMM for few tokens (inference / decode sizes, Ntok <= BLOCK_N <= 256).
+// With so few tokens the GEMM is a stream of compressed weights from HBM, and the big-tile
+// kernels above would occupy only a handful of SMs.  Here one CTA owns a 128-row slab of the
+// weights (1-CTA tcgen05.mma.sp, M = 128) and a slice of the reduction: a cluster of S CTAs
+// splits K, each accumulates its partial tile in tensor memory, parks it in its own shared
+// memory, and after a cluster barrier every CTA sums one share of the token rows over all S
+// partials through distributed shared memory -- in rank order, so the result is
+// deterministic and needs no global workspace.  The adapter K-steps ride on the last rank.
+//
+// What bounds the kernel is the number of weight bytes in flight, so the weights (values +
+// metadata, from HBM, read once) and the activations (from L2, re-read by every slab) travel
+// in two separate rings with their own producer threads: a deep one for the weights, a
+// shallow one for the activations.
+// =====================================================================================
+template <int BLOCK_N, int A_STAGES, int B_STAGES>
+struct SparseSkinnyCfg {
+    static constexpr int kABytes = kBlockM * 128;                    // compressed values of one k-block
+    static constexpr int kEBytes = 2048;                             // their metadata
+    static constexpr int kAStage = kABytes + kEBytes;
+    static constexpr int kBStage = BLOCK_N * 256;
+    static constexpr int kOffB = A_STAGES * kAStage;
+    static constexpr int kOffBar = kOffB + B_STAGES * kBStage;
+    static constexpr int kPartialBytes = BLOCK_N * kBlockM * 4;      // fp32 [token][feature], reuses the rings
+    static constexpr int kSmemBytes = kOffBar + 512 + 1024;
+    static constexpr int kTmemCols = BLOCK_N + 8 <= 32 ? 32 : (BLOCK_N + 8 <= 128 ? 128 : (BLOCK_N + 8 <= 256 ? 256 : 512));
+    static_assert(BLOCK_N % 16 == 0 && BLOCK_N >= 16 && BLOCK_N <= 256, "token tile");
+    static_assert(kPartialBytes <= kOffBar, "partial tile must fit in the pipeline buffers");
+    static_assert(kAStage % 1024 == 0 && kBStage % 1024 == 0 && kSmemBytes <= 232448, "shared memory layout");
+    static_assert(2 * (A_STAGES + B_STAGES) * 8 + 16 <= 512, "barrier block");
+};
+
+template <int BLOCK_N, int A_STAGES, int B_STAGES>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+sparse_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                          const __grid_constant__ CUtensorMap tmE, const __grid_constant__ CUtensorMap tmA2,
+                          const __grid_constant__ CUtensorMap tmB2, const SparseGemmParams p) {
+    using Cfg = SparseSkinnyCfg<BLOCK_N, A_STAGES, B_STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* fullA = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBar);
+    uint64_t* emptyA = fullA + A_STAGES;
+    uint64_t* fullB = emptyA + A_STAGES;
+    uint64_t* emptyB = fullB + B_STAGES;
+    uint64_t* tfull_bar = emptyB + B_STAGES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tfull_bar + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int splits = static_cast<int>(cluster_nctarank());
+    const int rank = static_cast<int>(cluster_ctarank());
+    const int m_blk = blockIdx.x / splits;
+    const int num_kb = p.K / 128;
+    const int kb_per = (num_kb + splits - 1) / splits;
+    const int kb0 = min(num_kb, rank * kb_per), kb1 = min(num_kb, kb0 + kb_per);
+    const int num_sb = kb1 - kb0;                                            // sparse k-blocks of this rank
+    const int num_ab = rank == splits - 1 ? (p.r + 63) / 64 : 0;            // adapter K-steps on the last rank
+    const int total_kb = num_sb + num_ab;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < A_STAGES; ++s) { mbar_init(&fullA[s], 1); mbar_init(&emptyA[s], 1); }
+        for (int s = 0; s < B_STAGES; ++s) { mbar_init(&fullB[s], 1); mbar_init(&emptyB[s], 1); }
+        mbar_init(&tfull_bar[0], 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, Cfg::kTmemCols);
+        tmem_relinquish();
+    }
+    if (warp == 0 && elect_one()) {
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmE);
+    }
+    if (warp == 2 && elect_one()) tma_prefetch_desc(&tmB);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    // Everything above overlaps the tail of the previous kernel in the stream when the launch
+    // allows it; nothing below may touch global memory before that kernel has finished.
+    griddep_launch_dependents();
+    griddep_wait();
+
+    if (warp == 0) {
+        // ---------------------------------------------------------- weight ring (values + metadata)
+        if (elect_one()) {
+            const uint64_t stream_once = l2_policy_evict_first();        // weights are read exactly once
+            PipeState ps;
+            for (int i = 0; i < total_kb; ++i) {
+                if (!mbar_wait(&emptyA[ps.stage], ps.phase ^ 1u, abort_flag)) break;
+                uint8_t* sA = smem + ps.stage * Cfg::kAStage;
+                uint64_t* bar = &fullA[ps.stage];
+                if (i < num_sb) {
+                    const int kb = kb0 + i;
+                    mbar_expect_tx(bar, Cfg::kAStage);
+                    tma_load_2d_hint(sA, &tmA, bar, kb * 64, m_blk * kBlockM, stream_once);
+                    tma_load_2d_hint(sA + Cfg::kABytes, &tmE, bar, 0, m_blk * num_kb + kb, stream_once);
+                } else {
+                    const int ab = i - num_sb;
+                    mbar_expect_tx(bar, Cfg::kABytes);
+                    if (p.a2_mn_major) {
+                        tma_load_2d(sA, &tmA2, bar, m_blk * kBlockM, ab * 64);
+                        tma_load_2d(sA + 8192, &tmA2, bar, m_blk * kBlockM + 64, ab * 64);
+                    } else {
+                        tma_load_2d(sA, &tmA2, bar, ab * 64, m_blk * kBlockM);
+                    }
+                }
+                ps.advance(A_STAGES);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------- MMA issue
+        if (elect_one()) {
+            constexpr uint32_t idesc_sp = make_idesc_bf16(kBlockM, BLOCK_N, false, false, true);
+            const uint32_t idesc_ad = make_idesc_bf16(kBlockM, BLOCK_N, p.a2_mn_major != 0, false, false);
+            PipeState pa, pb;
+            bool ok = true;
+            for (int i = 0; i < total_kb; ++i) {
+                if (!mbar_wait(&fullB[pb.stage], pb.phase, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(&fullA[pa.stage], pa.phase, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t sA = smem_u32(smem + pa.stage * Cfg::kAStage);
+                const uint32_t sE = sA + Cfg::kABytes;
+                const uint32_t sB = smem_u32(smem + Cfg::kOffB + pb.stage * Cfg::kBStage);
+                if (i < num_sb) {
+                    const uint32_t e_tmem = tmem_base + BLOCK_N + (i & 1) * 4;
+                    tmem_cp_128x128b(e_tmem, make_smem_desc(sE, 128, 128, kSwizzleNone));
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint64_t ad = make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
+                        const uint64_t bd =
+                            make_smem_desc(sB + (j >> 1) * (BLOCK_N * 128) + (j & 1) * 64, 16, 1024, kSwizzle128B);
+                        umma_bf16_sp(tmem_base, ad, bd, e_tmem + (j & 2), idesc_sp | (j & 1), (i | j) != 0 ? 1u : 0u);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint64_t ad = p.a2_mn_major ? make_smem_desc(sA + j * 2048, 8192, 1024, kSwizzle128B)
+                                                          : make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
+                        const uint64_t bd = make_smem_desc(sB + j * 32, 16, 1024, kSwizzle128B);
+                        umma_bf16(tmem_base, ad, bd, idesc_ad, (i | j) != 0 ? 1u : 0u);
+                    }
+                }
+                umma_commit(&emptyA[pa.stage]);
+                umma_commit(&emptyB[pb.stage]);
+                pa.advance(A_STAGES);
+                pb.advance(B_STAGES);
+            }
+            if (ok) umma_commit(&tfull_bar[0]);
+        }
+    } else if (warp == 2) {
+        // ---------------------------------------------------------- activation ring
+        if (elect_one()) {
+            PipeState ps;
+            for (int i = 0; i < total_kb; ++i) {
+                if (!mbar_wait(&emptyB[ps.stage], ps.phase ^ 1u, abort_flag)) break;
+                uint8_t* sB = smem + Cfg::kOffB + ps.stage * Cfg::kBStage;
+                uint64_t* bar = &fullB[ps.stage];
+                if (i < num_sb) {
+                    const int kb = kb0 + i;
+                    mbar_expect_tx(bar, Cfg::kBStage);
+                    tma_load_2d(sB, &tmB, bar, kb * 128, 0);
+                    tma_load_2d(sB + BLOCK_N * 128, &tmB, bar, kb * 128 + 64, 0);
+                } else {
+                    mbar_expect_tx(bar, BLOCK_N * 128);
+                    tma_load_2d(sB, &tmB2, bar, (i - num_sb) * 64, 0);
+                }
+                ps.advance(B_STAGES);
+            }
+        }
+        __syncwarp();
+    }
+
+    // ---------------------------------------------------------------- epilogue (warps 2..5)
+    // Park the fp32 partial tile in shared memory as [token][feature]; the pipeline buffers are
+    // free once the last MMA has completed (tfull).  A rank with no k-block contributes zeros.
+    float* partial = reinterpret_cast<float*>(smem);
+    bool ok = true;
+    if (warp >= 2) {
+        const int q = warp & 3;
+        if (total_kb > 0) ok = mbar_wait(&tfull_bar[0], 0u, abort_flag);
+        tc_fence_after_sync();
+        const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+        const int ncols = min(BLOCK_N, (p.Ntok + 15) & ~15);         // columns past the last token are never read
+#pragma unroll 1
+        for (int c0 = 0; c0 < ncols; c0 += 16) {
+            uint32_t v[16];
+            if (total_kb > 0 && ok) {
+                tmem_ld_16(t_row + c0, v);
+                tmem_ld_wait();
+            } else {
+#pragma unroll
+                for (int c = 0; c < 16; ++c) v[c] = 0u;
+            }
+#pragma unroll
+            for (int c = 0; c < 16; ++c) partial[(c0 + c) * kBlockM + q * 32 + lane] = __uint_as_float(v[c]);
+        }
+        tc_fence_before_sync();
+    }
+    __syncthreads();
+    cluster_sync_all();                                       // every rank's partial tile is in place
+
+    // Token rows are dealt round-robin to the ranks.  One warp sums one token row at a time: a
+    // lane owns four consecutive features, fetches its 16 bytes from every rank's partial tile
+    // (all S loads in flight together) and adds them in rank order.
+    if (!*abort_flag) {
+        const int ntok = min(p.Ntok, BLOCK_N);
+        const int mine = ntok > rank ? (ntok - rank + splits - 1) / splits : 0;
+        const uint32_t my_partial = smem_u32(partial);
+        for (int i = warp; i < mine; i += kGemmThreads / 32) {
+            const int n = rank + i * splits;
+            const uint32_t off = my_partial + static_cast<uint32_t>(n * kBlockM + lane * 4) * 4u;
+            float4 v[8];
+#pragma unroll
+            for (int s = 0; s < 8; ++s)
+                if (s < splits) v[s] = ld_shared_cluster_v4(mapa_shared(off, s));
+            float4 acc = v[0];
+#pragma unroll
+            for (int s = 1; s < 8; ++s)
+                if (s < splits) { acc.x += v[s].x; acc.y += v[s].y; acc.z += v[s].z; acc.w += v[s].w; }
+            uint2 o;
+            o.x = pack_bf16x2(acc.x, acc.y);
+            o.y = pack_bf16x2(acc.z, acc.w);
+            *reinterpret_cast<uint2*>(p.out + static_cast<size_t>(n) * p.M + m_blk * kBlockM + lane * 4) = o;
+        }
+    }
+    if (*abort_flag) drain_after_abort();
+    cluster_sync_all();                                       // peers may still be reading this CTA's tile
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, Cfg::kTmemCols);
     }
 }
 

@@ -96,25 +96,64 @@ static bool make_tmap_plain(CUtensorMap* tm, const void* base, int rows, int col
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Launch on clusters of two CTAs (cta_group::2 kernels).
+// Launch with thread-block clusters of `cluster` CTAs along x.
 template <typename... KArgs, typename... Args>
-static slope_status_t launch_pairs(void (*kern)(KArgs...), int grid, int threads, int smem_bytes,
-                                   cudaStream_t stream, Args&&... args) {
+static slope_status_t launch_cluster_ex(void (*kern)(KArgs...), int grid, int cluster, int threads, int smem_bytes,
+                                        bool overlap_prologue, cudaStream_t stream, Args&&... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid, 1, 1);
     cfg.blockDim = dim3(threads, 1, 1);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    // Programmatic dependent launch: the kernel may be scheduled while its predecessor in the
+    // stream drains; it synchronises on the device (griddepcontrol.wait) before touching memory.
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap_prologue ? 2 : 1;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? SLOPE_OK : SLOPE_ERR_CUDA;
+}
+
+template <typename... KArgs, typename... Args>
+static slope_status_t launch_cluster(void (*kern)(KArgs...), int grid, int cluster, int threads, int smem_bytes,
+                                     cudaStream_t stream, Args&&... args) {
+    return launch_cluster_ex(kern, grid, cluster, threads, smem_bytes, false, stream, std::forward<Args>(args)...);
+}
+
+// How many clusters of `cluster` CTAs of this kernel the device holds at once (0: query failed).
+template <typename Kernel>
+static int max_active_clusters(Kernel kern, int cluster, int threads, int smem_bytes, int sm_count) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cluster * sm_count, 1, 1);
+    cfg.blockDim = dim3(threads, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes;
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.x = cluster;
     attr.val.clusterDim.y = 1;
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    const cudaError_t err = cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? SLOPE_OK : SLOPE_ERR_CUDA;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    return n;
+}
+
+// Launch on clusters of two CTAs (cta_group::2 kernels).
+template <typename... KArgs, typename... Args>
+static slope_status_t launch_pairs(void (*kern)(KArgs...), int grid, int threads, int smem_bytes,
+                                   cudaStream_t stream, Args&&... args) {
+    return launch_cluster(kern, grid, 2, threads, smem_bytes, stream, std::forward<Args>(args)...);
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -245,13 +284,92 @@ static slope_status_t launch_sparse_quad(const void* act, int ntok, const void* 
     return launch_pairs(kern, 2 * pairs, Cfg::kThreads, Cfg::kSmemBytes, stream, tmA, tmB, tmE, tmA2, tmB2, tmO, p);
 }
 
-// Tile choice for the sparse GEMMs.  The 512-row tile moves 31 % fewer L2 bytes per FLOP but
+// Few tokens (inference / decode sizes): weight-streaming kernel, K split over a cluster.
+// K-splits (= cluster size) of the few-token kernel.  A CTA streams ceil(num_kb / s) k-blocks
+// of 18 KB.  Measured on B200: alone an SM takes in one k-block per ~0.23 us (about one TMA row
+// request per 2 ns), and once enough CTAs pull at the same time HBM is the limit (18 KB at
+// 6.5 TB/s = 0.0028 us per k-block and active CTA).  Every wave of clusters pays a fixed
+// start-up (launch, prologue, first-byte latency, epilogue), a split pays the cluster
+// reduction.  `capacity(s)` is the number of clusters of s CTAs the device holds at once.
+constexpr double kSkinnySmUs = 0.23, kSkinnyHbmUs = 0.0028, kSkinnyWaveUs = 4.0, kSkinnyReduceUs = 0.5,
+                 kSkinnyReducePerRankUs = 0.07;
+
+template <typename Capacity>
+static int skinny_splits(int slabs, int num_kb, Capacity capacity) {
+    int best_s = 1;
+    double best_cost = 1e30;
+    for (int s = 1; s <= 8; ++s) {
+        const int per = (num_kb + s - 1) / s;
+        if ((num_kb + per - 1) / per != s) continue;                 // a rank would be left without a k-block
+        if (s > 1 && per < 2) break;
+        const int cap = capacity(s);
+        if (cap <= 0) continue;
+        double cost = s > 1 ? kSkinnyReduceUs + kSkinnyReducePerRankUs * s : 0.0;
+        for (int left = slabs; left > 0; left -= cap) {
+            const int active = (left < cap ? left : cap) * s;
+            const double per_kb = active * kSkinnyHbmUs > kSkinnySmUs ? active * kSkinnyHbmUs : kSkinnySmUs;
+            cost += kSkinnyWaveUs + per * per_kb;
+        }
+        if (cost < best_cost - 1e-9) { best_cost = cost; best_s = s; }
+    }
+    return best_s;
+}
+
+template <int BLOCK_N, int A_STAGES, int B_STAGES>
+static slope_status_t launch_sparse_skinny(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
+                                           const void* act2, const void* fac2, int r, bool a2_mn, void* out,
+                                           cudaStream_t stream, const DeviceInfo& info) {
+    using Cfg = SparseSkinnyCfg<BLOCK_N, A_STAGES, B_STAGES>;
+    CUtensorMap tmA, tmB, tmE, tmA2, tmB2;
+    if (!make_tmap(&tmA, vals, M, K / 2, kBlockM, 64)) return SLOPE_ERR_CUDA;
+    if (!make_tmap(&tmB, act, ntok, K, BLOCK_N, 64)) return SLOPE_ERR_CUDA;
+    if (!make_tmap_meta(&tmE, meta, static_cast<size_t>(M) * K / 8)) return SLOPE_ERR_CUDA;
+    if (r > 0) {
+        const bool ok2 = a2_mn ? make_tmap(&tmA2, fac2, r, M, 64, 64) : make_tmap(&tmA2, fac2, M, r, kBlockM, 64);
+        if (!ok2 || !make_tmap(&tmB2, act2, ntok, r, BLOCK_N, 64)) return SLOPE_ERR_CUDA;
+    } else {
+        tmA2 = tmA;
+        tmB2 = tmB;
+    }
+    SparseGemmParams p;
+    p.M = M; p.K = K; p.Ntok = ntok; p.r = r; p.a2_mn_major = a2_mn ? 1 : 0;
+    p.meta = static_cast<const uint8_t*>(meta);
+    p.out = static_cast<uint16_t*>(out);
+    auto kern = sparse_gemm_skinny_kernel<BLOCK_N, A_STAGES, B_STAGES>;
+    if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
+
+    // co-resident clusters per cluster size, asked of the driver once per device
+    static std::mutex mu;
+    static int capacity[64][9];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SLOPE_ERR_CUDA;
+    int cap[9];
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (capacity[dev][1] == 0)
+            for (int s = 1; s <= 8; ++s)
+                capacity[dev][s] = max_active_clusters(kern, s, kGemmThreads, Cfg::kSmemBytes, info.sm_count);
+        for (int s = 1; s <= 8; ++s) cap[s] = capacity[dev][s];
+    }
+    if (cap[1] <= 0) return SLOPE_ERR_CUDA;
+    const int slabs = M / kBlockM, num_kb = K / 128;
+    int splits = skinny_splits(slabs, num_kb, [&](int s) { return cap[s]; });
+    return launch_cluster_ex(kern, slabs * splits, splits, kGemmThreads, Cfg::kSmemBytes, true, stream, tmA, tmB,
+                             tmE, tmA2, tmB2, p);
+}
+
+// Kernel choice for the sparse GEMMs.  Up to 256 tokens the GEMM is a weight stream from HBM and
+// runs on the skinny kernel.  Beyond that: the 512-row tile moves 31 % fewer L2 bytes per FLOP but
 // cannot overlap its epilogue with the next tile (tensor memory holds only one accumulator
 // set); that pays off once the reduction is long.  Short reductions keep the 256-row tile
 // with double-buffered accumulators.
 static slope_status_t launch_sparse_gemm(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                          const void* act2, const void* fac2, int r, bool a2_mn, void* out,
                                          cudaStream_t stream, const DeviceInfo& info) {
+    if (ntok <= 16) return launch_sparse_skinny<16, 10, 4>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
+    if (ntok <= 64) return launch_sparse_skinny<64, 8, 4>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
+    if (ntok <= 128) return launch_sparse_skinny<128, 7, 3>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
+    if (ntok <= 256) return launch_sparse_skinny<256, 5, 2>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
     return K >= 6144 ? launch_sparse_quad(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info)
                      : launch_sparse_pair(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
 }

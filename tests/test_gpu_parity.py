@@ -107,6 +107,13 @@ CASES = [
     (128, 128, 8, 16, 15),           # smallest legal problem
     (6144, 640, 264, 32, 16),        # forward reduction long enough for the 512-row-tile kernel
     (640, 6144, 264, 0, 17),         # same for the input-gradient GEMM
+    (4096, 512, 40, 16, 18),         # few tokens: weight-streaming kernel (64-token tile), K split over a cluster
+    (1024, 384, 200, 0, 19),         # 200 tokens (256-token tile)
+    (2048, 256, 64, 64, 20),         # exactly one 64-token tile with adapters
+    (256, 2048, 128, 32, 21),        # 128-token tile; dX has the long reduction
+    (1024, 512, 8, 64, 22),          # decode size: 16-token tile with adapters
+    (512, 1536, 16, 128, 23),        # 16 tokens, two adapter K-steps
+    (1152, 384, 104, 128, 24),       # 128-token tile, ragged, two adapter K-steps, odd number of k-blocks
 ]
 
 
@@ -146,6 +153,49 @@ def test_layer_against_oracle(B, oracle, d_in, d_out, b, r, seed):
     print(errs)
     for k, v in errs.items():
         assert v <= REL_TOL, (k, v, errs)
+
+
+def test_few_token_forward_in_a_cuda_graph_matches_eager_bitwise(B, oracle):
+    """The few-token kernel opts in to programmatic dependent launch; a captured chain of
+    launches (each reading the previous one's output) must replay to the eager result."""
+    import torch
+
+    d, b = 512, 8
+    Ws = [si.gaussian_bf16((d, d), 0.05, 40 + i) for i in range(3)]
+    layers = [GpuLayer(W) for W in Ws]
+    X = si.gaussian_bf16((b, d), 1.0, 44)
+    Xd = dev(B, X)
+
+    def chain(outs):
+        h = Xd
+        for layer, o in zip(layers, outs):
+            B.slope_linear_fwd(h, layer.Wc_vals, layer.Wc_meta, d, o)
+            h = o
+
+    eager = [torch.empty((b, d), dtype=torch.bfloat16, device="cuda") for _ in layers]
+    chain(eager)
+    torch.cuda.synchronize()
+    captured = [torch.zeros((b, d), dtype=torch.bfloat16, device="cuda") for _ in layers]
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        chain(captured)                       # warm-up outside the capture
+        stream.synchronize()
+        for o in captured:
+            o.zero_()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            chain(captured)
+    torch.cuda.synchronize()
+    for o in captured:
+        o.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    layers[0].poll()
+    for e, c in zip(eager, captured):
+        assert np.array_equal(B.bits_from_bf16(e), B.bits_from_bf16(c))
+    # and the chain's first link against the oracle
+    mask1, _ = check_selection(oracle, layers[0], Ws[0])
+    assert rel_fro(to_f64(B.bits_from_bf16(eager[0])), oracle.fwd_rows(X, Ws[0], mask1, np.arange(b), None, None)) <= REL_TOL
 
 
 def test_no_adapter_path_is_bitwise_the_rank0_path_and_deterministic(B, oracle):
