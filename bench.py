@@ -442,6 +442,7 @@ def main():
     if rank == 0 and not args.no_extras and world == 1:
         out["optimizer_tail"] = optimizer_tail_probe(torch, B, layers, stream, pk)
         out["burst"] = burst_probe(torch, B, layers, stream, pk)
+        out["inference_forward"] = inference_forward_probe(torch, B, wl, pk)
         out["dense_layer"] = dense_comparison(torch, B, layers, stream)
         out["e2e"] = e2e_run(torch, B, layers, de_flops, max(2, min(args.steps, 5)))
         out["cpu_baseline"] = cpu_baseline_sample(wl)
@@ -485,6 +486,82 @@ def optimizer_tail_probe(torch, B, layers, stream, pk, reps=20):
     return {"what": f"{reps} back-to-back launches, CUDA events; bytes: sparse_add 3 B and update 2.25 B per weight "
                     f"element; HBM peak {pk['hbm_gbs']} GB/s ({pk['src']}); the working set of sparse_add "
                     f"({3 * n / 1e6:.0f} MB) partly lives in the 126 MB L2 across launches", "rows": rows}
+
+
+def inference_forward_probe(torch, B, wl, pk, copies=12, reps=5):
+    """Forward only at decode sizes (8 and 64 tokens), without and with adapters (the workload's
+    rank, else 64 = 1.56 % of 4096, and 256 = 6.25 %): the GEMM is a stream of compressed weights
+    from HBM.  Each shape is timed as a CUDA graph of `copies` launches over distinct weight
+    copies (together larger than L2), best of `reps` replays; cuBLAS on the dense bf16 weight
+    in the same harness for comparison."""
+    dev = torch.device("cuda")
+    shapes = []
+    for lay in wl.layers:
+        if (lay.d_in, lay.d_out) not in shapes:
+            shapes.append((lay.d_in, lay.d_out))
+    ranks = [0, wl.rank if wl.rank else 64, 256]
+
+    def time_graph(fn):
+        side = torch.cuda.Stream()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            fn(); fn()
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                fn()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); graph.replay(); e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        return best * 1e3 / copies                         # microseconds per layer call
+
+    rows = []
+    for d_in, d_out in shapes[:3]:
+        W = B.bf16_from_bits(si.gaussian_bf16((d_out, d_in), 0.02, si.seed_for(9, 0, "W")), dev)
+        vals, meta, _ = B.alloc_compressed(d_out, d_in, dev)
+        B.slope_prune_24(W, vals, meta, None)
+        Wc = [(vals.clone(), meta.clone()) for _ in range(copies)]
+        Wd = [W.clone() for _ in range(copies)]
+        for b in (8, 64):
+            X = B.bf16_from_bits(si.gaussian_bf16((b, d_in), 1.0, si.seed_for(9, 0, "X")), dev)
+            Y = torch.empty((b, d_out), dtype=torch.bfloat16, device=dev)
+            us_dense = time_graph(lambda: [torch.matmul(X, w.t(), out=Y) for w in Wd])
+            for r in ranks:
+                if r:
+                    L = B.bf16_from_bits(si.gaussian_bf16((d_in, r), 0.01, si.seed_for(9, 0, "L")), dev)
+                    R = B.bf16_from_bits(si.gaussian_bf16((r, d_out), 0.01, si.seed_for(9, 0, "R")), dev)
+                    T = torch.empty((b, r), dtype=torch.bfloat16, device=dev)
+
+                    def run():
+                        for v, m in Wc:
+                            B.slope_adapter_fwd_bwd(0, X, None, L, None, b, d_out, d_in, r, T=T)
+                            B.slope_linear_fwd(X, v, m, d_out, Y, T, R)
+                else:
+                    def run():
+                        for v, m in Wc:
+                            B.slope_linear_fwd(X, v, m, d_out, Y)
+                us = time_graph(run)
+                nbytes = d_in * d_out * 1.125 + 2.0 * b * (d_in + d_out) + 2.0 * r * (d_in + d_out) + 4.0 * b * r
+                gbs = nbytes / (us * 1e-6) / 1e9
+                rows.append({"d_in": d_in, "d_out": d_out, "tokens": b, "rank": r, "us": round(us, 2),
+                             "algorithmic_bytes": int(nbytes), "gbs": round(gbs, 1),
+                             "frac_of_hbm_peak": round(gbs / pk["hbm_gbs"], 4),
+                             "cublas_dense_us": round(us_dense, 2), "speedup_vs_cublas_dense": round(us_dense / us, 3)})
+        del Wc, Wd
+    st = B.slope_poll_status()
+    if st != 0:
+        raise SystemExit(f"device status after the inference probe: {B.slope_status_string(st)}")
+    return {"what": f"forward only (adapter T = X L + fused sparse GEMM), CUDA graph of {copies} calls over distinct "
+                    f"weight copies, best of {reps} replays, us per call; bytes: 1.125 B per weight element "
+                    f"(values + metadata) + activations + adapter factors; HBM peak {pk['hbm_gbs']} GB/s "
+                    f"({pk['src']}); cuBLAS reads the dense bf16 weight (2 B per element, no adapter)",
+            "rows": rows}
 
 
 def burst_probe(torch, B, layers, stream, pk, launches=8):

@@ -1071,7 +1071,12 @@ sparse_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
     const int kb_per = (num_kb + splits - 1) / splits;
     const int kb0 = min(num_kb, rank * kb_per), kb1 = min(num_kb, kb0 + kb_per);
     const int num_sb = kb1 - kb0;                                            // sparse k-blocks of this rank
-    const int num_ab = rank == splits - 1 ? (p.r + 63) / 64 : 0;            // adapter K-steps on the last rank
+    // Dense K-steps (64 wide): the adapter product rides on the last rank; with no sparse part
+    // at all (K == 0: a plain few-token dense GEMM) they are split over the ranks instead.
+    const int all_ab = (p.r + 63) / 64;
+    const int ab_per = num_kb == 0 ? (all_ab + splits - 1) / splits : all_ab;
+    const int ab0 = num_kb == 0 ? min(all_ab, rank * ab_per) : 0;
+    const int num_ab = num_kb == 0 ? min(all_ab, ab0 + ab_per) - ab0 : (rank == splits - 1 ? all_ab : 0);
     const int total_kb = num_sb + num_ab;
 
     if (threadIdx.x == 0) {
@@ -1114,7 +1119,7 @@ sparse_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
                     tma_load_2d_hint(sA, &tmA, bar, kb * 64, m_blk * kBlockM, stream_once);
                     tma_load_2d_hint(sA + Cfg::kABytes, &tmE, bar, 0, m_blk * num_kb + kb, stream_once);
                 } else {
-                    const int ab = i - num_sb;
+                    const int ab = ab0 + i - num_sb;
                     mbar_expect_tx(bar, Cfg::kABytes);
                     if (p.a2_mn_major) {
                         tma_load_2d(sA, &tmA2, bar, m_blk * kBlockM, ab * 64);
@@ -1181,7 +1186,7 @@ sparse_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
                     tma_load_2d(sB + BLOCK_N * 128, &tmB, bar, kb * 128 + 64, 0);
                 } else {
                     mbar_expect_tx(bar, BLOCK_N * 128);
-                    tma_load_2d(sB, &tmB2, bar, (i - num_sb) * 64, 0);
+                    tma_load_2d(sB, &tmB2, bar, (ab0 + i - num_sb) * 64, 0);
                 }
                 ps.advance(B_STAGES);
             }
@@ -1239,7 +1244,8 @@ sparse_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
             uint2 o;
             o.x = pack_bf16x2(acc.x, acc.y);
             o.y = pack_bf16x2(acc.z, acc.w);
-            *reinterpret_cast<uint2*>(p.out + static_cast<size_t>(n) * p.M + m_blk * kBlockM + lane * 4) = o;
+            const int m = m_blk * kBlockM + lane * 4;
+            if (m < p.M) *reinterpret_cast<uint2*>(p.out + static_cast<size_t>(n) * p.M + m) = o;
         }
     }
     if (*abort_flag) drain_after_abort();

@@ -321,13 +321,21 @@ static slope_status_t launch_sparse_skinny(const void* act, int ntok, const void
                                            cudaStream_t stream, const DeviceInfo& info) {
     using Cfg = SparseSkinnyCfg<BLOCK_N, A_STAGES, B_STAGES>;
     CUtensorMap tmA, tmB, tmE, tmA2, tmB2;
-    if (!make_tmap(&tmA, vals, M, K / 2, kBlockM, 64)) return SLOPE_ERR_CUDA;
-    if (!make_tmap(&tmB, act, ntok, K, BLOCK_N, 64)) return SLOPE_ERR_CUDA;
-    if (!make_tmap_meta(&tmE, meta, static_cast<size_t>(M) * K / 8)) return SLOPE_ERR_CUDA;
     if (r > 0) {
         const bool ok2 = a2_mn ? make_tmap(&tmA2, fac2, r, M, 64, 64) : make_tmap(&tmA2, fac2, M, r, kBlockM, 64);
         if (!ok2 || !make_tmap(&tmB2, act2, ntok, r, BLOCK_N, 64)) return SLOPE_ERR_CUDA;
-    } else {
+    }
+    if (K > 0) {
+        if (!make_tmap(&tmA, vals, M, K / 2, kBlockM, 64)) return SLOPE_ERR_CUDA;
+        if (!make_tmap(&tmB, act, ntok, K, BLOCK_N, 64)) return SLOPE_ERR_CUDA;
+        if (!make_tmap_meta(&tmE, meta, static_cast<size_t>(M) * K / 8)) return SLOPE_ERR_CUDA;
+    } else {                                  // dense-only: the sparse maps are never used for a load
+        if (r <= 0) return SLOPE_ERR_SHAPE;
+        tmA = tmA2;
+        tmB = tmB2;
+        tmE = tmA2;
+    }
+    if (r <= 0) {
         tmA2 = tmA;
         tmB2 = tmB;
     }
@@ -352,10 +360,25 @@ static slope_status_t launch_sparse_skinny(const void* act, int ntok, const void
         for (int s = 1; s <= 8; ++s) cap[s] = capacity[dev][s];
     }
     if (cap[1] <= 0) return SLOPE_ERR_CUDA;
-    const int slabs = M / kBlockM, num_kb = K / 128;
-    int splits = skinny_splits(slabs, num_kb, [&](int s) { return cap[s]; });
+    const int slabs = (M + kBlockM - 1) / kBlockM, num_kb = K > 0 ? K / 128 : (r + 63) / 64;
+    const int splits = skinny_splits(slabs, num_kb, [&](int s) { return cap[s]; });
     return launch_cluster_ex(kern, slabs * splits, splits, kGemmThreads, Cfg::kSmemBytes, true, stream, tmA, tmB,
                              tmE, tmA2, tmB2, p);
+}
+
+// Few-token GEMM  out[ntok x M] = act * A_2:4^T (+ act2 * fac2^T)  on the weight-streaming
+// kernel, token tile chosen by the token count.  K == 0 runs the dense product alone
+// (out = act2 * fac2^T with reduction length r), which serves the adapter's T = X L and
+// dT = dY R^T at inference sizes.
+constexpr int kSkinnyMaxTokens = 256;
+
+static slope_status_t launch_skinny(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
+                                    const void* act2, const void* fac2, int r, bool a2_mn, void* out,
+                                    cudaStream_t stream, const DeviceInfo& info) {
+    if (ntok <= 16) return launch_sparse_skinny<16, 10, 4>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
+    if (ntok <= 64) return launch_sparse_skinny<64, 8, 4>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
+    if (ntok <= 128) return launch_sparse_skinny<128, 7, 3>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
+    return launch_sparse_skinny<256, 5, 2>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
 }
 
 // Kernel choice for the sparse GEMMs.  Up to 256 tokens the GEMM is a weight stream from HBM and
@@ -366,10 +389,8 @@ static slope_status_t launch_sparse_skinny(const void* act, int ntok, const void
 static slope_status_t launch_sparse_gemm(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                          const void* act2, const void* fac2, int r, bool a2_mn, void* out,
                                          cudaStream_t stream, const DeviceInfo& info) {
-    if (ntok <= 16) return launch_sparse_skinny<16, 10, 4>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
-    if (ntok <= 64) return launch_sparse_skinny<64, 8, 4>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
-    if (ntok <= 128) return launch_sparse_skinny<128, 7, 3>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
-    if (ntok <= 256) return launch_sparse_skinny<256, 5, 2>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
+    if (ntok <= kSkinnyMaxTokens)
+        return launch_skinny(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
     return K >= 6144 ? launch_sparse_quad(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info)
                      : launch_sparse_pair(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
 }
@@ -414,7 +435,7 @@ static int adapter_splits(int b, int rows) {
 static bool dims_ok(int d_out, int d_in) {
     return d_out > 0 && d_in > 0 && d_out % 128 == 0 && d_in % 128 == 0;
 }
-static bool rank_ok(int r) { return r >= 0 && r <= 128 && r % 16 == 0; }
+static bool rank_ok(int r) { return r >= 0 && r <= 256 && r % 16 == 0; }
 
 }  // namespace slope
 
@@ -548,6 +569,8 @@ slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY, c
         if (!aligned16(X) || !aligned16(L) || !aligned16(T)) return SLOPE_ERR_ALIGNMENT;
         if (slope_status_t st = check_arch(info)) return st;
         // T[b x r] = X[b x d_in] * L[d_in x r]   (A = X, K contiguous; B = L^T stored [K x N])
+        if (b <= kSkinnyMaxTokens)            // few tokens: split d_in over a cluster instead of one CTA
+            return launch_skinny(nullptr, b, nullptr, nullptr, r, 0, X, L, d_in, true, T, stream, info);
         return r <= 64 ? launch_dense<false, true, 64, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info)
                        : launch_dense<false, true, 128, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info);
     }
@@ -559,7 +582,9 @@ slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY, c
     if (slope_status_t st = check_arch(info)) return st;
     slope_status_t st;
     // dT[b x r] = dY[b x d_out] * R[r x d_out]^T   (both K contiguous)
-    st = r <= 64 ? launch_dense<false, false, 64, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info)
+    st = b <= kSkinnyMaxTokens
+             ? launch_skinny(nullptr, b, nullptr, nullptr, r, 0, dY, R, d_out, false, dT, stream, info)
+         : r <= 64 ? launch_dense<false, false, 64, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info)
                  : launch_dense<false, false, 128, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info);
     if (st) return st;
     // dL[d_in x r] = X^T dT and dR^T[d_out x r] = dY^T T: operands stored [K x M] / [K x N] with

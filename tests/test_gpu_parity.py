@@ -114,6 +114,8 @@ CASES = [
     (1024, 512, 8, 64, 22),          # decode size: 16-token tile with adapters
     (512, 1536, 16, 128, 23),        # 16 tokens, two adapter K-steps
     (1152, 384, 104, 128, 24),       # 128-token tile, ragged, two adapter K-steps, odd number of k-blocks
+    (512, 768, 264, 256, 25),        # largest rank (6.25 % of a 4096-wide layer): two adapter column tiles
+    (1024, 512, 16, 256, 26),        # largest rank at decode size
 ]
 
 
