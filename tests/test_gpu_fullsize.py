@@ -77,3 +77,36 @@ def test_full_size_layer(B, oracle, key, idx):
     # finite everywhere, not just on the sample
     for tns in (Y, dX, dWc):
         assert bool(torch.isfinite(tns.float()).all())
+
+
+INFERENCE_CASES = [
+    ("c4_llama7b_adapter", 0, 8), ("c4_llama7b_adapter", 4, 8), ("c4_llama7b_adapter", 6, 8),
+    ("c4_llama7b_adapter", 0, 64), ("c4_llama7b_adapter", 6, 64), ("c5_llama13b_block", 4, 16),
+]
+
+
+@pytest.mark.parametrize("key,idx,tokens", INFERENCE_CASES)
+def test_full_size_inference_forward(B, oracle, key, idx, tokens):
+    """Forward only at decode sizes on full-size layers (the few-token kernel with its K-split over
+    a cluster): every output element against the oracle, without and with the adapters."""
+    wl = si.WORKLOADS[key]
+    lay = wl.layers[idx]
+    t = si.layer_tensors(wl, idx, tokens=tokens)
+    W, X, L, R = t["W"], t["X"], t.get("L"), t.get("R")
+    layer = GpuLayer(W)
+    _, _, mask1 = oracle.prune24(W)
+    assert np.array_equal(layer.mask1.cpu().numpy(), mask1)
+    Xd = B.bf16_from_bits(X)
+    rows = np.arange(tokens)
+    Y0 = layer.fwd(Xd)
+    errs = {"Y": rel_fro(to_f64(B.bits_from_bf16(Y0)), oracle.fwd_rows(X, W, mask1, rows, None, None))}
+    if wl.rank:
+        Ld, Rd = B.bf16_from_bits(L), B.bf16_from_bits(R)
+        T = layer.adapter_T(Xd, Ld)
+        Y1 = layer.fwd(Xd, T, Rd)
+        errs["T"] = rel_fro(to_f64(B.bits_from_bf16(T)), oracle.adapter_T_rows(X, L, rows))
+        errs["Y+adapter"] = rel_fro(to_f64(B.bits_from_bf16(Y1)), oracle.fwd_rows(X, W, mask1, rows, L, R))
+    layer.poll()
+    print(key, lay.name, tokens, errs)
+    for k, v in errs.items():
+        assert v <= REL_TOL, (k, v, errs)
