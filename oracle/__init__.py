@@ -124,6 +124,29 @@ def decompress(vals: np.ndarray, nib: np.ndarray) -> np.ndarray:
     return dense
 
 
+def prune_nm(W: np.ndarray, n: int, m: int):
+    """O9: general N:M first pass.  Returns (WR[d_out,d_in] u16 dense with +0 at pruned entries, mask1)."""
+    W = _u16(W)
+    d_out, d_in = W.shape
+    assert 0 < n < m <= 64 and d_in % m == 0 and d_in % 8 == 0
+    WR = np.empty((d_out, d_in), np.uint16)
+    mask = np.empty((d_out, d_in // 8), np.uint8)
+    _load().slope_oracle_prune_nm(_p(W), d_out, d_in, n, m, _p(WR), _p(mask))
+    return WR, mask
+
+
+def double_prune_nm(W: np.ndarray, mask1: np.ndarray, n: int, m: int):
+    """O10: general N:M second pass along the columns.  Returns (WRC[d_out,d_in] u16 dense, mask2)."""
+    W = _u16(W)
+    mask1 = _u8(mask1)
+    d_out, d_in = W.shape
+    assert 0 < n < m <= 64 and d_out % m == 0 and mask1.shape == (d_out, d_in // 8)
+    WRC = np.empty((d_out, d_in), np.uint16)
+    mask2 = np.empty((d_out, d_in // 8), np.uint8)
+    _load().slope_oracle_double_prune_nm(_p(W), _p(mask1), d_out, d_in, n, m, _p(WRC), _p(mask2))
+    return WRC, mask2
+
+
 def mask_to_bool(mask: np.ndarray, cols: int) -> np.ndarray:
     """Bit mask (LSB-first bytes) -> boolean [rows, cols]."""
     return np.unpackbits(np.asarray(mask, np.uint8), axis=1, bitorder="little")[:, :cols].astype(bool)

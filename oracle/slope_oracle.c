@@ -14,7 +14,9 @@
  * selection rule, structural invariants, Lemma 1's closed form (9.375 % extra
  * zeros for 2:4), numpy fp64 matmul on the masked dense matrices, central
  * finite differences on tiny inputs, and the fused-adapter identity of
- * Eq. (concat).
+ * Eq. (concat).  The general N:M passes (O9, O10) are pinned by subset
+ * enumeration on tie-heavy groups, by agreement with the 2:4 path, and by
+ * Eq. (sparsity_ratio) for seven (N, M) patterns on Gaussian data.
  *
  * Conventions
  *   W  [d_out x d_in]   weight (Sec. "Sparse Plus Low-rank Pretraining")
@@ -371,6 +373,73 @@ void slope_oracle_update_transposed(const uint16_t *Wc_new, const uint8_t *mask1
                     v = Wc_new[i * (d_in / 2) + 2 * g + rank];
                 }
                 valsT[j * (d_out / 2) + 2 * h + t] = v;
+            }
+        }
+}
+
+/* Choose the n largest of m 15-bit magnitudes, one at a time: each round takes the
+ * largest magnitude not taken yet, the lowest position among equals.  taken[t] = 1
+ * for the kept positions. */
+static void topn_of_m(const uint32_t *key, int n, int m, int *taken) {
+    for (int t = 0; t < m; ++t) taken[t] = 0;
+    for (int round = 0; round < n; ++round) {
+        int best = -1;
+        for (int t = 0; t < m; ++t) {
+            if (taken[t]) continue;
+            if (best < 0 || key[t] > key[best]) best = t;     /* strict: lower index wins ties */
+        }
+        taken[best] = 1;
+    }
+}
+
+/* O9 -- general N:M first pass (Lemma 1's "row-wise N:M pruned" A^R; the accuracy
+ * experiments emulate N:M by pruning the dense weight): in every group of m
+ * consecutive entries of a row keep the n of largest magnitude.  Output is the
+ * dense matrix with the pruned entries set to +0, and the bit mask. */
+void slope_oracle_prune_nm(const uint16_t *W, int d_out, int d_in, int n, int m,
+                           uint16_t *WR, uint8_t *mask1)
+{
+    long mrow = d_in / 8;
+    memset(mask1, 0, (size_t)d_out * mrow);
+    for (long i = 0; i < d_out; ++i)
+        for (long g = 0; g < d_in / m; ++g) {
+            uint32_t key[64];
+            int taken[64];
+            for (int t = 0; t < m; ++t) key[t] = W[i * d_in + m * g + t] & 0x7FFFu;
+            topn_of_m(key, n, m, taken);
+            for (int t = 0; t < m; ++t) {
+                long j = m * g + t;
+                WR[i * d_in + j] = taken[t] ? W[i * d_in + j] : (uint16_t)0;
+                if (taken[t]) mask1[i * mrow + (j >> 3)] |= (uint8_t)(1u << (j & 7));
+            }
+        }
+}
+
+/* O10 -- general N:M second pass (Lemma 1's A^{R,C}): on the row-wise pruned
+ * matrix, in every group of m consecutive entries of a COLUMN keep the n of
+ * largest magnitude; entries the first pass removed enter with magnitude zero.
+ * Output is dense, in W's orientation; mask2 = kept by both passes. */
+void slope_oracle_double_prune_nm(const uint16_t *W, const uint8_t *mask1, int d_out, int d_in,
+                                  int n, int m, uint16_t *WRC, uint8_t *mask2)
+{
+    long mrow = d_in / 8;
+    memset(mask2, 0, (size_t)d_out * mrow);
+    for (long j = 0; j < d_in; ++j)
+        for (long h = 0; h < d_out / m; ++h) {
+            uint32_t key[64];
+            uint16_t v[64];
+            int kept1[64], taken[64];
+            for (int t = 0; t < m; ++t) {
+                long i = m * h + t;
+                kept1[t] = mask_get(mask1, mrow, i, j);
+                v[t] = kept1[t] ? W[i * d_in + j] : (uint16_t)0;
+                key[t] = v[t] & 0x7FFFu;
+            }
+            topn_of_m(key, n, m, taken);
+            for (int t = 0; t < m; ++t) {
+                long i = m * h + t;
+                WRC[i * d_in + j] = taken[t] ? v[t] : (uint16_t)0;
+                if (taken[t] && kept1[t]) mask2[i * mrow + (j >> 3)] |= (uint8_t)(1u << (j & 7));
             }
         }
 }

@@ -347,3 +347,87 @@ def test_update_transposed_reproduces_double_prune(oracle):
         rows = 4 * np.arange(64)[None, :] + q
         sel[:, t::2] = m2T[np.arange(384)[:, None], rows]
     assert np.array_equal(out != 0, sel)
+
+
+# ----------------------------------------------------------------------------- P9: general N:M (O9, O10)
+NM_PATTERNS = [(1, 2), (2, 4), (1, 4), (2, 8), (4, 8), (3, 8), (4, 16)]
+
+
+def _brute_force_group(keys, n):
+    """All n-subsets of one group: largest sum of magnitudes, ties -> lexicographically smallest."""
+    best, best_sum = None, -1
+    for comb in itertools.combinations(range(len(keys)), n):
+        s = int(sum(int(keys[t]) for t in comb))
+        if s > best_sum:                                  # combinations come in lexicographic order
+            best, best_sum = comb, s
+    return best
+
+
+def test_p9_nm_equals_the_2_4_path(oracle):
+    W = si.gaussian_bf16((64, 128), 0.02, 91)
+    vals, nib, mask1 = oracle.prune24(W)
+    WR, m1 = oracle.prune_nm(W, 2, 4)
+    assert np.array_equal(m1, mask1)
+    keep = oracle.mask_to_bool(mask1, 128)
+    assert np.array_equal(WR, np.where(keep, W, 0).astype(np.uint16))
+    assert np.array_equal(WR[keep].reshape(64, 64), vals)
+    _, _, mask2 = oracle.double_prune(W, mask1)
+    WRC, m2 = oracle.double_prune_nm(W, m1, 2, 4)
+    assert np.array_equal(m2, mask2)
+    assert np.array_equal(WRC, np.where(oracle.mask_to_bool(mask2, 128), W, 0).astype(np.uint16))
+
+
+@pytest.mark.parametrize("n,m", NM_PATTERNS)
+def test_p9_nm_brute_force_with_ties(oracle, n, m):
+    """Tie-heavy alphabet (few distinct magnitudes, both signs and zeros) against subset enumeration,
+    for both passes."""
+    rng = np.random.Generator(np.random.PCG64(900 + 10 * m + n))
+    alphabet = si.f32_to_bf16_bits(np.array([0.0, -0.0, 0.5, -0.5, 1.0, -1.0, 1.5, 3.0], np.float32))
+    d_out, d_in = 2 * m, 16 * max(1, m // 8) * 2
+    d_in = max(d_in, 2 * m)
+    W = rng.choice(alphabet, size=(d_out, d_in)).astype(np.uint16)
+    WR, mask1 = oracle.prune_nm(W, n, m)
+    keep1 = oracle.mask_to_bool(mask1, d_in)
+    key = (W & 0x7FFF).astype(np.int64)
+    for i in range(d_out):
+        for g in range(d_in // m):
+            want = _brute_force_group(key[i, m * g:m * g + m], n)
+            got = tuple(np.flatnonzero(keep1[i, m * g:m * g + m]))
+            assert got == want, (i, g, key[i, m * g:m * g + m], got, want)
+    assert np.array_equal(WR, np.where(keep1, W, 0).astype(np.uint16))
+    WRC, mask2 = oracle.double_prune_nm(W, mask1, n, m)
+    keep2 = oracle.mask_to_bool(mask2, d_in)
+    keyR = np.where(keep1, key, 0)
+    for j in range(d_in):
+        for h in range(d_out // m):
+            col = keyR[m * h:m * h + m, j]
+            want = set(_brute_force_group(col, n))
+            got = set(np.flatnonzero(keep2[m * h:m * h + m, j]))
+            # second-pass picks that the first pass had removed (zeros filling up the n slots) are not in mask2
+            assert got == {t for t in want if keep1[m * h + t, j]}, (j, h, col, got, want)
+    assert np.array_equal(WRC, np.where(keep2, W, 0).astype(np.uint16))
+
+
+@pytest.mark.parametrize("n,m", NM_PATTERNS)
+def test_p9_nm_structure_and_lemma1(oracle, n, m):
+    """Exactly n per row group, at most n per column group, mask2 inside mask1, and the extra zeros of
+    Eq. (sparsity_ratio) on Gaussian data (for 1:2 and 2:4 also the values the text prints)."""
+    d = 1024
+    W = si.gaussian_bf16((d, d), 0.02, 9000 + 10 * m + n)
+    WR, mask1 = oracle.prune_nm(W, n, m)
+    WRC, mask2 = oracle.double_prune_nm(W, mask1, n, m)
+    k1, k2 = oracle.mask_to_bool(mask1, d), oracle.mask_to_bool(mask2, d)
+    assert np.all(k1.reshape(d, d // m, m).sum(-1) == n)
+    assert np.all(k2.T.reshape(d, d // m, m).sum(-1) <= n)
+    assert not np.any(k2 & ~k1)
+    assert np.array_equal(WR, np.where(k1, W, 0).astype(np.uint16))
+    assert np.array_equal(WRC, np.where(k2, W, 0).astype(np.uint16))
+    extra = k1.mean() - k2.mean()
+    assert abs(extra - lemma1(n, m)) < 1.5e-3, (extra, lemma1(n, m))
+    printed = read_golden_lemma().get(f"{n}:{m}")
+    if printed is not None:
+        assert abs(extra - printed) < 1.5e-3
+    # the proof's premise: kept entries per column group ~ Binomial(m, n/m)
+    hist = np.bincount(k1.T.reshape(d, d // m, m).sum(-1).ravel(), minlength=m + 1) / (d * d // m)
+    binom = np.array([math.comb(m, j) * (n / m) ** j * (1 - n / m) ** (m - j) for j in range(m + 1)])
+    assert np.allclose(hist, binom, atol=4e-3)
