@@ -443,6 +443,7 @@ def main():
         out["optimizer_tail"] = optimizer_tail_probe(torch, B, layers, stream, pk)
         out["burst"] = burst_probe(torch, B, layers, stream, pk)
         out["inference_forward"] = inference_forward_probe(torch, B, wl, pk)
+        out["nm_masked_dense"] = nm_probe(torch, B, layers, stream, pk)
         out["dense_layer"] = dense_comparison(torch, B, layers, stream)
         out["e2e"] = e2e_run(torch, B, layers, de_flops, max(2, min(args.steps, 5)))
         out["cpu_baseline"] = cpu_baseline_sample(wl)
@@ -486,6 +487,43 @@ def optimizer_tail_probe(torch, B, layers, stream, pk, reps=20):
     return {"what": f"{reps} back-to-back launches, CUDA events; bytes: sparse_add 3 B and update 2.25 B per weight "
                     f"element; HBM peak {pk['hbm_gbs']} GB/s ({pk['src']}); the working set of sparse_add "
                     f"({3 * n / 1e6:.0f} MB) partly lives in the 126 MB L2 across launches", "rows": rows}
+
+
+def nm_probe(torch, B, layers, stream, pk, reps=10):
+    """General N:M pruning to masked-dense matrices on the largest layer: both passes and the
+    gradient mask, HBM-bound, against the measured HBM peak (2 B in + 2 B out per element, plus
+    the 1/8 B mask read and / or written)."""
+    s = max(layers, key=lambda l: l.d_in * l.d_out)
+    n_el = s.d_in * s.d_out
+    WR = torch.empty_like(s.W)
+    WRC = torch.empty_like(s.W)
+    m1 = torch.empty_like(s.mask1)
+    m2 = torch.empty_like(s.mask1)
+    rows = []
+    for n, m in ((1, 2), (2, 4), (2, 8), (4, 16)):
+        calls = {
+            "prune_nm": (lambda: B.slope_prune_nm(s.W, n, m, WR, m1), 4.125 * n_el),
+            "double_prune_nm": (lambda: B.slope_double_prune_nm(WR, m1, n, m, WRC, m2), 4.25 * n_el),
+        }
+        if (n, m) == (2, 4):
+            calls["apply_mask"] = (lambda: B.slope_apply_mask(s.W, m1, WRC), 4.125 * n_el)
+        for op, (fn, nbytes) in calls.items():
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(reps):
+                fn()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / reps
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            rows.append({"op": op, "pattern": f"{n}:{m}", "d_in": s.d_in, "d_out": s.d_out, "ms": round(ms, 4),
+                         "algorithmic_bytes": int(nbytes), "gbs": round(gbs, 1),
+                         "frac_of_hbm_peak": round(gbs / pk["hbm_gbs"], 4)})
+    return {"what": f"{reps} back-to-back launches on the largest layer ({n_el * 2 / 1e6:.0f} MB dense, working set of "
+                    f"one call > L2), CUDA events; HBM peak {pk['hbm_gbs']} GB/s ({pk['src']})", "rows": rows}
 
 
 def inference_forward_probe(torch, B, wl, pk, copies=12, reps=5):

@@ -152,6 +152,32 @@ slope_status_t slope_update_sparse_matrix(const void* Wc_vals, const void* mask1
                                           int d_out, int d_in, void* WTc_vals, void* stream);
 
 /*
+ * General N:M magnitude pruning to masked-dense matrices: the matrices A^R and A^{R,C} of
+ * Lemma 1 / Eq. (sparsity_ratio) for any pattern, and the emulation of N:M sparsity on dense
+ * GEMMs that the accuracy experiments use (Sec. "Experiment Setup").  m in {2, 4, 8, 16},
+ * 0 < n < m; d_out, d_in multiples of 128.  Selection as for 2:4: largest 15-bit bf16
+ * magnitude, the lower position wins ties.  All matrices dense row-major bf16 [d_out x d_in],
+ * masks [d_out x d_in/8] bytes (bit j%8 of byte j/8), W's orientation.
+ *
+ *   slope_prune_nm         W_R  = W with, in every group of m consecutive entries of a ROW, all but
+ *                          the n largest set to +0; mask1_bits (optional, may be NULL) = kept.
+ *   slope_double_prune_nm  W_RC = second pass on the already pruned matrix (entries outside
+ *                          mask1_bits count as zeros): in every group of m consecutive entries
+ *                          of a COLUMN keep the n largest; mask2_bits (optional) = kept by
+ *                          both passes.
+ *   slope_apply_mask       out = G where the mask bit is set, +0 elsewhere (a dense weight
+ *                          gradient restricted to a static pattern, Eq. (sparse_backward_weight)).
+ * The output may be the input matrix itself (in-place); calling slope_prune_nm on the dense
+ * master weight every step gives the dynamic-mask (re-selection) variants.
+ */
+slope_status_t slope_prune_nm(const void* W, int d_out, int d_in, int n, int m,
+                              void* W_R, void* mask1_bits, void* stream);
+slope_status_t slope_double_prune_nm(const void* W, const void* mask1_bits, int d_out, int d_in,
+                                     int n, int m, void* W_RC, void* mask2_bits, void* stream);
+slope_status_t slope_apply_mask(const void* G, const void* mask_bits, int d_out, int d_in,
+                                void* out, void* stream);
+
+/*
  * dL[d_in x r] = X[b x d_in]^T dT[b x r] without any allocation, for callers that cannot
  * call cudaMalloc or hand over a workspace (code running inside a host application whose
  * memory pool is closed to it, or in a section where allocation is forbidden).

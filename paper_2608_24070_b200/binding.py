@@ -29,6 +29,7 @@ EXPORTS = (
     "slope_meta_to_canonical", "slope_poll_status", "slope_launch_count", "slope_status_string",
     "slope_adapter_dl_noalloc", "slope_adapter_dl_noalloc_max_scratch_bytes",
     "slope_sparse_add", "slope_update_sparse_matrix", "slope_selftest_wait_timeout",
+    "slope_prune_nm", "slope_double_prune_nm", "slope_apply_mask",
 )
 
 
@@ -67,6 +68,12 @@ def lib() -> ctypes.CDLL:
         L.slope_sparse_add.restype = ci
         L.slope_update_sparse_matrix.argtypes = [vp, vp, vp, ci, ci, vp, vp]
         L.slope_update_sparse_matrix.restype = ci
+        L.slope_prune_nm.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp]
+        L.slope_prune_nm.restype = ci
+        L.slope_double_prune_nm.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, vp]
+        L.slope_double_prune_nm.restype = ci
+        L.slope_apply_mask.argtypes = [vp, vp, ci, ci, vp, vp]
+        L.slope_apply_mask.restype = ci
         L.slope_selftest_wait_timeout.argtypes = [ctypes.c_uint, vp, vp]
         L.slope_selftest_wait_timeout.restype = ci
         L.slope_poll_status.argtypes = [vp]
@@ -176,6 +183,23 @@ def slope_update_sparse_matrix(Wc_vals, mask1_bits, WTc_meta, WTc_vals):
     d_out, half = Wc_vals.shape
     _check("slope_update_sparse_matrix", lib().slope_update_sparse_matrix(
         _ptr(Wc_vals), _ptr(mask1_bits), _ptr(WTc_meta), d_out, half * 2, _ptr(WTc_vals), _stream()))
+
+
+def slope_prune_nm(W, n, m, W_R, mask1_bits=None):
+    d_out, d_in = W.shape
+    _check("slope_prune_nm", lib().slope_prune_nm(_ptr(W), d_out, d_in, int(n), int(m), _ptr(W_R), _ptr(mask1_bits),
+                                                  _stream()))
+
+
+def slope_double_prune_nm(W, mask1_bits, n, m, W_RC, mask2_bits=None):
+    d_out, d_in = W.shape
+    _check("slope_double_prune_nm", lib().slope_double_prune_nm(_ptr(W), _ptr(mask1_bits), d_out, d_in, int(n), int(m),
+                                                                _ptr(W_RC), _ptr(mask2_bits), _stream()))
+
+
+def slope_apply_mask(G, mask_bits, out):
+    d_out, d_in = G.shape
+    _check("slope_apply_mask", lib().slope_apply_mask(_ptr(G), _ptr(mask_bits), d_out, d_in, _ptr(out), _stream()))
 
 
 def slope_meta_to_canonical(meta_hw, rows, cols, meta_canon):

@@ -9,6 +9,7 @@
 #include <utility>
 
 #include "gemm_kernels.cuh"
+#include "nm_kernels.cuh"
 #include "prune_kernels.cuh"
 
 namespace slope {
@@ -631,6 +632,66 @@ slope_status_t slope_update_sparse_matrix(const void* Wc_vals, const void* mask1
     update_transposed_kernel<<<grid, 256, kUpdSmemBytes, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint4*>(Wc_vals), static_cast<const uint8_t*>(mask1_bits),
         static_cast<const uint4*>(WTc_meta), d_out, d_in, static_cast<uint4*>(WTc_vals));
+    return launch_result();
+}
+
+// ------------------------------------------------------------------ general N:M (masked dense)
+static bool nm_ok(int n, int m) { return (m == 2 || m == 4 || m == 8 || m == 16) && n > 0 && n < m; }
+
+slope_status_t slope_prune_nm(const void* W, int d_out, int d_in, int n, int m, void* W_R, void* mask1_bits,
+                              void* stream_) {
+    if (!W || !W_R) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(d_out, d_in) || !nm_ok(n, m)) return SLOPE_ERR_SHAPE;
+    if (!aligned16(W) || !aligned16(W_R) || !aligned16(mask1_bits)) return SLOPE_ERR_ALIGNMENT;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const size_t chunks = static_cast<size_t>(d_out) * d_in / 16;
+    const int grid = info.sm_count * 8;
+    const uint4* in = static_cast<const uint4*>(W);
+    uint4* out = static_cast<uint4*>(W_R);
+    uint16_t* mask = static_cast<uint16_t*>(mask1_bits);
+    switch (m) {
+        case 2: prune_nm_kernel<2><<<grid, 256, 0, stream>>>(in, chunks, n, out, mask); break;
+        case 4: prune_nm_kernel<4><<<grid, 256, 0, stream>>>(in, chunks, n, out, mask); break;
+        case 8: prune_nm_kernel<8><<<grid, 256, 0, stream>>>(in, chunks, n, out, mask); break;
+        default: prune_nm_kernel<16><<<grid, 256, 0, stream>>>(in, chunks, n, out, mask); break;
+    }
+    return launch_result();
+}
+
+slope_status_t slope_double_prune_nm(const void* W, const void* mask1_bits, int d_out, int d_in, int n, int m,
+                                     void* W_RC, void* mask2_bits, void* stream_) {
+    if (!W || !mask1_bits || !W_RC) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(d_out, d_in) || !nm_ok(n, m)) return SLOPE_ERR_SHAPE;
+    if (!aligned16(W) || !aligned16(W_RC) || !aligned16(mask1_bits) || !aligned16(mask2_bits))
+        return SLOPE_ERR_ALIGNMENT;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int grid = info.sm_count * 8;
+    const uint4* in = static_cast<const uint4*>(W);
+    const uint8_t* m1 = static_cast<const uint8_t*>(mask1_bits);
+    uint4* out = static_cast<uint4*>(W_RC);
+    uint8_t* m2 = static_cast<uint8_t*>(mask2_bits);
+    switch (m) {
+        case 2: double_prune_nm_kernel<2><<<grid, 256, 0, stream>>>(in, m1, d_out, d_in, n, out, m2); break;
+        case 4: double_prune_nm_kernel<4><<<grid, 256, 0, stream>>>(in, m1, d_out, d_in, n, out, m2); break;
+        case 8: double_prune_nm_kernel<8><<<grid, 256, 0, stream>>>(in, m1, d_out, d_in, n, out, m2); break;
+        default: double_prune_nm_kernel<16><<<grid, 256, 0, stream>>>(in, m1, d_out, d_in, n, out, m2); break;
+    }
+    return launch_result();
+}
+
+slope_status_t slope_apply_mask(const void* G, const void* mask_bits, int d_out, int d_in, void* out, void* stream) {
+    if (!G || !mask_bits || !out) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(d_out, d_in)) return SLOPE_ERR_SHAPE;
+    if (!aligned16(G) || !aligned16(mask_bits) || !aligned16(out)) return SLOPE_ERR_ALIGNMENT;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    apply_mask_kernel<<<info.sm_count * 8, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4*>(G), static_cast<const uint16_t*>(mask_bits),
+        static_cast<size_t>(d_out) * d_in / 16, static_cast<uint4*>(out));
     return launch_result();
 }
 
