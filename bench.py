@@ -266,6 +266,9 @@ def main():
     ap.add_argument("--impl", default="slope", choices=["slope", "reference"])
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling only)")
     ap.add_argument("--no-extras", action="store_true", help="skip dense comparison, e2e and CPU baseline")
+    ap.add_argument("--cusparselt-context", action="store_true",
+                    help="also time the forward GEMMs through torch's semi-structured sparse matmul (cuSPARSELt, "
+                         "the library the paper builds on); context only, off by default")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "slope" and not args.tokens else args.warmup
 
@@ -445,6 +448,8 @@ def main():
         out["inference_forward"] = inference_forward_probe(torch, B, wl, pk)
         out["nm_masked_dense"] = nm_probe(torch, B, layers, stream, pk)
         out["dense_layer"] = dense_comparison(torch, B, layers, stream)
+        if args.cusparselt_context:
+            out["cusparselt_context"] = cusparselt_context(torch, B, layers, stream)
         out["e2e"] = e2e_run(torch, B, layers, de_flops, max(2, min(args.steps, 5)))
         out["cpu_baseline"] = cpu_baseline_sample(wl)
     elif rank == 0:
@@ -667,6 +672,54 @@ def dense_comparison(torch, B, layers, stream, reps=5):
     return {"what": "torch.matmul (cuBLAS) Y=XW^T, dX=dY W, dW=dY^T X vs slope fwd+dX+masked dW, same shapes, interleaved",
             "dense_ms": round(t_dense, 4), "slope_ms": round(t_slope, 4), "speedup": round(t_dense / t_slope, 3),
             "layers": rows}
+
+
+def cusparselt_context(torch, B, layers, stream, reps=10):
+    """Context, not a target: the forward GEMM of each distinct layer shape through
+    torch.sparse.to_sparse_semi_structured + F.linear (cuSPARSELt), next to slope_linear_fwd, with
+    the relative error of both against torch.matmul on the same masked dense weight."""
+    rows, seen = [], set()
+    try:
+        from torch.sparse import to_sparse_semi_structured
+        version = torch.backends.cusparselt.version() if torch.backends.cusparselt.is_available() else None
+    except Exception as ex:                                 # noqa: BLE001
+        return {"unavailable": f"{type(ex).__name__}: {ex}"}
+    for s in layers:
+        if (s.d_in, s.d_out) in seen:
+            continue
+        seen.add((s.d_in, s.d_out))
+        try:
+            shifts = torch.arange(8, device=s.W.device, dtype=torch.uint8)
+            keep = ((s.mask1.unsqueeze(-1) >> shifts) & 1).bool().view(s.d_out, s.d_in)     # slope_prune_24's mask
+            Wp = (s.W * keep).contiguous()
+            Ws = to_sparse_semi_structured(Wp)
+            ref = torch.matmul(s.X, Wp.t()).float()
+
+            def timed(fn):
+                fn()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for _ in range(reps):
+                    y = fn()
+                e1.record(stream)
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1) / reps, y
+
+            ms_lib, y_lib = timed(lambda: torch.nn.functional.linear(s.X, Ws))
+            ms_own, _ = timed(lambda: (B.slope_linear_fwd(s.X, s.Wc_vals, s.Wc_meta, s.d_out, s.Y), s.Y)[1])
+            flop = 2.0 * s.b * s.d_in * s.d_out
+            rows.append({"d_in": s.d_in, "d_out": s.d_out, "tokens": s.b,
+                         "cusparselt_ms": round(ms_lib, 4), "cusparselt_tflops_dense_eq": round(flop / ms_lib / 1e9, 1),
+                         "cusparselt_rel_err_vs_dense": round(float((y_lib.float() - ref).norm() / ref.norm()), 5),
+                         "slope_fwd_ms": round(ms_own, 4), "slope_tflops_dense_eq": round(flop / ms_own / 1e9, 1),
+                         "slope_rel_err_vs_dense": round(float((s.Y.float() - ref).norm() / ref.norm()), 5)})
+            del Ws, Wp, ref, y_lib
+        except Exception as ex:                             # noqa: BLE001
+            rows.append({"d_in": s.d_in, "d_out": s.d_out, "failed": f"{type(ex).__name__}: {str(ex)[:200]}"})
+    return {"what": f"forward GEMM through torch.sparse.to_sparse_semi_structured + F.linear (cuSPARSELt {version}) vs "
+                    f"slope_linear_fwd, {reps} back-to-back launches each, CUDA events; both on slope_prune_24's mask, "
+                    f"errors against torch.matmul on the masked dense weight", "rows": rows}
 
 
 def e2e_run(torch, B, layers, de_flops, steps):
