@@ -641,37 +641,58 @@ def burst_probe(torch, B, layers, stream, pk, launches=8):
 
 
 def dense_comparison(torch, B, layers, stream, reps=5):
-    """fwd+bwd of the same layers as dense bf16 GEMMs (torch.matmul -> cuBLAS), interleaved with the
-    SLoPe stages fwd/dX/dW (no pruning, no adapter) in the same process."""
-    t_dense = t_slope = 0.0
+    """fwd+bwd of the same layers as dense bf16 GEMMs, once through torch.matmul (cuBLAS) and once
+    through this library's own dense tcgen05 kernels, interleaved with the SLoPe stages
+    fwd/dX/dW (no pruning, no adapter) in the same process."""
+    totals = {"cublas": 0.0, "inhouse": 0.0, "slope": 0.0}
     rows = []
     for s in layers:
         Wd = s.W
-        ed = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-        es = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-        md, ms_ = [], []
-        for _ in range(reps + 1):
-            ed[0].record(stream)
+        Yd = torch.empty_like(s.Y)
+        dXd = torch.empty_like(s.dX)
+        dWd = torch.empty_like(s.W)
+
+        def cublas():
             Y = torch.matmul(s.X, Wd.t())
             dX = torch.matmul(s.dY, Wd)
             dW = torch.matmul(s.dY.t(), s.X)
-            ed[1].record(stream)
-            es[0].record(stream)
+            del Y, dX, dW
+
+        def inhouse():
+            B.slope_dense_linear_fwd(s.X, Wd, Yd)
+            B.slope_dense_linear_bwd_dx(s.dY, Wd, dXd)
+            B.slope_dense_linear_bwd_dw(s.dY, s.X, dWd)
+
+        def slope():
             B.slope_linear_fwd(s.X, s.Wc_vals, s.Wc_meta, s.d_out, s.Y)
             B.slope_linear_bwd_dx(s.dY, s.WTc_vals, s.WTc_meta, s.d_in, s.dX)
             B.slope_linear_bwd_dw_masked(s.dY, s.X, s.mask1, s.dWc)
-            es[1].record(stream)
+
+        arms = {"cublas": cublas, "inhouse": inhouse, "slope": slope}
+        times = {k: [] for k in arms}
+        for _ in range(reps + 1):
+            evs = {}
+            for k, fn in arms.items():
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                fn()
+                e1.record(stream)
+                evs[k] = (e0, e1)
             torch.cuda.synchronize()
-            md.append(ed[0].elapsed_time(ed[1]))
-            ms_.append(es[0].elapsed_time(es[1]))
-            del Y, dX, dW
-        d, sl = statistics.median(md[1:]), statistics.median(ms_[1:])
-        t_dense += d
-        t_slope += sl
-        rows.append({"layer": s.name, "dense_ms": round(d, 4), "slope_ms": round(sl, 4), "speedup": round(d / sl, 3)})
-    return {"what": "torch.matmul (cuBLAS) Y=XW^T, dX=dY W, dW=dY^T X vs slope fwd+dX+masked dW, same shapes, interleaved",
-            "dense_ms": round(t_dense, 4), "slope_ms": round(t_slope, 4), "speedup": round(t_dense / t_slope, 3),
-            "layers": rows}
+            for k, (e0, e1) in evs.items():
+                times[k].append(e0.elapsed_time(e1))
+        med = {k: statistics.median(v[1:]) for k, v in times.items()}
+        for k in totals:
+            totals[k] += med[k]
+        rows.append({"layer": s.name, "dense_ms": round(med["cublas"], 4), "inhouse_dense_ms": round(med["inhouse"], 4),
+                     "slope_ms": round(med["slope"], 4), "speedup": round(med["cublas"] / med["slope"], 3),
+                     "speedup_vs_inhouse_dense": round(med["inhouse"] / med["slope"], 3)})
+        del Yd, dXd, dWd
+    return {"what": "dense layer Y=XW^T, dX=dY W, dW=dY^T X through torch.matmul (cuBLAS) and through the library's own "
+                    "dense tcgen05 kernels (slope_dense_linear_*) vs slope fwd+dX+masked dW, same shapes, interleaved",
+            "dense_ms": round(totals["cublas"], 4), "inhouse_dense_ms": round(totals["inhouse"], 4),
+            "slope_ms": round(totals["slope"], 4), "speedup": round(totals["cublas"] / totals["slope"], 3),
+            "speedup_vs_inhouse_dense": round(totals["inhouse"] / totals["slope"], 3), "layers": rows}
 
 
 def cusparselt_context(torch, B, layers, stream, reps=10):

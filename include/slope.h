@@ -178,6 +178,23 @@ slope_status_t slope_apply_mask(const void* G, const void* mask_bits, int d_out,
                                 void* out, void* stream);
 
 /*
+ * The dense bf16 layer on the same tcgen05 pipeline (CTA-pair 256 x 256 tiles, no sparsity):
+ *   slope_dense_linear_fwd      Y [b x d_out]    = X  W^T
+ *   slope_dense_linear_bwd_dx   dX[b x d_in]     = dY W
+ *   slope_dense_linear_bwd_dw   dW[d_out x d_in] = dY^T X
+ * for a dense row-major W[d_out x d_in]; fp32 accumulation, one rounding to bf16.  They are the
+ * dense layer of Eq. (forward) / Eq. (backward_input) / Eq. (backward_weight) that the sparse
+ * path is compared with, and they run N:M-emulated layers on the masked-dense matrices of
+ * slope_prune_nm / slope_double_prune_nm (mask the weight gradient with slope_apply_mask).
+ */
+slope_status_t slope_dense_linear_fwd(const void* X, int b, const void* W, int d_out, int d_in,
+                                      void* Y, void* stream);
+slope_status_t slope_dense_linear_bwd_dx(const void* dY, int b, const void* W, int d_out, int d_in,
+                                         void* dX, void* stream);
+slope_status_t slope_dense_linear_bwd_dw(const void* dY, const void* X, int b, int d_out, int d_in,
+                                         void* dW, void* stream);
+
+/*
  * dL[d_in x r] = X[b x d_in]^T dT[b x r] without any allocation, for callers that cannot
  * call cudaMalloc or hand over a workspace (code running inside a host application whose
  * memory pool is closed to it, or in a section where allocation is forbidden).

@@ -30,6 +30,7 @@ EXPORTS = (
     "slope_adapter_dl_noalloc", "slope_adapter_dl_noalloc_max_scratch_bytes",
     "slope_sparse_add", "slope_update_sparse_matrix", "slope_selftest_wait_timeout",
     "slope_prune_nm", "slope_double_prune_nm", "slope_apply_mask",
+    "slope_dense_linear_fwd", "slope_dense_linear_bwd_dx", "slope_dense_linear_bwd_dw",
 )
 
 
@@ -68,6 +69,11 @@ def lib() -> ctypes.CDLL:
         L.slope_sparse_add.restype = ci
         L.slope_update_sparse_matrix.argtypes = [vp, vp, vp, ci, ci, vp, vp]
         L.slope_update_sparse_matrix.restype = ci
+        L.slope_dense_linear_fwd.argtypes = [vp, ci, vp, ci, ci, vp, vp]
+        L.slope_dense_linear_bwd_dx.argtypes = [vp, ci, vp, ci, ci, vp, vp]
+        L.slope_dense_linear_bwd_dw.argtypes = [vp, vp, ci, ci, ci, vp, vp]
+        for name in ("slope_dense_linear_fwd", "slope_dense_linear_bwd_dx", "slope_dense_linear_bwd_dw"):
+            getattr(L, name).restype = ci
         L.slope_prune_nm.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp]
         L.slope_prune_nm.restype = ci
         L.slope_double_prune_nm.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, vp]
@@ -183,6 +189,23 @@ def slope_update_sparse_matrix(Wc_vals, mask1_bits, WTc_meta, WTc_vals):
     d_out, half = Wc_vals.shape
     _check("slope_update_sparse_matrix", lib().slope_update_sparse_matrix(
         _ptr(Wc_vals), _ptr(mask1_bits), _ptr(WTc_meta), d_out, half * 2, _ptr(WTc_vals), _stream()))
+
+
+def slope_dense_linear_fwd(X, W, Y):
+    (b, d_in), d_out = X.shape, W.shape[0]
+    _check("slope_dense_linear_fwd", lib().slope_dense_linear_fwd(_ptr(X), b, _ptr(W), d_out, d_in, _ptr(Y), _stream()))
+
+
+def slope_dense_linear_bwd_dx(dY, W, dX):
+    (b, d_out), d_in = dY.shape, W.shape[1]
+    _check("slope_dense_linear_bwd_dx", lib().slope_dense_linear_bwd_dx(_ptr(dY), b, _ptr(W), d_out, d_in, _ptr(dX),
+                                                                        _stream()))
+
+
+def slope_dense_linear_bwd_dw(dY, X, dW):
+    (b, d_out), d_in = dY.shape, X.shape[1]
+    _check("slope_dense_linear_bwd_dw", lib().slope_dense_linear_bwd_dw(_ptr(dY), _ptr(X), b, d_out, d_in, _ptr(dW),
+                                                                        _stream()))
 
 
 def slope_prune_nm(W, n, m, W_R, mask1_bits=None):

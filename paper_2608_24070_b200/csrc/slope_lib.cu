@@ -549,6 +549,43 @@ slope_status_t slope_linear_bwd_dw_masked(const void* dY, const void* X, int b, 
                                                              static_cast<cudaStream_t>(stream), info);
 }
 
+// ------------------------------------------------------------------ dense layer on the same pipeline
+static slope_status_t dense_args(const void* a, const void* b_, const void* c, int b, int d_out, int d_in) {
+    if (!a || !b_ || !c) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(d_out, d_in) || b < 8 || b % 8 != 0) return SLOPE_ERR_SHAPE;
+    if (!aligned16(a) || !aligned16(b_) || !aligned16(c)) return SLOPE_ERR_ALIGNMENT;
+    return SLOPE_OK;
+}
+
+slope_status_t slope_dense_linear_fwd(const void* X, int b, const void* W, int d_out, int d_in, void* Y, void* stream) {
+    if (slope_status_t st = dense_args(X, W, Y, b, d_out, d_in)) return st;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    // Y[b x d_out] = X[b x d_in] * W[d_out x d_in]^T: both operands K-contiguous
+    return launch_dense_pair<false, false, 256, kEpiStore, 6>(X, W, b, d_out, d_in, Y, nullptr,
+                                                              static_cast<cudaStream_t>(stream), info);
+}
+
+slope_status_t slope_dense_linear_bwd_dx(const void* dY, int b, const void* W, int d_out, int d_in, void* dX,
+                                         void* stream) {
+    if (slope_status_t st = dense_args(dY, W, dX, b, d_out, d_in)) return st;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    // dX[b x d_in] = dY[b x d_out] * W[d_out x d_in]: W is the [K x N] operand
+    return launch_dense_pair<false, true, 256, kEpiStore, 6>(dY, W, b, d_in, d_out, dX, nullptr,
+                                                             static_cast<cudaStream_t>(stream), info);
+}
+
+slope_status_t slope_dense_linear_bwd_dw(const void* dY, const void* X, int b, int d_out, int d_in, void* dW,
+                                         void* stream) {
+    if (slope_status_t st = dense_args(dY, X, dW, b, d_out, d_in)) return st;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    // dW[d_out x d_in] = dY[b x d_out]^T * X[b x d_in]: both operands stored [K x .]
+    return launch_dense_pair<true, true, 256, kEpiStore, 6>(dY, X, d_out, d_in, b, dW, nullptr,
+                                                            static_cast<cudaStream_t>(stream), info);
+}
+
 static size_t adapter_partial_bytes(int b, int rows, int r) {
     return ((static_cast<size_t>(adapter_splits(b, rows)) * rows * r * sizeof(float)) + 255) & ~size_t(255);
 }

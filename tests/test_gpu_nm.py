@@ -122,3 +122,84 @@ def test_nm_argument_errors(B):
             B.slope_prune_nm(W, n, m, W, None)
         assert e.value.status == 2
     assert B.slope_poll_status() == 0
+
+
+# ------------------------------------------------------------------ dense layer on the same pipeline
+def _dense_dw_from_oracle(oracle, dY, X, d_out, d_in):
+    """Dense dW = dY^T X from the masked-gradient oracle: the masks "positions 0,1" and "positions 2,3"
+    of every group together cover every entry exactly once."""
+    lo = np.full((d_out, d_in // 8), 0x33, np.uint8)          # bits 0,1 and 4,5 of every byte
+    hi = np.full((d_out, d_in // 8), 0xCC, np.uint8)
+    rows = np.arange(d_out)
+    a = oracle.dw_rows(dY, X, lo, rows).reshape(d_out, d_in // 4, 2)
+    b = oracle.dw_rows(dY, X, hi, rows).reshape(d_out, d_in // 4, 2)
+    return np.concatenate([a, b], axis=-1).reshape(d_out, d_in)
+
+
+@pytest.mark.parametrize("d_in,d_out,b", [(384, 640, 776), (1024, 256, 264), (128, 128, 8)])
+def test_dense_layer_against_oracle(B, oracle, d_in, d_out, b):
+    import torch
+    from helpers import REL_TOL, rel_fro, to_f64
+
+    W = si.gaussian_bf16((d_out, d_in), 0.02, 501)
+    X = si.gaussian_bf16((b, d_in), 1.0, 502)
+    dY = si.gaussian_bf16((b, d_out), 1.0, 503)
+    Wd, Xd, dYd = B.bf16_from_bits(W), B.bf16_from_bits(X), B.bf16_from_bits(dY)
+    Y = torch.empty((b, d_out), dtype=torch.bfloat16, device="cuda")
+    dX = torch.empty((b, d_in), dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty((d_out, d_in), dtype=torch.bfloat16, device="cuda")
+    B.slope_dense_linear_fwd(Xd, Wd, Y)
+    B.slope_dense_linear_bwd_dx(dYd, Wd, dX)
+    B.slope_dense_linear_bwd_dw(dYd, Xd, dW)
+    assert B.slope_poll_status() == 0
+    full = np.full((d_out, d_in // 8), 0xFF, np.uint8)        # every entry kept: the dense layer
+    rows = np.arange(b)
+    errs = {
+        "Y": rel_fro(to_f64(B.bits_from_bf16(Y)), oracle.fwd_rows(X, W, full, rows)),
+        "dX": rel_fro(to_f64(B.bits_from_bf16(dX)), oracle.dx_rows(dY, W, full, rows)),
+        "dW": rel_fro(to_f64(B.bits_from_bf16(dW)), _dense_dw_from_oracle(oracle, dY, X, d_out, d_in)),
+    }
+    print(errs)
+    for k, v in errs.items():
+        assert v <= REL_TOL, (k, v, errs)
+
+
+def test_emulated_2_8_layer_matches_oracle_on_the_masks(B, oracle):
+    """An N:M-emulated layer (2:8): prune, double prune, dense GEMMs on the masked-dense matrices and the
+    masked weight gradient, against the oracle evaluated with the same (oracle-made) masks."""
+    import torch
+    from helpers import REL_TOL, rel_fro, to_f64
+
+    n, m, d_in, d_out, b = 2, 8, 512, 384, 264
+    W = si.gaussian_bf16((d_out, d_in), 0.02, 511)
+    X = si.gaussian_bf16((b, d_in), 1.0, 512)
+    dY = si.gaussian_bf16((b, d_out), 1.0, 513)
+    _, mask1 = oracle.prune_nm(W, n, m)
+    _, mask2 = oracle.double_prune_nm(W, mask1, n, m)
+    Wd, Xd, dYd = B.bf16_from_bits(W), B.bf16_from_bits(X), B.bf16_from_bits(dY)
+    WR, WRC = torch.empty_like(Wd), torch.empty_like(Wd)
+    m1 = torch.empty((d_out, d_in // 8), dtype=torch.uint8, device="cuda")
+    B.slope_prune_nm(Wd, n, m, WR, m1)
+    B.slope_double_prune_nm(WR, m1, n, m, WRC, None)
+    Y = torch.empty((b, d_out), dtype=torch.bfloat16, device="cuda")
+    dX = torch.empty((b, d_in), dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty((d_out, d_in), dtype=torch.bfloat16, device="cuda")
+    B.slope_dense_linear_fwd(Xd, WR, Y)
+    B.slope_dense_linear_bwd_dx(dYd, WRC, dX)
+    B.slope_dense_linear_bwd_dw(dYd, Xd, dW)
+    B.slope_apply_mask(dW, m1, dW)
+    assert B.slope_poll_status() == 0
+    assert np.array_equal(m1.cpu().numpy(), mask1)
+    rows = np.arange(b)
+    keep1 = oracle.mask_to_bool(mask1, d_in)
+    want_dW = np.where(keep1, _dense_dw_from_oracle(oracle, dY, X, d_out, d_in), 0.0)
+    errs = {
+        "Y": rel_fro(to_f64(B.bits_from_bf16(Y)), oracle.fwd_rows(X, W, mask1, rows)),
+        "dX": rel_fro(to_f64(B.bits_from_bf16(dX)), oracle.dx_rows(dY, W, mask2, rows)),
+        "dW": rel_fro(to_f64(B.bits_from_bf16(dW)), want_dW),
+    }
+    print(errs)
+    for k, v in errs.items():
+        assert v <= REL_TOL, (k, v, errs)
+    got = B.bits_from_bf16(dW)
+    assert not np.any(got[~keep1] & 0x7FFF)                   # exact zeros outside the mask
