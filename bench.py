@@ -447,6 +447,7 @@ def main():
         out["burst"] = burst_probe(torch, B, layers, stream, pk)
         out["inference_forward"] = inference_forward_probe(torch, B, wl, pk)
         out["nm_masked_dense"] = nm_probe(torch, B, layers, stream, pk)
+        out["small_configs_hot_cold"] = small_config_probe(torch, B, stream, pk)
         out["dense_layer"] = dense_comparison(torch, B, layers, stream)
         if args.cusparselt_context:
             out["cusparselt_context"] = cusparselt_context(torch, B, layers, stream)
@@ -492,6 +493,82 @@ def optimizer_tail_probe(torch, B, layers, stream, pk, reps=20):
     return {"what": f"{reps} back-to-back launches, CUDA events; bytes: sparse_add 3 B and update 2.25 B per weight "
                     f"element; HBM peak {pk['hbm_gbs']} GB/s ({pk['src']}); the working set of sparse_add "
                     f"({3 * n / 1e6:.0f} MB) partly lives in the 126 MB L2 across launches", "rows": rows}
+
+
+def small_config_probe(torch, B, stream, pk, min_launches=48):
+    """The two small configurations (one 512 x 512 layer with 256 tokens; GPT-2-small with 8192 tokens),
+    every op of every layer, device time per launch from a CUDA graph of back-to-back launches (no host
+    overhead; includes the ~1 us gap between dependent kernels): "hot" = all launches on one buffer set
+    (operands stay in L2), "cold" = the launches cycle through enough separate buffer sets (at least 4,
+    together more than 160 MB) that every operand has left L2 when its turn comes again.
+    Roofline time t* = max(dense-equivalent FLOP / peak, bytes / HBM peak)."""
+    dev = torch.device("cuda")
+    side = torch.cuda.Stream()
+
+    def graph_us(calls):
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            for fn in calls[:4]:
+                fn()
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for fn in calls:
+                    fn()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(5):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); graph.replay(); e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        return best * 1e3 / len(calls)
+
+    rows = []
+    for key in ("c1_single_512", "c2_gpt2_small"):
+        wl = si.WORKLOADS[key]
+        for idx, lay in enumerate(wl.layers):
+            n_w = lay.d_in * lay.d_out
+            act = 2.0 * wl.tokens * (lay.d_in + lay.d_out)
+            set_bytes = 2.0 * n_w * 2.25 + 2.0 * act                      # W + both compressed copies, X, dY, Y, dX
+            nsets = int(min(128, max(4, -(-160e6 // set_bytes))))
+            sets = []
+            for _ in range(nsets):
+                s = LayerState(B, torch, wl, idx, wl.tokens, dev)
+                B.slope_prune_24(s.W, s.Wc_vals, s.Wc_meta, s.mask1)
+                B.slope_double_prune(s.W, s.mask1, s.WTc_vals, s.WTc_meta, None)
+                sets.append(s)
+            flop = 2.0 * wl.tokens * n_w
+            ops = {
+                "prune_24": (lambda s: B.slope_prune_24(s.W, s.Wc_vals, s.Wc_meta, s.mask1), 0.0, 3.25 * n_w, None),
+                "double_prune": (lambda s: B.slope_double_prune(s.W, s.mask1, s.WTc_vals, s.WTc_meta, None), 0.0,
+                                 3.25 * n_w, None),
+                "linear_fwd": (lambda s: B.slope_linear_fwd(s.X, s.Wc_vals, s.Wc_meta, s.d_out, s.Y), flop,
+                               act + 1.125 * n_w, 2.0 * pk["bf16"]),
+                "linear_bwd_dx": (lambda s: B.slope_linear_bwd_dx(s.dY, s.WTc_vals, s.WTc_meta, s.d_in, s.dX), flop,
+                                  act + 1.125 * n_w, 2.0 * pk["bf16"]),
+                "linear_bwd_dw_masked": (lambda s: B.slope_linear_bwd_dw_masked(s.dY, s.X, s.mask1, s.dWc), flop,
+                                         act + 1.125 * n_w, pk["bf16"]),
+            }
+            launches = nsets * max(1, -(-min_launches // nsets))
+            for op, (fn, fl, nbytes, peak_tf) in ops.items():
+                hot = graph_us([lambda fn=fn: fn(sets[0])] * launches)
+                cold = graph_us([lambda fn=fn, s=sets[i % nsets]: fn(s) for i in range(launches)])
+                t_star = max(fl / (peak_tf * 1e12) if peak_tf else 0.0, nbytes / (pk["hbm_gbs"] * 1e9)) * 1e6
+                rows.append({"workload": key, "layer": lay.name, "d_in": lay.d_in, "d_out": lay.d_out,
+                             "tokens": wl.tokens, "op": op, "buffer_sets": nsets, "hot_us": round(hot, 2),
+                             "cold_us": round(cold, 2), "roofline_us": round(t_star, 2),
+                             "roofline_frac_cold": round(t_star / cold, 3),
+                             "tflops_dense_eq_cold": round(fl / cold / 1e6, 1) if fl else None})
+            del sets
+    st = B.slope_poll_status()
+    if st != 0:
+        raise SystemExit(f"device status after the small-config probe: {B.slope_status_string(st)}")
+    return {"what": f"us per launch from CUDA graphs of >= {min_launches} launches (best of 5 replays); hot = one buffer "
+                    f"set, cold = cycling through buffer_sets sets (> 160 MB together); t* from burst peaks (dense "
+                    f"{pk['bf16']} TFLOP/s, sparse := 2x, HBM {pk['hbm_gbs']} GB/s)", "rows": rows}
 
 
 def nm_probe(torch, B, layers, stream, pk, reps=10):
