@@ -73,7 +73,7 @@ prune_nm_kernel(const uint4* W, size_t n_chunks, int n, uint4* out, uint16_t* __
     static_assert(M == 2 || M == 4 || M == 8 || M == 16, "group size");
     const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
     for (size_t c = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; c < n_chunks; c += stride) {
-        const uint4 a = W[2 * c], b = W[2 * c + 1];
+        const uint4 a = __ldcs(W + 2 * c), b = __ldcs(W + 2 * c + 1);       // streamed: read once
         uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
         uint32_t keep = 0;
 #pragma unroll
@@ -92,8 +92,8 @@ prune_nm_kernel(const uint4* W, size_t n_chunks, int n, uint4* out, uint16_t* __
             const uint32_t hi = (keep >> (2 * q + 1)) & 1u ? 0xFFFF0000u : 0u;
             w[q] &= lo | hi;
         }
-        out[2 * c] = make_uint4(w[0], w[1], w[2], w[3]);
-        out[2 * c + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+        __stcs(out + 2 * c, make_uint4(w[0], w[1], w[2], w[3]));
+        __stcs(out + 2 * c + 1, make_uint4(w[4], w[5], w[6], w[7]));
         if (mask != nullptr) mask[c] = static_cast<uint16_t>(keep);
     }
 }
@@ -118,7 +118,7 @@ double_prune_nm_kernel(const uint4* W, const uint8_t* __restrict__ mask1, int d_
         uint32_t m1[M];
 #pragma unroll
         for (int t = 0; t < M; ++t) {
-            const uint4 v = W[base + static_cast<size_t>(t) * row_u4];
+            const uint4 v = __ldcs(W + base + static_cast<size_t>(t) * row_u4);
             w[t][0] = v.x; w[t][1] = v.y; w[t][2] = v.z; w[t][3] = v.w;
             m1[t] = mask1[base + static_cast<size_t>(t) * row_u4];
         }
@@ -144,7 +144,7 @@ double_prune_nm_kernel(const uint4* W, const uint8_t* __restrict__ mask1, int d_
                 const uint32_t hi = (both >> (2 * q + 1)) & 1u ? 0xFFFF0000u : 0u;
                 w[t][q] &= lo | hi;
             }
-            out[base + static_cast<size_t>(t) * row_u4] = make_uint4(w[t][0], w[t][1], w[t][2], w[t][3]);
+            __stcs(out + base + static_cast<size_t>(t) * row_u4, make_uint4(w[t][0], w[t][1], w[t][2], w[t][3]));
             if (mask2 != nullptr) mask2[base + static_cast<size_t>(t) * row_u4] = static_cast<uint8_t>(both);
         }
     }
@@ -156,7 +156,7 @@ __global__ void __launch_bounds__(256)
 apply_mask_kernel(const uint4* G, const uint16_t* __restrict__ mask, size_t n_chunks, uint4* out) {
     const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
     for (size_t c = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; c < n_chunks; c += stride) {
-        const uint4 a = G[2 * c], b = G[2 * c + 1];
+        const uint4 a = __ldcs(G + 2 * c), b = __ldcs(G + 2 * c + 1);
         uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
         const uint32_t keep = mask[c];
 #pragma unroll
@@ -165,8 +165,8 @@ apply_mask_kernel(const uint4* G, const uint16_t* __restrict__ mask, size_t n_ch
             const uint32_t hi = (keep >> (2 * q + 1)) & 1u ? 0xFFFF0000u : 0u;
             w[q] &= lo | hi;
         }
-        out[2 * c] = make_uint4(w[0], w[1], w[2], w[3]);
-        out[2 * c + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+        __stcs(out + 2 * c, make_uint4(w[0], w[1], w[2], w[3]));
+        __stcs(out + 2 * c + 1, make_uint4(w[4], w[5], w[6], w[7]));
     }
 }
 

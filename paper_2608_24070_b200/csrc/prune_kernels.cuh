@@ -224,12 +224,12 @@ __global__ void __launch_bounds__(256) meta_to_canonical_kernel(const uint16_t* 
 
 // "sparseAdd": out = beta * A + gamma * B on two compressed value arrays with one pattern
 // (fp32 arithmetic, one rounding to bf16).  Pure streaming: 16-byte vectors, grid-stride.
-__global__ void __launch_bounds__(256) sparse_add_kernel(const uint4* __restrict__ A, const uint4* __restrict__ B,
-                                                         float beta, float gamma, size_t n_vec,
-                                                         uint4* __restrict__ out) {
+// `out` may be A or B (every thread reads its vectors before it writes them), hence no __restrict__.
+__global__ void __launch_bounds__(256) sparse_add_kernel(const uint4* A, const uint4* B, float beta, float gamma,
+                                                         size_t n_vec, uint4* out) {
     for (size_t idx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; idx < n_vec;
          idx += static_cast<size_t>(gridDim.x) * blockDim.x) {
-        const uint4 a = __ldg(A + idx), b = __ldg(B + idx);
+        const uint4 a = A[idx], b = B[idx];
         const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
         uint32_t r[4];
 #pragma unroll

@@ -179,6 +179,10 @@ static bool set_smem(Kernel k, int bytes) {
     return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
 }
 
+// Grid of the grid-stride streaming kernels: many short blocks per SM keep the tail of the last
+// wave short (masked copy of a 90 MB matrix: 78 % of the HBM peak with 8 blocks per SM, 91 % with 32).
+constexpr int kStreamBlocksPerSm = 32;
+
 // ------------------------------------------------------------------ dense GEMM launch
 struct DenseProblem {
     const void* A = nullptr;
@@ -650,7 +654,7 @@ slope_status_t slope_sparse_add(const void* A_vals, const void* B_vals, float be
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
     const size_t n_vec = static_cast<size_t>(rows) * cols / 2 / 8;
-    sparse_add_kernel<<<info.sm_count * 8, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+    sparse_add_kernel<<<info.sm_count * kStreamBlocksPerSm, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint4*>(A_vals), static_cast<const uint4*>(B_vals), beta, gamma, n_vec,
         static_cast<uint4*>(out_vals));
     return launch_result();
@@ -684,7 +688,7 @@ slope_status_t slope_prune_nm(const void* W, int d_out, int d_in, int n, int m, 
     if (slope_status_t st = check_arch(info)) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const size_t chunks = static_cast<size_t>(d_out) * d_in / 16;
-    const int grid = info.sm_count * 8;
+    const int grid = info.sm_count * kStreamBlocksPerSm;
     const uint4* in = static_cast<const uint4*>(W);
     uint4* out = static_cast<uint4*>(W_R);
     uint16_t* mask = static_cast<uint16_t*>(mask1_bits);
@@ -706,7 +710,7 @@ slope_status_t slope_double_prune_nm(const void* W, const void* mask1_bits, int 
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    const int grid = info.sm_count * 8;
+    const int grid = info.sm_count * kStreamBlocksPerSm;
     const uint4* in = static_cast<const uint4*>(W);
     const uint8_t* m1 = static_cast<const uint8_t*>(mask1_bits);
     uint4* out = static_cast<uint4*>(W_RC);
@@ -726,7 +730,7 @@ slope_status_t slope_apply_mask(const void* G, const void* mask_bits, int d_out,
     if (!aligned16(G) || !aligned16(mask_bits) || !aligned16(out)) return SLOPE_ERR_ALIGNMENT;
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
-    apply_mask_kernel<<<info.sm_count * 8, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+    apply_mask_kernel<<<info.sm_count * kStreamBlocksPerSm, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint4*>(G), static_cast<const uint16_t*>(mask_bits),
         static_cast<size_t>(d_out) * d_in / 16, static_cast<uint4*>(out));
     return launch_result();
