@@ -110,3 +110,86 @@ def test_full_size_inference_forward(B, oracle, key, idx, tokens):
     print(key, lay.name, tokens, errs)
     for k, v in errs.items():
         assert v <= REL_TOL, (k, v, errs)
+
+
+def test_more_than_2_31_activation_elements(B, oracle):
+    """524296 tokens x 4096 features: activations and outputs of 2^31 + 32768 elements each, so every
+    64-bit index path (TMA row coordinates, output offsets, the token reduction of the weight gradient
+    over 8193 k-blocks) is exercised.  The activations are a seeded 2048-token block repeated 256 times
+    plus 8 more rows, so the oracle needs only the block: row n of the big tensors is block row n % 2048,
+    and dY^T X = 256 * (block term) + (term of the first 8 block rows)."""
+    import torch
+
+    d, blk, reps, extra = 4096, 2048, 256, 8
+    b = blk * reps + extra
+    W = si.gaussian_bf16((d, d), 0.02, 901)
+    Xb = si.gaussian_bf16((blk, d), 1.0, 902)
+    dYb = si.gaussian_bf16((blk, d), 1.0, 903)
+    layer = GpuLayer(W)
+    _, _, mask1 = oracle.prune24(W)
+    _, _, mask2 = oracle.double_prune(W, mask1)
+    assert np.array_equal(layer.mask1.cpu().numpy(), mask1) and np.array_equal(layer.mask2.cpu().numpy(), mask2)
+
+    def tiled(bits):
+        small = B.bf16_from_bits(bits)
+        big = torch.empty((b, d), dtype=torch.bfloat16, device="cuda")
+        big[: blk * reps].view(reps, blk, d).copy_(small.unsqueeze(0).expand(reps, blk, d))
+        big[blk * reps:] = small[:extra]
+        return big
+
+    X, dY = tiled(Xb), tiled(dYb)
+    assert X.numel() > 2 ** 31
+    Y = layer.fwd(X)
+    dX = layer.dx(dY)
+    dWc = layer.dw(dY, X)
+    layer.poll()
+    rows = np.concatenate([np.arange(3), si.sample_indices(b, 24, 904), np.arange(b - extra - 3, b)])   # incl. the last rows
+    pick = lambda t: to_f64(B.bits_from_bf16(t[torch.as_tensor(rows, device="cuda", dtype=torch.long)]))
+    errs = {
+        "Y": rel_fro(pick(Y), oracle.fwd_rows(Xb, W, mask1, rows % blk)),
+        "dX": rel_fro(pick(dX), oracle.dx_rows(dYb, W, mask2, rows % blk)),
+    }
+    orows = si.sample_indices(d, 32, 905)
+    want = reps * oracle.dw_rows(dYb, Xb, mask1, orows) + oracle.dw_rows(dYb[:extra], Xb[:extra], mask1, orows)
+    got = to_f64(B.bits_from_bf16(dWc[torch.as_tensor(orows, device="cuda", dtype=torch.long)]))
+    errs["dWc"] = rel_fro(got, want)
+    print(errs)
+    for k, v in errs.items():
+        assert v <= REL_TOL, (k, v, errs)
+    for t in (Y, dX):
+        assert bool(torch.isfinite(t[-extra:].float()).all())
+
+
+def test_pruning_a_matrix_of_more_than_2_31_elements(B, oracle):
+    """W[65792 x 32768] (2^31 + 8.4 M elements, 4.3 GB): a seeded 256-row block repeated 257 times.  Both
+    pruning passes work on groups inside 128 x 128 tiles, so every 256-row slab of the outputs must equal
+    the oracle's outputs for the block; the first, a middle and the last slab are compared bit for bit."""
+    import torch
+
+    blk, reps, d_in = 256, 257, 32768
+    d_out = blk * reps
+    Wb = si.gaussian_bf16((blk, d_in), 0.02, 911)
+    vals_b, nib_b, mask_b = oracle.prune24(Wb)
+    valsT_b, nibT_b, mask2_b = oracle.double_prune(Wb, mask_b)
+    meta_b = oracle.canonical_to_hw(oracle.pack_canonical(nib_b))            # 2 row blocks x 256 column blocks
+    metaT_b = oracle.canonical_to_hw(oracle.pack_canonical(nibT_b)).reshape(d_in // 128, 2, 2048)
+    small = B.bf16_from_bits(Wb)
+    W = torch.empty((d_out, d_in), dtype=torch.bfloat16, device="cuda")
+    W.view(reps, blk, d_in).copy_(small.unsqueeze(0).expand(reps, blk, d_in))
+    assert W.numel() > 2 ** 31
+    vals, meta, mask1 = B.alloc_compressed(d_out, d_in)
+    valsT, metaT, _ = B.alloc_compressed(d_in, d_out)
+    mask2 = torch.empty_like(mask1)
+    B.slope_prune_24(W, vals, meta, mask1)
+    B.slope_double_prune(W, mask1, valsT, metaT, mask2)
+    assert B.slope_poll_status() == 0
+    meta_rows = meta.view(d_out // 128, (d_in // 128) * 2048)
+    metaT_blocks = metaT.view(d_in // 128, d_out // 128, 2048)
+    for t in (0, 131, reps - 1):
+        rows = slice(t * blk, (t + 1) * blk)
+        assert np.array_equal(B.bits_from_bf16(vals[rows]), vals_b), t
+        assert np.array_equal(mask1[rows].cpu().numpy(), mask_b), t
+        assert np.array_equal(mask2[rows].cpu().numpy(), mask2_b), t
+        assert np.array_equal(meta_rows[2 * t: 2 * t + 2].cpu().numpy().reshape(-1), meta_b.reshape(-1)), t
+        assert np.array_equal(B.bits_from_bf16(valsT[:, t * (blk // 2): (t + 1) * (blk // 2)].contiguous()), valsT_b), t
+        assert np.array_equal(metaT_blocks[:, 2 * t: 2 * t + 2].contiguous().cpu().numpy(), metaT_b), t
