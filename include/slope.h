@@ -88,6 +88,11 @@ slope_status_t slope_double_prune(const void* W, const void* mask1_bits, int d_o
  * Eq. (concat):  Y[b x d_out] = X[b x d_in] (W^R)^T  (+ T[b x r] R[r x d_out]).
  * Wc_vals / Wc_meta come from slope_prune_24.  T = X L is produced by
  * slope_adapter_fwd_bwd(phase 0).  r = 0 (T, R ignored) leaves the adapter out.
+ * With b <= 256 (inference, decode: the paper's forward-only inference measurements) the
+ * same call runs on a kernel that streams the compressed weight once from HBM and splits the
+ * reduction over a thread-block cluster; that launch is issued with programmatic stream
+ * serialisation and synchronises on the device before it touches memory, so stream order
+ * holds as for any other call.  All calls of this library can be captured in CUDA graphs.
  */
 slope_status_t slope_linear_fwd(const void* X, int b, const void* Wc_vals, const void* Wc_meta,
                                 int d_out, int d_in, const void* T, const void* R, int r,
