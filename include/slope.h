@@ -92,7 +92,8 @@ slope_status_t slope_double_prune(const void* W, const void* mask1_bits, int d_o
  * same call runs on a kernel that streams the compressed weight once from HBM and splits the
  * reduction over a thread-block cluster; that launch is issued with programmatic stream
  * serialisation and synchronises on the device before it touches memory, so stream order
- * holds as for any other call.  All calls of this library can be captured in CUDA graphs.
+ * holds as for any other call.  Every compute call of this library can be captured in a CUDA
+ * graph (slope_poll_status synchronises the stream and cannot).
  */
 slope_status_t slope_linear_fwd(const void* X, int b, const void* Wc_vals, const void* Wc_meta,
                                 int d_out, int d_in, const void* T, const void* R, int r,
