@@ -543,6 +543,29 @@ __device__ __forceinline__ void raster_tile(int tile, int num_m, int num_n, int&
     n = local / gm;
 }
 
+// Work items of the persistent CTA-pair GEMM.  Items are tiles in raster order; when the tiles
+// left over after the last full round of the machine (num_tiles mod num_pairs) fill at most
+// half of the pairs, each of them is cut into two half-width items, so that the last round
+// takes half the time instead of a full tile time on a half-empty machine (4096 x 4096 weight
+// gradient: 256 tiles on 74 pairs = 3 rounds + 34 tiles -> 68 half items: 3.5 instead of 4 rounds).
+struct PairWork {
+    int m_pair, n0, width;
+};
+template <int BLOCK_N, bool SPLIT_TAIL>
+__device__ __forceinline__ bool pair_work(int item, int num_pairs, int num_m, int num_n, PairWork& w) {
+    const int num_tiles = num_m * num_n;
+    const int full = (num_tiles / num_pairs) * num_pairs, rem = num_tiles - full;
+    const bool split = SPLIT_TAIL && rem > 0 && 2 * rem <= num_pairs;
+    if (item >= (split ? full + 2 * rem : num_tiles)) return false;
+    const bool halved = split && item >= full;
+    const int tile = halved ? full + ((item - full) >> 1) : item;
+    int n_blk;
+    raster_tile(tile, num_m, num_n, w.m_pair, n_blk);
+    w.width = halved ? BLOCK_N / 2 : BLOCK_N;
+    w.n0 = n_blk * BLOCK_N + (halved && ((item - full) & 1) ? BLOCK_N / 2 : 0);
+    return true;
+}
+
 // Dense CTA-pair GEMM: D[M x N] = A[M x K] * B[N x K]^T with a 256 x BLOCK_N tile per pair
 // (each CTA: 128 rows of A, BLOCK_N/2 rows of B, 128 x BLOCK_N accumulator rows).
 template <int BLOCK_N, int STAGES>
@@ -576,7 +599,8 @@ dense_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     const int num_m = (p.M + 2 * kBlockM - 1) / (2 * kBlockM);
     const int num_n = (p.N + BLOCK_N - 1) / BLOCK_N;
     const int num_kb = (p.K + 63) / 64;
-    const int num_tiles = num_m * num_n;
+    // halving needs B loads of any width: the [K x N] operand is loaded in 64-column chunks
+    constexpr bool kSplitTail = B_MN && BLOCK_N == 256;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
@@ -600,17 +624,19 @@ dense_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
             tma_prefetch_desc(&tmB);
             PipeState ps;
             bool ok = true;
-            for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
-                int m_pair, n_blk;
-                raster_tile(tile, num_m, num_n, m_pair, n_blk);
-                const int m0 = (m_pair * 2 + static_cast<int>(cta)) * kBlockM;
-                const int n0 = n_blk * BLOCK_N + static_cast<int>(cta) * Cfg::kHalfN;
+            PairWork w;
+            for (int item = pair_id; ok && pair_work<BLOCK_N, kSplitTail>(item, num_pairs, num_m, num_n, w);
+                 item += num_pairs) {
+                const int half_w = w.width / 2;                       // B rows (columns of D) this CTA stages
+                const int m0 = (w.m_pair * 2 + static_cast<int>(cta)) * kBlockM;
+                const int n0 = w.n0 + static_cast<int>(cta) * half_w;
+                const uint32_t stage_tx = kSplitTail ? 2 * (Cfg::kABytes + half_w * 128) : 2 * Cfg::kStageBytes;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&empty_bar[ps.stage], ps.phase ^ 1u, abort_flag)) { ok = false; break; }
                     uint8_t* sA = smem + ps.stage * Cfg::kStageBytes;
                     uint8_t* sB = sA + Cfg::kABytes;
                     const uint32_t bar = mapa_shared(smem_u32(&full_bar[ps.stage]), 0);
-                    if (cta == 0) mbar_expect_tx(&full_bar[ps.stage], 2 * Cfg::kStageBytes);
+                    if (cta == 0) mbar_expect_tx(&full_bar[ps.stage], stage_tx);
                     if (A_MN) {
                         tma_load_2d_pair(sA, &tmA, bar, m0, kb * 64);
                         tma_load_2d_pair(sA + 8192, &tmA, bar, m0 + 64, kb * 64);
@@ -620,7 +646,7 @@ dense_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                     if (B_MN) {
 #pragma unroll
                         for (int h = 0; h < Cfg::kHalfN / 64; ++h)
-                            tma_load_2d_pair(sB + h * 8192, &tmB, bar, n0 + h * 64, kb * 64);
+                            if (h * 64 < half_w) tma_load_2d_pair(sB + h * 8192, &tmB, bar, n0 + h * 64, kb * 64);
                     } else {
                         tma_load_2d_pair(sB, &tmB, bar, kb * 64, n0);
                     }
@@ -630,11 +656,15 @@ dense_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         }
     } else if (warp == 1) {
         if (cta == 0 && elect_one()) {
-            constexpr uint32_t idesc = make_idesc_bf16(2 * kBlockM, BLOCK_N, A_MN, B_MN, false);
+            constexpr uint32_t idesc_full = make_idesc_bf16(2 * kBlockM, BLOCK_N, A_MN, B_MN, false);
+            constexpr uint32_t idesc_half = make_idesc_bf16(2 * kBlockM, BLOCK_N / 2, A_MN, B_MN, false);
             PipeState ps;
             bool ok = true;
             int it = 0;
-            for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
+            PairWork w;
+            for (int item = pair_id; ok && pair_work<BLOCK_N, kSplitTail>(item, num_pairs, num_m, num_n, w);
+                 item += num_pairs, ++it) {
+                const uint32_t idesc = w.width == BLOCK_N ? idesc_full : idesc_half;
                 const int acc = it & 1;
                 const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
                 if (!mbar_wait(&tempty_bar[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -663,9 +693,10 @@ dense_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
         const int q = warp & 3;
         bool ok = true;
         int it = 0;
-        for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
-            int m_pair, n_blk;
-            raster_tile(tile, num_m, num_n, m_pair, n_blk);
+        PairWork w;
+        for (int item = pair_id; ok && pair_work<BLOCK_N, kSplitTail>(item, num_pairs, num_m, num_n, w);
+             item += num_pairs, ++it) {
+            const int m_pair = w.m_pair;
             const int acc = it & 1;
             const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
             if (!mbar_wait(&tfull_bar[acc], acc_phase, abort_flag)) { ok = false; break; }
@@ -673,11 +704,11 @@ dense_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
             const uint32_t t_row = tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
             const int m = (m_pair * 2 + static_cast<int>(cta)) * kBlockM + q * 32 + lane;
 #pragma unroll 1
-            for (int c0 = 0; c0 < BLOCK_N; c0 += 16) {
+            for (int c0 = 0; c0 < w.width; c0 += 16) {
                 uint32_t v[16];
                 tmem_ld_16(t_row + c0, v);
                 tmem_ld_wait();
-                const int n0 = n_blk * BLOCK_N + c0;
+                const int n0 = w.n0 + c0;
                 if (m >= p.M || n0 >= p.N) continue;
                 if (EPI == kEpiStore) {
                     uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + static_cast<size_t>(m) * p.N + n0);
