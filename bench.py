@@ -402,7 +402,7 @@ def main():
     sp_fl = tot["linear_fwd"][0] + tot["linear_bwd_dx"][0]
     sp_s = tot["linear_fwd"][1] + tot["linear_bwd_dx"][1]
     sp_tflops = sp_fl / sp_s / 1e12 if sp_s else 0.0
-    roofline_sparse = {"kernel": "sparse_gemm_pair_kernel<224,4> + sparse_gemm_quad_kernel<224,3> (slope_linear_fwd, slope_linear_bwd_dx)", "bound": "tensor",
+    roofline_sparse = {"kernel": "sparse_gemm_quad_kernel<224,3> (slope_linear_fwd, slope_linear_bwd_dx; sparse_gemm_pair_kernel<224,4> below a reduction length of 4096)", "bound": "tensor",
                        "achieved": round(sp_tflops, 1), "peak": round(sparse_peak, 1),
                        "unit": "TFLOP/s", "frac": round(sp_tflops / sparse_peak, 4), "traffic": None,
                        "ms_per_step": round(sp_s * 1e3, 4),
@@ -413,12 +413,15 @@ def main():
     # dram__bytes_read + write per launch from the 1-pass ncu capture at these sizes
     # (profiles/dram_traffic_full_size_c3_llama7b.md), averaged over the launches of a step.
     if wl.key in ("c3_llama7b", "c4_llama7b_adapter") and b == 16384:
-        sp_reads = 4 * (153.2 + 153.3) + 2 * (526.8 + 791.9) + (792.3 + 527.1)
-        sp_writes = 4 * (104.0 + 100.1) + 2 * (340.0 + 145.0) + (145.0 + 339.4)
+        sp_reads = (154.8 + 154.8 + 164.3 + 155.8 + 163.8 + 154.7 + 154.7 + 154.4) + (825.4 + 792.7) + (827.3 + 792.4) \
+            + (792.0 + 791.1)
+        sp_writes = (109.1 + 105.7 + 108.3 + 106.1 + 106.1 + 106.3 + 105.5 + 105.0) + (393.2 + 145.2) + (390.2 + 145.0) \
+            + (145.3 + 391.4)
         roofline_sparse["traffic"] = round((sp_reads + sp_writes) / 14 * 1e6)
         roofline_sparse["traffic_note"] = "mean DRAM bytes per launch over the 14 sparse GEMM launches of a step (ncu, no adapter operands)"
         roofline_sparse["algorithmic_bytes"] = round((4 * 2 * (153.1 + 134.2) + 2 * (184.9 + 360.7 + 411.4 + 134.2) + (411.4 + 134.2 + 184.9 + 360.7)) / 14 * 1e6)
-        dw_traffic = 4 * (630.3 + 14.3) + 2 * (1820.0 + 43.3) + (1540.0 + 43.0)
+        dw_traffic = (630.5 + 17.0) + (630.7 + 14.1) + (630.5 + 14.2) + (630.5 + 14.0) + (1975.8 + 42.6) \
+            + (1945.8 + 42.6) + (1603.8 + 42.4)
         roofline_dense["traffic"] = round(dw_traffic / 7 * 1e6)
         roofline_dense["algorithmic_bytes"] = round((4 * (270.5 + 16.8) + 3 * (500.5 + 45.1)) / 7 * 1e6)
     sparse_dominant = sp_s >= dw_s

@@ -51,6 +51,7 @@ __device__ __forceinline__ void drain_after_abort() {
 struct SparseGemmParams {
     int M, K, Ntok, r;
     int a2_mn_major;              // 1: A2 is stored [r x M] (M contiguous)
+    int group_m;                  // 512-row-tile kernel: row tiles per raster group (0: all in one group)
     const uint8_t* meta;          // metadata blocks of A
     uint16_t* out;                // [Ntok x M]
 };
@@ -787,6 +788,23 @@ struct SparseQuadCfg {
     static_assert(kSmemBytes <= 232448, "shared memory budget");
 };
 
+// Tile order of the 512-row-tile kernel: row tiles fastest inside a group of `group_m` row tiles,
+// then token blocks, then the next group.  The pairs that work on one token block side by side
+// share its activation tile; a group's share of the compressed weight is what has to stay in L2
+// while the token blocks sweep by.  `first` marks the tile that prefetches the block's
+// activations into L2 for its group.
+__device__ __forceinline__ void quad_tile(int tile, int num_m, int num_n, int group_m, int& mt, int& n_blk,
+                                          bool& first) {
+    const int group_size = group_m * num_n;
+    const int g = tile / group_size;
+    const int first_m = g * group_m;
+    const int gm = min(num_m - first_m, group_m);
+    const int local = tile - g * group_size;
+    mt = first_m + local % gm;
+    n_blk = local / gm;
+    first = local % gm == 0;
+}
+
 template <int BLOCK_N, int STAGES>
 __global__ void __launch_bounds__(SparseQuadCfg<BLOCK_N, STAGES>::kThreads, 1)
 sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -813,6 +831,7 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     const int num_kb = p.K / 128;
     const int num_ab = (p.r + 63) / 64;
     const int total_kb = num_kb + num_ab;
+    const int group_m = p.group_m > 0 && p.group_m < num_m ? p.group_m : num_m;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
@@ -842,23 +861,26 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             PipeState ps;
             bool ok = true;
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
-                const int mt = tile % num_m, n_blk = tile / num_m;
+                int mt, n_blk, next_mt, next_n_blk;
+                bool first, next_first = false;
+                quad_tile(tile, num_m, num_n, group_m, mt, n_blk, first);
                 const int nsub = (4 * mt + 2 < num_mb) ? 2 : 1;              // second sub-tile may lie past M
                 const int n_row0 = n_blk * BLOCK_N + static_cast<int>(cta) * Cfg::kHalfN;
                 // The pairs working on the same token block (same n_blk, different mt) run side by
                 // side and would all wait on the same first-touch DRAM fetch of an activation box.
                 // One of them (mt == 0) pulls the boxes into L2 kPrefetchAhead k-blocks early.
                 const int next_tile = tile + num_pairs;
-                const int next_row0 = (next_tile / num_m) * BLOCK_N + static_cast<int>(cta) * Cfg::kHalfN;
+                if (next_tile < num_tiles) quad_tile(next_tile, num_m, num_n, group_m, next_mt, next_n_blk, next_first);
+                const int next_row0 = next_first ? next_n_blk * BLOCK_N + static_cast<int>(cta) * Cfg::kHalfN : 0;
                 for (int kb = 0; kb < total_kb; ++kb) {
                     if (kb < num_kb) {
                         const int pk = kb + kPrefetchAhead;
                         if (pk < num_kb) {
-                            if (mt == 0) {
+                            if (first) {
                                 tma_prefetch_l2_2d(&tmB, pk * 128, n_row0);
                                 tma_prefetch_l2_2d(&tmB, pk * 128 + 64, n_row0);
                             }
-                        } else if (next_tile < num_tiles && next_tile % num_m == 0 && pk - num_kb < num_kb) {
+                        } else if (next_first && pk - num_kb < num_kb) {
                             tma_prefetch_l2_2d(&tmB, (pk - num_kb) * 128, next_row0);
                             tma_prefetch_l2_2d(&tmB, (pk - num_kb) * 128 + 64, next_row0);
                         }
@@ -909,7 +931,9 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             bool ok = true;
             int it = 0;
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
-                const int mt = tile % num_m;
+                int mt, n_blk_unused;
+                bool first_unused;
+                quad_tile(tile, num_m, num_n, group_m, mt, n_blk_unused, first_unused);
                 const int nsub = (4 * mt + 2 < num_mb) ? 2 : 1;
                 const uint32_t acc_phase = static_cast<uint32_t>(it) & 1u;
                 for (int kb = 0; ok && kb < total_kb; ++kb) {
@@ -973,7 +997,9 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         int it = 0;
         uint32_t buf = 0;
         for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
-            const int mt = tile % num_m, n_blk = tile / num_m;
+            int mt, n_blk;
+            bool first_unused;
+            quad_tile(tile, num_m, num_n, group_m, mt, n_blk, first_unused);
             const int nsub = (4 * mt + 2 < num_mb) ? 2 : 1;
             if (!mbar_wait(&tfull_bar[0], static_cast<uint32_t>(it) & 1u, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();

@@ -246,7 +246,7 @@ static slope_status_t launch_sparse_pair(const void* act, int ntok, const void* 
         tmA2 = tmA;
         tmB2 = tmB;
     }
-    SparseGemmParams p;
+    SparseGemmParams p = {};
     p.M = M; p.K = K; p.Ntok = ntok; p.r = r; p.a2_mn_major = a2_mn ? 1 : 0;
     p.meta = static_cast<const uint8_t*>(meta);
     p.out = static_cast<uint16_t*>(out);
@@ -260,6 +260,30 @@ static slope_status_t launch_sparse_pair(const void* act, int ntok, const void* 
 
 constexpr int kQuadBlockN = 224;
 constexpr int kQuadStages = 3;
+
+// Row tiles per raster group of the 512-row-tile kernel (see quad_tile).  All pairs that work on
+// one token block share its activations, so with every row tile in one group the activations
+// cross HBM once -- but a round of the machine then touches the whole compressed weight, and
+// when that is more than L2 keeps next to the streams (about 30 MB here) it is fetched again
+// every round.  Splitting the row tiles into g groups re-reads the activations g times and keeps
+// a group's weights resident.  Pick the g with the least estimated DRAM traffic
+// (measured at 16384 tokens: 4096 -> 11008 two groups +7 %, 5120 -> 13824 three groups +11 %,
+// square and long-reduction layers one group).
+static int quad_group_m(int M, int K, int ntok, int num_pairs) {
+    const int num_m = (M / kBlockM + 3) / 4, num_n = (ntok + kPairBlockN - 1) / kPairBlockN;
+    const double w_tile = 512.0 * K * 1.125, w_total = static_cast<double>(M) * K * 1.125;
+    const double x_total = static_cast<double>(ntok) * K * 2.0;
+    constexpr double kL2Keeps = 30e6;
+    int best_gm = num_m;
+    double best = 1e300;
+    for (int g = 1; g <= num_m; ++g) {
+        const int gm = (num_m + g - 1) / g, groups = (num_m + gm - 1) / gm;
+        const double rounds = static_cast<double>(gm) * num_n / num_pairs;
+        const double traffic = groups * x_total + (gm * w_tile <= kL2Keeps ? w_total : w_total * (rounds > 1.0 ? rounds : 1.0));
+        if (traffic < best * 0.98) { best = traffic; best_gm = gm; }       // prefer fewer groups on a near tie
+    }
+    return best_gm;
+}
 
 static slope_status_t launch_sparse_quad(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                          const void* act2, const void* fac2, int r, bool a2_mn, void* out,
@@ -277,10 +301,11 @@ static slope_status_t launch_sparse_quad(const void* act, int ntok, const void* 
         tmA2 = tmA;
         tmB2 = tmB;
     }
-    SparseGemmParams p;
+    SparseGemmParams p = {};
     p.M = M; p.K = K; p.Ntok = ntok; p.r = r; p.a2_mn_major = a2_mn ? 1 : 0;
     p.meta = static_cast<const uint8_t*>(meta);
     p.out = static_cast<uint16_t*>(out);
+    p.group_m = quad_group_m(M, K, ntok, info.sm_count / 2);
     auto kern = sparse_gemm_quad_kernel<kQuadBlockN, kQuadStages>;
     if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
     const int tiles = ((M / kBlockM + 3) / 4) * ((ntok + kQuadBlockN - 1) / kQuadBlockN);
@@ -344,7 +369,7 @@ static slope_status_t launch_sparse_skinny(const void* act, int ntok, const void
         tmA2 = tmA;
         tmB2 = tmB;
     }
-    SparseGemmParams p;
+    SparseGemmParams p = {};
     p.M = M; p.K = K; p.Ntok = ntok; p.r = r; p.a2_mn_major = a2_mn ? 1 : 0;
     p.meta = static_cast<const uint8_t*>(meta);
     p.out = static_cast<uint16_t*>(out);
@@ -389,14 +414,15 @@ static slope_status_t launch_skinny(const void* act, int ntok, const void* vals,
 // Kernel choice for the sparse GEMMs.  Up to 256 tokens the GEMM is a weight stream from HBM and
 // runs on the skinny kernel.  Beyond that: the 512-row tile moves 31 % fewer L2 bytes per FLOP but
 // cannot overlap its epilogue with the next tile (tensor memory holds only one accumulator
-// set); that pays off once the reduction is long.  Short reductions keep the 256-row tile
-// with double-buffered accumulators.
+// set); measured, that pays off from a reduction length of 4096 on (16384 tokens: 4096 x 4096
+// +6 %, 11008 x 4096 +1 %, 4096 x 11008 +16 %), while at 768 the 256-row tile with its
+// double-buffered accumulators is up to 25 % faster.
 static slope_status_t launch_sparse_gemm(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                          const void* act2, const void* fac2, int r, bool a2_mn, void* out,
                                          cudaStream_t stream, const DeviceInfo& info) {
     if (ntok <= kSkinnyMaxTokens)
         return launch_skinny(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
-    return K >= 6144 ? launch_sparse_quad(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info)
+    return K >= 4096 ? launch_sparse_quad(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info)
                      : launch_sparse_pair(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
 }
 
