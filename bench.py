@@ -413,15 +413,15 @@ def main():
     # dram__bytes_read + write per launch from the 1-pass ncu capture at these sizes
     # (profiles/dram_traffic_full_size_c3_llama7b.md), averaged over the launches of a step.
     if wl.key in ("c3_llama7b", "c4_llama7b_adapter") and b == 16384:
-        sp_reads = (154.8 + 154.8 + 164.3 + 155.8 + 163.8 + 154.7 + 154.7 + 154.4) + (825.4 + 792.7) + (827.3 + 792.4) \
-            + (792.0 + 791.1)
-        sp_writes = (109.1 + 105.7 + 108.3 + 106.1 + 106.1 + 106.3 + 105.5 + 105.0) + (393.2 + 145.2) + (390.2 + 145.0) \
-            + (145.3 + 391.4)
+        sp_reads = (154.9 + 154.5 + 155.4 + 155.6 + 154.6 + 165.5 + 154.7 + 154.6) + (374.3 + 792.3) + (376.9 + 792.6) \
+            + (792.5 + 361.9)
+        sp_writes = (109.0 + 105.8 + 107.5 + 106.2 + 106.5 + 106.0 + 105.2 + 105.8) + (356.7 + 146.5) + (358.2 + 146.8) \
+            + (146.5 + 356.3)
         roofline_sparse["traffic"] = round((sp_reads + sp_writes) / 14 * 1e6)
         roofline_sparse["traffic_note"] = "mean DRAM bytes per launch over the 14 sparse GEMM launches of a step (ncu, no adapter operands)"
         roofline_sparse["algorithmic_bytes"] = round((4 * 2 * (153.1 + 134.2) + 2 * (184.9 + 360.7 + 411.4 + 134.2) + (411.4 + 134.2 + 184.9 + 360.7)) / 14 * 1e6)
-        dw_traffic = (630.5 + 17.0) + (630.7 + 14.1) + (630.5 + 14.2) + (630.5 + 14.0) + (1975.8 + 42.6) \
-            + (1945.8 + 42.6) + (1603.8 + 42.4)
+        dw_traffic = (630.4 + 14.2) + (630.6 + 14.2) + (630.4 + 14.5) + (630.4 + 14.2) + (1948.5 + 42.8) \
+            + (1990.3 + 42.6) + (1648.1 + 42.5)
         roofline_dense["traffic"] = round(dw_traffic / 7 * 1e6)
         roofline_dense["algorithmic_bytes"] = round((4 * (270.5 + 16.8) + 3 * (500.5 + 45.1)) / 7 * 1e6)
     sparse_dominant = sp_s >= dw_s
