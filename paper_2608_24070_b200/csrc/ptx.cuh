@@ -217,8 +217,12 @@ __device__ __forceinline__ uint32_t mapa_shared(uint32_t local_saddr, uint32_t r
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_saddr), "r"(rank));
     return r;
 }
+// Arrive on an mbarrier of a CTA of the cluster.  Used to hand a drained tensor-memory accumulator
+// back to the MMA issuer: what has to be ordered is the tcgen05.ld traffic (tcgen05.wait::ld and
+// tcgen05.fence::before_thread_sync precede the call), not memory, so no cluster-scope release is
+// attached -- that fence cost every epilogue warp about 1.3 us per tile.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_saddr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_saddr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_saddr) : "memory");
 }
 // 2-D tiled load into this CTA's shared memory whose completion bytes are counted on an
 // mbarrier that may live in the other CTA of the pair (`bar_cluster_saddr`).  No multicast.
