@@ -816,8 +816,8 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + Cfg::kOffBar);
     uint64_t* empty_bar = full_bar + STAGES;
-    uint64_t* tfull_bar = empty_bar + STAGES;                // [1]
-    uint64_t* tempty_bar = tfull_bar + 1;                    // [2], one per sub-tile accumulator
+    uint64_t* tfull_bar = empty_bar + STAGES;                // [2], one per sub-tile accumulator
+    uint64_t* tempty_bar = tfull_bar + 2;                    // [2]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -836,6 +836,7 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         mbar_init(&tfull_bar[0], 1);
+        mbar_init(&tfull_bar[1], 1);
         mbar_init(&tempty_bar[0], 2 * Cfg::kEpiWarps);
         mbar_init(&tempty_bar[1], 2 * Cfg::kEpiWarps);
         *abort_flag = 0;
@@ -970,12 +971,15 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                                 umma_bf16_pair(d_tmem, ad, bd, idesc_ad, 1u);
                             }
                         }
+                        // sub-tile s is complete with its last k-block: its drain may start while the
+                        // other sub-tile's last MMAs still run
+                        if (kb == total_kb - 1) umma_commit_pair(&tfull_bar[s], 3);
                     }
                     if (!ok) break;
                     umma_commit_pair(&empty_bar[ps.stage], 3);
                     ps.advance(STAGES);
                 }
-                if (ok) umma_commit_pair(&tfull_bar[0], 3);
+                if (ok && nsub == 1) umma_commit_pair(&tfull_bar[1], 3);        // keep both barriers in phase
             }
         }
     } else {
@@ -1001,33 +1005,58 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             bool first_unused;
             quad_tile(tile, num_m, num_n, group_m, mt, n_blk, first_unused);
             const int nsub = (4 * mt + 2 < num_mb) ? 2 : 1;
+            uint32_t pk[2][kMyBlocks][16];
+            // ---- first accumulator (its drain is what the next tile's first MMA waits for).  Two
+            //      16-column loads in flight per wait: the warps of a 320-thread CTA are allocated
+            //      registers as twelve, which caps a thread at 168, and 128 of them hold the two
+            //      packed accumulators.
             if (!mbar_wait(&tfull_bar[0], static_cast<uint32_t>(it) & 1u, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
-            uint32_t pk[2][kMyBlocks][16];
+            {
+                const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
 #pragma unroll
-            for (int s = 0; s < 2; ++s) {
-                if (s < nsub) {
-                    const uint32_t t_row = tmem_base + s * BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
+                for (int j = 0; j < kMyBlocks; ++j) {
+                    const int c0 = (2 * j + half) * Cfg::kStoreRows;
+                    if (c0 < BLOCK_N) {
+                        uint32_t v0[16], v1[16];
+                        tmem_ld_16(t_row + c0, v0);
+                        tmem_ld_16(t_row + c0 + 16, v1);
+                        tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < kMyBlocks; ++j) {
-                        const int c0 = (2 * j + half) * Cfg::kStoreRows;
-                        if (c0 < BLOCK_N) {
-                            uint32_t v0[16], v1[16];
-                            tmem_ld_16(t_row + c0, v0);
-                            tmem_ld_16(t_row + c0 + 16, v1);
-                            tmem_ld_wait();
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                pk[s][j][i] = pack_bf16x2(__uint_as_float(v0[2 * i]), __uint_as_float(v0[2 * i + 1]));
-                                pk[s][j][8 + i] = pack_bf16x2(__uint_as_float(v1[2 * i]), __uint_as_float(v1[2 * i + 1]));
-                            }
+                        for (int i = 0; i < 8; ++i) {
+                            pk[0][j][i] = pack_bf16x2(__uint_as_float(v0[2 * i]), __uint_as_float(v0[2 * i + 1]));
+                            pk[0][j][8 + i] = pack_bf16x2(__uint_as_float(v1[2 * i]), __uint_as_float(v1[2 * i + 1]));
                         }
                     }
                 }
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&tempty_bar[s]), 0));
             }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&tempty_bar[0]), 0));
+            // ---- second accumulator
+            if (!mbar_wait(&tfull_bar[1], static_cast<uint32_t>(it) & 1u, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            if (nsub == 2) {
+                const uint32_t t_row = tmem_base + BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
+#pragma unroll
+                for (int j = 0; j < kMyBlocks; ++j) {
+                    const int c0 = (2 * j + half) * Cfg::kStoreRows;
+                    if (c0 < BLOCK_N) {
+                        uint32_t v0[16], v1[16];
+                        tmem_ld_16(t_row + c0, v0);
+                        tmem_ld_16(t_row + c0 + 16, v1);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            pk[1][j][i] = pack_bf16x2(__uint_as_float(v0[2 * i]), __uint_as_float(v0[2 * i + 1]));
+                            pk[1][j][8 + i] = pack_bf16x2(__uint_as_float(v1[2 * i]), __uint_as_float(v1[2 * i + 1]));
+                        }
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&tempty_bar[1]), 0));
 #pragma unroll
             for (int s = 0; s < 2; ++s) {
                 if (s < nsub) {
