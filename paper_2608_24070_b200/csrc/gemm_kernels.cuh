@@ -928,7 +928,37 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         if (cta == 0 && elect_one()) {
             constexpr uint32_t idesc_sp = make_idesc_bf16(2 * kBlockM, BLOCK_N, false, false, true);
             const uint32_t idesc_ad = make_idesc_bf16(2 * kBlockM, BLOCK_N, p.a2_mn_major != 0, false, false);
-            PipeState ps;
+            // the MMAs of sub-tile s for k-block kb out of pipeline stage `stage`
+            auto issue = [&](int s, int kb, int stage) {
+                const uint32_t st = smem_u32(smem + stage * Cfg::kStageBytes);
+                const uint32_t sB = st + Cfg::kOffB;
+                const uint32_t d_tmem = tmem_base + s * BLOCK_N;
+                const uint32_t sA = st + s * Cfg::kABytes;
+                if (kb < num_kb) {
+                    const uint32_t e_tmem = tmem_base + Cfg::kECol + (kb & 1) * 8 + s * 4;
+                    tmem_cp_128x128b_pair(e_tmem, make_smem_desc(st + Cfg::kOffE + s * Cfg::kEBytes, 128, 128,
+                                                                 kSwizzleNone));
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint64_t ad = make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
+                        const uint64_t bd = make_smem_desc(sB + (j >> 1) * (Cfg::kHalfN * 128) + (j & 1) * 64, 16, 1024,
+                                                           kSwizzle128B);
+                        umma_bf16_sp_pair(d_tmem, ad, bd, e_tmem + (j & 2), idesc_sp | (j & 1), (kb | j) != 0 ? 1u : 0u);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint64_t ad = p.a2_mn_major ? make_smem_desc(sA + j * 2048, 8192, 1024, kSwizzle128B)
+                                                          : make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
+                        const uint64_t bd = make_smem_desc(sB + j * 32, 16, 1024, kSwizzle128B);
+                        umma_bf16_pair(d_tmem, ad, bd, idesc_ad, 1u);
+                    }
+                }
+                // sub-tile s is complete with its last k-block: its drain may start while the other
+                // sub-tile's last MMAs still run
+                if (kb == total_kb - 1) umma_commit_pair(&tfull_bar[s], 3);
+            };
+            PipeState ps;                                     // stage that sub-tile 0 consumes next
             bool ok = true;
             int it = 0;
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
@@ -936,46 +966,43 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 bool first_unused;
                 quad_tile(tile, num_m, num_n, group_m, mt, n_blk_unused, first_unused);
                 const int nsub = (4 * mt + 2 < num_mb) ? 2 : 1;
-                const uint32_t acc_phase = static_cast<uint32_t>(it) & 1u;
-                for (int kb = 0; ok && kb < total_kb; ++kb) {
+                const uint32_t acc_parity = (static_cast<uint32_t>(it) & 1u) ^ 1u;
+                if (!mbar_wait(&tempty_bar[0], acc_parity, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                // The epilogue hands the second accumulator back a little after the first.  Until
+                // then sub-tile 0 runs ahead through the stages that are already full (they cannot
+                // be released before sub-tile 1 has used them too); then sub-tile 1 catches up.
+                PipeState pc = ps;                            // stage that sub-tile 1 consumes (and releases) next
+                int kb0 = 0;
+                bool ready1 = nsub == 1;
+                while (ok && !ready1) {
+                    ready1 = mbar_test(&tempty_bar[1], acc_parity);
+                    if (ready1) break;
+                    if (kb0 < total_kb && kb0 < STAGES) {
+                        if (!mbar_wait(&full_bar[ps.stage], ps.phase, abort_flag)) { ok = false; break; }
+                        tc_fence_after_sync();
+                        issue(0, kb0, ps.stage);
+                        ps.advance(STAGES);
+                        ++kb0;
+                    } else {
+                        ok = mbar_wait(&tempty_bar[1], acc_parity, abort_flag);
+                        ready1 = true;
+                    }
+                }
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (nsub == 2) {
+                    for (int kb1 = 0; kb1 < kb0; ++kb1) {       // catch up
+                        issue(1, kb1, pc.stage);
+                        umma_commit_pair(&empty_bar[pc.stage], 3);
+                        pc.advance(STAGES);
+                    }
+                }
+                for (int kb = kb0; kb < total_kb; ++kb) {        // in step
                     if (!mbar_wait(&full_bar[ps.stage], ps.phase, abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t st = smem_u32(smem + ps.stage * Cfg::kStageBytes);
-                    const uint32_t sB = st + Cfg::kOffB;
-                    for (int s = 0; s < nsub; ++s) {
-                        if (kb == 0) {                        // accumulator s must have been drained
-                            if (!mbar_wait(&tempty_bar[s], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
-                            tc_fence_after_sync();
-                        }
-                        const uint32_t d_tmem = tmem_base + s * BLOCK_N;
-                        const uint32_t sA = st + s * Cfg::kABytes;
-                        if (kb < num_kb) {
-                            const uint32_t e_tmem = tmem_base + Cfg::kECol + (kb & 1) * 8 + s * 4;
-                            tmem_cp_128x128b_pair(e_tmem, make_smem_desc(st + Cfg::kOffE + s * Cfg::kEBytes, 128, 128,
-                                                                         kSwizzleNone));
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const uint64_t ad = make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
-                                const uint64_t bd = make_smem_desc(sB + (j >> 1) * (Cfg::kHalfN * 128) + (j & 1) * 64,
-                                                                   16, 1024, kSwizzle128B);
-                                umma_bf16_sp_pair(d_tmem, ad, bd, e_tmem + (j & 2), idesc_sp | (j & 1),
-                                                  (kb | j) != 0 ? 1u : 0u);
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const uint64_t ad = p.a2_mn_major
-                                                        ? make_smem_desc(sA + j * 2048, 8192, 1024, kSwizzle128B)
-                                                        : make_smem_desc(sA + j * 32, 16, 1024, kSwizzle128B);
-                                const uint64_t bd = make_smem_desc(sB + j * 32, 16, 1024, kSwizzle128B);
-                                umma_bf16_pair(d_tmem, ad, bd, idesc_ad, 1u);
-                            }
-                        }
-                        // sub-tile s is complete with its last k-block: its drain may start while the
-                        // other sub-tile's last MMAs still run
-                        if (kb == total_kb - 1) umma_commit_pair(&tfull_bar[s], 3);
-                    }
-                    if (!ok) break;
+                    issue(0, kb, ps.stage);
+                    if (nsub == 2) issue(1, kb, ps.stage);
                     umma_commit_pair(&empty_bar[ps.stage], 3);
                     ps.advance(STAGES);
                 }

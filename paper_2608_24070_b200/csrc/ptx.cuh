@@ -51,6 +51,18 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 // One try: the hardware may park the thread for up to kSuspendHintNs while the phase is
 // pending (it wakes as soon as the phase completes), so a waiting role costs no issue slots.
 constexpr uint32_t kSuspendHintNs = 20000;
+// Non-blocking test of a phase (try_wait may suspend the thread for up to the hint).
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
