@@ -412,18 +412,30 @@ static slope_status_t launch_skinny(const void* act, int ntok, const void* vals,
 }
 
 // Kernel choice for the sparse GEMMs.  Up to 256 tokens the GEMM is a weight stream from HBM and
-// runs on the skinny kernel.  Beyond that: the 512-row tile moves 31 % fewer L2 bytes per FLOP but
-// cannot overlap its epilogue with the next tile (tensor memory holds only one accumulator
-// set); measured, that pays off from a reduction length of 4096 on (16384 tokens: 4096 x 4096
-// +6 %, 11008 x 4096 +1 %, 4096 x 11008 +16 %), while at 768 the 256-row tile with its
-// double-buffered accumulators is up to 25 % faster.
+// runs on the few-token kernel.  Beyond that: the 512-row tile moves 31 % fewer L2 bytes per FLOP
+// but cannot overlap its epilogue with the next tile (tensor memory holds only one accumulator
+// set).  Measured at 16384 tokens it is 6 % faster per unit of work at a reduction length of
+// 4096 and 14-16 % at 11008, while at 768 the 256-row tile with its double-buffered accumulators
+// is up to 25 % faster.  The choice compares rounds of the machine (tiles / CTA pairs, rounded
+// up) times the relative cost of a tile, so that a shape whose 512-row tiles fill the last
+// round badly (4096 x 4096 with 4096 tokens: 152 tiles on 74 pairs) keeps the 256-row tile.
+static bool prefer_quad_tile(int M, int K, int ntok, int num_pairs) {
+    const int num_n = (ntok + kPairBlockN - 1) / kPairBlockN;
+    const int tiles_pair = ((M + 255) / 256) * num_n, tiles_quad = ((M + 511) / 512) * num_n;
+    const double gain = K >= 8192 ? 0.14 : K >= 4096 ? 0.06 : K >= 2048 ? -0.05 : -0.25;
+    const double cost_pair = (tiles_pair + num_pairs - 1) / num_pairs;
+    const double cost_quad = 2.0 * (1.0 - gain) * ((tiles_quad + num_pairs - 1) / num_pairs);
+    return cost_quad < cost_pair;
+}
+
 static slope_status_t launch_sparse_gemm(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                          const void* act2, const void* fac2, int r, bool a2_mn, void* out,
                                          cudaStream_t stream, const DeviceInfo& info) {
     if (ntok <= kSkinnyMaxTokens)
         return launch_skinny(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
-    return K >= 4096 ? launch_sparse_quad(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info)
-                     : launch_sparse_pair(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
+    return prefer_quad_tile(M, K, ntok, info.sm_count / 2)
+               ? launch_sparse_quad(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info)
+               : launch_sparse_pair(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
 }
 
 template <bool A_MN, bool B_MN, int BLOCK_N, int EPI, int STAGES>

@@ -105,7 +105,7 @@ CASES = [
     (384, 640, 776, 32, 13),         # ragged token tail, several tiles in every dimension
     (768, 256, 1000, 128, 14),
     (128, 128, 8, 16, 15),           # smallest legal problem
-    (6144, 640, 264, 32, 16),        # forward reduction long enough for the 512-row-tile kernel
+    (6144, 640, 264, 32, 16),        # long forward reduction (48 k-blocks) on the 256-row tile
     (640, 6144, 264, 0, 17),         # same for the input-gradient GEMM
     (4096, 512, 40, 16, 18),         # few tokens: weight-streaming kernel (64-token tile), K split over a cluster
     (1024, 384, 200, 0, 19),         # 200 tokens (256-token tile)
@@ -152,6 +152,39 @@ def test_layer_against_oracle(B, oracle, d_in, d_out, b, r, seed):
         errs["dT"] = rel_fro(g(dT), oracle.adapter_dT_rows(dY, R, rows))
         errs["dL"] = rel_fro(g(dL), oracle.adapter_dL_rows(X, dY, R, np.arange(d_in)))
         errs["dR"] = rel_fro(g(dR), oracle.adapter_dR_cols(X, L, dY, np.arange(d_out)))
+    print(errs)
+    for k, v in errs.items():
+        assert v <= REL_TOL, (k, v, errs)
+
+
+@pytest.mark.parametrize("d_in,d_out,b,r", [(4096, 1024, 4104, 32), (1024, 4096, 4104, 0)])
+def test_512_row_tile_kernel_on_sampled_rows(B, oracle, d_in, d_out, b, r):
+    """Shapes for which the kernel choice takes the 512-row tile (38 tiles fill one round where 76
+    256-row tiles would need two), with a ragged token tail: sampled token rows against the oracle."""
+    W = si.gaussian_bf16((d_out, d_in), 0.02, 131)
+    X = si.gaussian_bf16((b, d_in), 1.0, 132)
+    dY = si.gaussian_bf16((b, d_out), 1.0, 133)
+    L = si.gaussian_bf16((d_in, r), 0.01, 134) if r else None
+    R = si.gaussian_bf16((r, d_out), 0.01, 135) if r else None
+    layer = GpuLayer(W)
+    _, _, mask1 = oracle.prune24(W)
+    _, _, mask2 = oracle.double_prune(W, mask1)
+    Xd, dYd = dev(B, X), dev(B, dY)
+    if r:
+        Ld, Rd = dev(B, L), dev(B, R)
+        T = layer.adapter_T(Xd, Ld)
+        Y = layer.fwd(Xd, T, Rd)
+        dT, _, _ = layer.adapter_bwd(Xd, dYd, Ld, Rd, T)
+        dX = layer.dx(dYd, dT, Ld)
+    else:
+        Y = layer.fwd(Xd)
+        dX = layer.dx(dYd)
+    layer.poll()
+    rows = np.concatenate([np.arange(4), si.sample_indices(b, 40, 136), np.arange(b - 4, b)])
+    errs = {
+        "Y": rel_fro(to_f64(B.bits_from_bf16(Y))[rows], oracle.fwd_rows(X, W, mask1, rows, L, R)),
+        "dX": rel_fro(to_f64(B.bits_from_bf16(dX))[rows], oracle.dx_rows(dY, W, mask2, rows, L, R)),
+    }
     print(errs)
     for k, v in errs.items():
         assert v <= REL_TOL, (k, v, errs)
