@@ -370,3 +370,68 @@ def test_optional_masks_and_run_to_run_determinism(B, oracle):
     first, second = run(), run()
     for a, c in zip(first, second):
         assert np.array_equal(a, c)
+
+
+def _fuzz_shapes():
+    """Seeded shapes that hit every branch of the kernel choice: few-token tiles of all four widths with
+    one to eight K-splits, 256-row and 512-row sparse tiles, weight-gradient launches with and without
+    halved last-round tiles, one-CTA weight-gradient tiles, ranks from 16 to 256."""
+    rng = np.random.Generator(np.random.PCG64(20260824))
+    shapes = []
+    for _ in range(20):
+        d_in = 128 * int(rng.integers(1, 25))
+        d_out = 128 * int(rng.integers(1, 25))
+        b = 8 * int(rng.choice([1, 2, 5, 8, 13, 16, 27, 32, 33, 70, 129, 300]))
+        r = int(rng.choice([0, 16, 48, 64, 112, 128, 256]))
+        shapes.append((d_in, d_out, b, r))
+    shapes += [(2560, 5120, 2048, 0),      # dW: 10 x 20 = 200 tiles -> 2 rounds + 52 tiles (no halving: more than half the pairs)
+               (2304, 2560, 1000, 16),     # dW: 90 tiles -> 1 round + 16 tiles, halved
+               (4096, 1280, 3080, 64)]     # 512-row sparse tiles with a partial last row tile (1280 = 2.5 tiles)
+    return shapes
+
+
+@pytest.mark.parametrize("d_in,d_out,b,r", _fuzz_shapes())
+def test_seeded_shape_sweep_on_sampled_outputs(B, oracle, d_in, d_out, b, r):
+    seed = 7000 + d_in // 128 * 31 + d_out // 128 * 7 + b + r
+    W = si.gaussian_bf16((d_out, d_in), 0.02, seed)
+    X = si.gaussian_bf16((b, d_in), 1.0, seed + 1)
+    dY = si.gaussian_bf16((b, d_out), 1.0, seed + 2)
+    L = si.gaussian_bf16((d_in, r), 0.01, seed + 3) if r else None
+    R = si.gaussian_bf16((r, d_out), 0.01, seed + 4) if r else None
+    layer = GpuLayer(W)
+    _, _, mask1 = oracle.prune24(W)
+    _, _, mask2 = oracle.double_prune(W, mask1)
+    assert np.array_equal(layer.mask1.cpu().numpy(), mask1) and np.array_equal(layer.mask2.cpu().numpy(), mask2)
+    Xd, dYd = dev(B, X), dev(B, dY)
+    if r:
+        Ld, Rd = dev(B, L), dev(B, R)
+        T = layer.adapter_T(Xd, Ld)
+        Y = layer.fwd(Xd, T, Rd)
+        dT, dL, dR = layer.adapter_bwd(Xd, dYd, Ld, Rd, T)
+        dX = layer.dx(dYd, dT, Ld)
+    else:
+        Y = layer.fwd(Xd)
+        dX = layer.dx(dYd)
+    dWc = layer.dw(dYd, Xd)
+    layer.poll()
+    rows = np.unique(np.concatenate([np.arange(min(b, 3)), si.sample_indices(b, min(b, 24), seed + 5), np.arange(b - min(b, 3), b)]))
+    orows = np.unique(np.concatenate([np.arange(2), si.sample_indices(d_out, min(d_out, 24), seed + 6), np.arange(d_out - 2, d_out)]))
+    g = lambda t: to_f64(B.bits_from_bf16(t))
+    errs = {
+        "Y": rel_fro(g(Y)[rows], oracle.fwd_rows(X, W, mask1, rows, L, R)),
+        "dX": rel_fro(g(dX)[rows], oracle.dx_rows(dY, W, mask2, rows, L, R)),
+        "dWc": rel_fro(g(dWc)[orows], oracle.dw_rows(dY, X, mask1, orows)),
+    }
+    if r:
+        jrows = np.unique(np.concatenate([np.arange(2), si.sample_indices(d_in, min(d_in, 16), seed + 7)]))
+        icols = np.unique(np.concatenate([np.arange(2), si.sample_indices(d_out, min(d_out, 32), seed + 8)]))
+        errs["T"] = rel_fro(g(T)[rows], oracle.adapter_T_rows(X, L, rows))
+        errs["dT"] = rel_fro(g(dT)[rows], oracle.adapter_dT_rows(dY, R, rows))
+        errs["dL"] = rel_fro(g(dL)[jrows], oracle.adapter_dL_rows(X, dY, R, jrows))
+        errs["dR"] = rel_fro(g(dR)[:, icols], oracle.adapter_dR_cols(X, L, dY, icols))
+    for k, v in errs.items():
+        assert v <= REL_TOL, (k, v, errs)
+    import torch
+
+    for t in (Y, dX, dWc):
+        assert bool(torch.isfinite(t.float()).all())
