@@ -288,19 +288,45 @@ struct SplitKReduce {
     int M, N, splits, transpose;
 };
 
+// A block takes 32 consecutive rows at a time: 16-byte loads of the partial sums, summed in split
+// order; the transposed output goes through a padded shared-memory tile so that both the reads
+// and the 2-byte writes are contiguous.  N (the adapter rank) is a multiple of 16, at most 256.
 __global__ void __launch_bounds__(256) splitk_reduce_kernel(const SplitKReduce r0, const SplitKReduce r1) {
-    const size_t total0 = static_cast<size_t>(r0.M) * r0.N;
-    const size_t total1 = static_cast<size_t>(r1.M) * r1.N;
-    for (size_t gidx = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; gidx < total0 + total1;
-         gidx += static_cast<size_t>(gridDim.x) * blockDim.x) {
-        const bool second = gidx >= total0;
+    __shared__ float tile[32][257];
+    const int units0 = (r0.M + 31) / 32, units1 = (r1.M + 31) / 32;
+    for (int u = blockIdx.x; u < units0 + units1; u += gridDim.x) {
+        const bool second = u >= units0;
         const SplitKReduce& r = second ? r1 : r0;
-        const size_t idx = second ? gidx - total0 : gidx;
-        const size_t total = second ? total1 : total0;
-        float acc = 0.0f;
-        for (int s = 0; s < r.splits; ++s) acc += r.ws[static_cast<size_t>(s) * total + idx];
-        const size_t m = idx / r.N, n = idx % r.N;
-        r.out[r.transpose ? n * static_cast<size_t>(r.M) + m : idx] = to_bf16(acc);
+        const int m0 = 32 * (second ? u - units0 : u);
+        const int rows = min(32, r.M - m0);
+        const size_t total = static_cast<size_t>(r.M) * r.N;
+        const float4* ws4 = reinterpret_cast<const float4*>(r.ws + static_cast<size_t>(m0) * r.N);
+        const size_t split_stride4 = total / 4;
+        const int chunks = rows * r.N / 4;
+        for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
+            float4 acc = ws4[c];
+            for (int s = 1; s < r.splits; ++s) {
+                const float4 t = ws4[static_cast<size_t>(s) * split_stride4 + c];
+                acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+            }
+            if (r.transpose) {
+                const int mm = (4 * c) / r.N, n = (4 * c) % r.N;
+                tile[mm][n] = acc.x; tile[mm][n + 1] = acc.y; tile[mm][n + 2] = acc.z; tile[mm][n + 3] = acc.w;
+            } else {
+                uint2 o;
+                o.x = pack_bf16x2(acc.x, acc.y);
+                o.y = pack_bf16x2(acc.z, acc.w);
+                *reinterpret_cast<uint2*>(r.out + static_cast<size_t>(m0) * r.N + 4 * static_cast<size_t>(c)) = o;
+            }
+        }
+        if (r.transpose) {
+            __syncthreads();
+            for (int e = threadIdx.x; e < 32 * r.N; e += blockDim.x) {
+                const int n = e >> 5, mm = e & 31;
+                if (mm < rows) r.out[static_cast<size_t>(n) * r.M + m0 + mm] = to_bf16(tile[mm][n]);
+            }
+            __syncthreads();
+        }
     }
 }
 
