@@ -147,6 +147,16 @@ def double_prune_nm(W: np.ndarray, mask1: np.ndarray, n: int, m: int):
     return WRC, mask2
 
 
+def mask_difference(mask_a: np.ndarray, mask_b: np.ndarray) -> int:
+    """O11: number of element positions in which two bit masks [rows, cols/8] differ."""
+    mask_a, mask_b = _u8(mask_a), _u8(mask_b)
+    assert mask_a.shape == mask_b.shape
+    rows, mrow = mask_a.shape
+    fn = _load().slope_oracle_mask_difference
+    fn.restype = ctypes.c_longlong
+    return int(fn(_p(mask_a), _p(mask_b), rows, mrow * 8))
+
+
 def mask_to_bool(mask: np.ndarray, cols: int) -> np.ndarray:
     """Bit mask (LSB-first bytes) -> boolean [rows, cols]."""
     return np.unpackbits(np.asarray(mask, np.uint8), axis=1, bitorder="little")[:, :cols].astype(bool)

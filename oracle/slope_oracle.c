@@ -444,6 +444,19 @@ void slope_oracle_double_prune_nm(const uint16_t *W, const uint8_t *mask1, int d
         }
 }
 
+/* O11 -- mask difference (supplementary "Comparison with Dynamic Sparsity: SR-STE":
+ * the number of mask elements in which the mask of an iteration differs from the
+ * converged one): count of element positions whose mask bits differ. */
+long long slope_oracle_mask_difference(const uint8_t *mask_a, const uint8_t *mask_b, int rows, int cols)
+{
+    long long diff = 0;
+    long mrow = cols / 8;
+    for (long i = 0; i < rows; ++i)
+        for (long j = 0; j < cols; ++j)
+            diff += mask_get(mask_a, mrow, i, j) != mask_get(mask_b, mrow, i, j);
+    return diff;
+}
+
 int slope_oracle_max_threads(void)
 {
 #ifdef _OPENMP

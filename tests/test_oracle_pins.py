@@ -431,3 +431,22 @@ def test_p9_nm_structure_and_lemma1(oracle, n, m):
     hist = np.bincount(k1.T.reshape(d, d // m, m).sum(-1).ravel(), minlength=m + 1) / (d * d // m)
     binom = np.array([math.comb(m, j) * (n / m) ** j * (1 - n / m) ** (m - j) for j in range(m + 1)])
     assert np.allclose(hist, binom, atol=4e-3)
+
+
+# ----------------------------------------------------------------------------- P10: mask difference (O11)
+def test_p10_mask_difference(oracle):
+    rng = np.random.Generator(np.random.PCG64(1001))
+    a = rng.integers(0, 256, size=(24, 40), dtype=np.uint8)
+    b = rng.integers(0, 256, size=(24, 40), dtype=np.uint8)
+    want = int((np.unpackbits(a, axis=1, bitorder="little") != np.unpackbits(b, axis=1, bitorder="little")).sum())
+    assert oracle.mask_difference(a, b) == want
+    assert oracle.mask_difference(a, a) == 0
+    assert oracle.mask_difference(a, ~a) == 24 * 320
+    # a worked case: the 2:4 masks of two matrices that differ in one group only, (1,2 kept) -> (0,3 kept):
+    # all four positions of that group change
+    W = si.f32_to_bf16_bits(np.tile(np.array([0.1, 2.0, 3.0, 0.2], np.float32), (4, 8)))
+    V = W.copy()
+    V[2, 4:8] = si.f32_to_bf16_bits(np.array([5.0, 0.2, 0.1, 4.0], np.float32))
+    _, _, m1 = oracle.prune24(W)
+    _, _, m2 = oracle.prune24(V)
+    assert oracle.mask_difference(m1, m2) == 4
