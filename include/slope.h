@@ -184,6 +184,16 @@ slope_status_t slope_apply_mask(const void* G, const void* mask_bits, int d_out,
                                 void* out, void* stream);
 
 /*
+ * Mask difference (supplementary "Comparison with Dynamic Sparsity: SR-STE": how many mask
+ * elements an iteration's mask differs in from the converged one): writes to the device
+ * uint64 *count_out (8-byte aligned) the number of element positions whose bits differ in
+ * the two masks [rows x cols/8].  With slope_prune_nm on the dense weight every step this
+ * measures how much a dynamically re-selected mask still moves.
+ */
+slope_status_t slope_mask_difference(const void* mask_a, const void* mask_b, int rows, int cols,
+                                     void* count_out, void* stream);
+
+/*
  * The dense bf16 layer on the same tcgen05 pipeline (CTA-pair 256 x 256 tiles, no sparsity):
  *   slope_dense_linear_fwd      Y [b x d_out]    = X  W^T
  *   slope_dense_linear_bwd_dx   dX[b x d_in]     = dY W

@@ -30,7 +30,7 @@ EXPORTS = (
     "slope_adapter_dl_noalloc", "slope_adapter_dl_noalloc_max_scratch_bytes",
     "slope_sparse_add", "slope_update_sparse_matrix", "slope_selftest_wait_timeout",
     "slope_prune_nm", "slope_double_prune_nm", "slope_apply_mask",
-    "slope_dense_linear_fwd", "slope_dense_linear_bwd_dx", "slope_dense_linear_bwd_dw",
+    "slope_dense_linear_fwd", "slope_dense_linear_bwd_dx", "slope_dense_linear_bwd_dw", "slope_mask_difference",
 )
 
 
@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.slope_dense_linear_bwd_dw.argtypes = [vp, vp, ci, ci, ci, vp, vp]
         for name in ("slope_dense_linear_fwd", "slope_dense_linear_bwd_dx", "slope_dense_linear_bwd_dw"):
             getattr(L, name).restype = ci
+        L.slope_mask_difference.argtypes = [vp, vp, ci, ci, vp, vp]
+        L.slope_mask_difference.restype = ci
         L.slope_prune_nm.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp]
         L.slope_prune_nm.restype = ci
         L.slope_double_prune_nm.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, vp]
@@ -206,6 +208,12 @@ def slope_dense_linear_bwd_dw(dY, X, dW):
     (b, d_out), d_in = dY.shape, X.shape[1]
     _check("slope_dense_linear_bwd_dw", lib().slope_dense_linear_bwd_dw(_ptr(dY), _ptr(X), b, d_out, d_in, _ptr(dW),
                                                                         _stream()))
+
+
+def slope_mask_difference(mask_a, mask_b, count_out):
+    rows, mrow = mask_a.shape
+    _check("slope_mask_difference", lib().slope_mask_difference(_ptr(mask_a), _ptr(mask_b), rows, mrow * 8,
+                                                                _ptr(count_out), _stream()))
 
 
 def slope_prune_nm(W, n, m, W_R, mask1_bits=None):

@@ -170,4 +170,21 @@ apply_mask_kernel(const uint4* G, const uint16_t* __restrict__ mask, size_t n_ch
     }
 }
 
+// Number of element positions in which two bit masks differ (the per-iteration mask change
+// that the comparison with dynamically re-selected masks plots).  16-byte loads, popcount of the
+// XOR, one integer atomic per warp: the count is exact whatever the order.
+__global__ void __launch_bounds__(256)
+mask_difference_kernel(const uint4* __restrict__ a, const uint4* __restrict__ b, size_t n_vec,
+                       unsigned long long* __restrict__ count) {
+    unsigned int local = 0;
+    const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+    for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_vec; i += stride) {
+        const uint4 x = __ldcs(a + i), y = __ldcs(b + i);
+        local += __popc(x.x ^ y.x) + __popc(x.y ^ y.y) + __popc(x.z ^ y.z) + __popc(x.w ^ y.w);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) local += __shfl_xor_sync(0xFFFFFFFFu, local, o);
+    if ((threadIdx.x & 31) == 0 && local != 0) atomicAdd(count, static_cast<unsigned long long>(local));
+}
+
 }  // namespace slope

@@ -774,6 +774,23 @@ slope_status_t slope_apply_mask(const void* G, const void* mask_bits, int d_out,
     return launch_result();
 }
 
+slope_status_t slope_mask_difference(const void* mask_a, const void* mask_b, int rows, int cols, void* count_out,
+                                     void* stream_) {
+    if (!mask_a || !mask_b || !count_out) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(rows, cols)) return SLOPE_ERR_SHAPE;
+    if (!aligned16(mask_a) || !aligned16(mask_b) || (reinterpret_cast<uintptr_t>(count_out) & 7u) != 0)
+        return SLOPE_ERR_ALIGNMENT;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (cudaMemsetAsync(count_out, 0, sizeof(unsigned long long), stream) != cudaSuccess) return SLOPE_ERR_CUDA;
+    const size_t n_vec = static_cast<size_t>(rows) * cols / 8 / 16;
+    mask_difference_kernel<<<info.sm_count * kStreamBlocksPerSm, 256, 0, stream>>>(
+        static_cast<const uint4*>(mask_a), static_cast<const uint4*>(mask_b), n_vec,
+        static_cast<unsigned long long*>(count_out));
+    return launch_result();
+}
+
 slope_status_t slope_selftest_wait_timeout(unsigned int limit_us, void* gave_up_flag, void* stream) {
     if (!gave_up_flag || limit_us == 0 || limit_us > 100000) return SLOPE_ERR_INVALID_ARG;
     DeviceInfo info;

@@ -203,3 +203,29 @@ def test_emulated_2_8_layer_matches_oracle_on_the_masks(B, oracle):
         assert v <= REL_TOL, (k, v, errs)
     got = B.bits_from_bf16(dW)
     assert not np.any(got[~keep1] & 0x7FFF)                   # exact zeros outside the mask
+
+
+def test_mask_difference_of_re_selected_masks(B, oracle):
+    """A dense weight drifts for a few "steps"; its 2:4 mask is re-selected every step (the dynamic-mask
+    variant) and compared with the last one: the GPU count equals the oracle's on the oracle's masks."""
+    import torch
+
+    d_out, d_in = 512, 1024
+    W0 = si.gaussian_bf16((d_out, d_in), 0.02, 601)
+    masks_o, masks_g = [], []
+    count = torch.zeros(1, dtype=torch.int64, device="cuda")
+    for step in range(4):
+        drift = si.gaussian_bf16((d_out, d_in), 0.004 * step, 610 + step)
+        W = si.f32_to_bf16_bits((W0.astype(np.uint32) << 16).view(np.float32) + (drift.astype(np.uint32) << 16).view(np.float32))
+        _, m_o = oracle.prune_nm(W, 2, 4)
+        Wd = B.bf16_from_bits(W)
+        m_g = torch.empty((d_out, d_in // 8), dtype=torch.uint8, device="cuda")
+        B.slope_prune_nm(Wd, 2, 4, Wd, m_g)
+        assert np.array_equal(m_g.cpu().numpy(), m_o)
+        masks_o.append(m_o)
+        masks_g.append(m_g)
+    for step in range(4):
+        B.slope_mask_difference(masks_g[step], masks_g[-1], count)
+        assert B.slope_poll_status() == 0
+        assert int(count.item()) == oracle.mask_difference(masks_o[step], masks_o[-1])
+    assert oracle.mask_difference(masks_o[0], masks_o[-1]) > 0
