@@ -450,6 +450,7 @@ def main():
         out["burst"] = burst_probe(torch, B, layers, stream, pk)
         out["inference_forward"] = inference_forward_probe(torch, B, wl, pk)
         out["nm_masked_dense"] = nm_probe(torch, B, layers, stream, pk)
+        out["forward_speedup_by_shape"] = forward_shape_sweep(torch, B, stream)
         out["small_configs_hot_cold"] = small_config_probe(torch, B, stream, pk)
         out["dense_layer"] = dense_comparison(torch, B, layers, stream)
         if args.cusparselt_context:
@@ -496,6 +497,43 @@ def optimizer_tail_probe(torch, B, layers, stream, pk, reps=20):
     return {"what": f"{reps} back-to-back launches, CUDA events; bytes: sparse_add 3 B and update 2.25 B per weight "
                     f"element; HBM peak {pk['hbm_gbs']} GB/s ({pk['src']}); the working set of sparse_add "
                     f"({3 * n / 1e6:.0f} MB) partly lives in the 126 MB L2 across launches", "rows": rows}
+
+
+def forward_shape_sweep(torch, B, stream, tokens=2048, reps=20):
+    """The setting of the paper's per-shape speedup figure (attention d -> d, upsample d -> 4d and
+    downsample 4d -> d matrices, batch 2048): forward GEMM, slope_linear_fwd against torch.matmul on
+    the dense weight, back-to-back launches timed with CUDA events, interleaved."""
+    dev = torch.device("cuda")
+    rows = []
+    for d in (1024, 2048, 4096, 8192):
+        for kind, d_in, d_out in (("attention", d, d), ("upsample", d, 4 * d), ("downsample", 4 * d, d)):
+            W = B.bf16_from_bits(si.gaussian_bf16((d_out, d_in), 0.02, si.seed_for(8, 0, "W")), dev)
+            X = B.bf16_from_bits(si.gaussian_bf16((tokens, d_in), 1.0, si.seed_for(8, 0, "X")), dev)
+            vals, meta, _ = B.alloc_compressed(d_out, d_in, dev)
+            B.slope_prune_24(W, vals, meta, None)
+            Y = torch.empty((tokens, d_out), dtype=torch.bfloat16, device=dev)
+
+            def timed(fn):
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for _ in range(reps):
+                    fn()
+                e1.record(stream)
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1) / reps * 1e3
+
+            us_dense = timed(lambda: torch.matmul(X, W.t(), out=Y))
+            us_sparse = timed(lambda: B.slope_linear_fwd(X, vals, meta, d_out, Y))
+            flop = 2.0 * tokens * d_in * d_out
+            rows.append({"kind": kind, "d_in": d_in, "d_out": d_out, "tokens": tokens, "dense_us": round(us_dense, 1),
+                         "slope_us": round(us_sparse, 1), "speedup": round(us_dense / us_sparse, 3),
+                         "slope_tflops_dense_eq": round(flop / us_sparse / 1e6, 1)})
+            del W, X, vals, meta, Y
+    return {"what": f"forward only, {tokens} tokens, {reps} back-to-back launches each (includes host launch overhead "
+                    f"for the smallest shapes), torch.matmul (cuBLAS) dense against slope_linear_fwd", "rows": rows}
 
 
 def small_config_probe(torch, B, stream, pk, min_launches=48):

@@ -227,13 +227,16 @@ static slope_status_t launch_dense(const void* A, const void* B, int M, int N, i
 }
 
 // ------------------------------------------------------------------ CTA-pair launches (main GEMMs)
-constexpr int kPairBlockN = 224;
+constexpr int kPairBlockN = 224;             // token tile of the big-tile kernels
 constexpr int kPairStages = 4;
+constexpr int kPairNarrowBlockN = 128;       // narrower 256-row tile for shapes with few tiles
+constexpr int kPairNarrowStages = 5;
 
+template <int BLOCK_N, int STAGES>
 static slope_status_t launch_sparse_pair(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                          const void* act2, const void* fac2, int r, bool a2_mn, void* out,
                                          cudaStream_t stream, const DeviceInfo& info) {
-    using Cfg = SparsePairCfg<kPairBlockN, kPairStages>;
+    using Cfg = SparsePairCfg<BLOCK_N, STAGES>;
     CUtensorMap tmA, tmB, tmE, tmA2, tmB2, tmO;
     if (!make_tmap(&tmA, vals, M, K / 2, kBlockM, 64)) return SLOPE_ERR_CUDA;
     if (!make_tmap(&tmB, act, ntok, K, Cfg::kHalfN, 64)) return SLOPE_ERR_CUDA;
@@ -250,9 +253,9 @@ static slope_status_t launch_sparse_pair(const void* act, int ntok, const void* 
     p.M = M; p.K = K; p.Ntok = ntok; p.r = r; p.a2_mn_major = a2_mn ? 1 : 0;
     p.meta = static_cast<const uint8_t*>(meta);
     p.out = static_cast<uint16_t*>(out);
-    auto kern = sparse_gemm_pair_kernel<kPairBlockN, kPairStages>;
+    auto kern = sparse_gemm_pair_kernel<BLOCK_N, STAGES>;
     if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
-    const int tiles = ((M / kBlockM + 1) / 2) * ((ntok + kPairBlockN - 1) / kPairBlockN);
+    const int tiles = ((M / kBlockM + 1) / 2) * ((ntok + BLOCK_N - 1) / BLOCK_N);
     const int max_pairs = info.sm_count / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
     return launch_pairs(kern, 2 * pairs, Cfg::kThreads, Cfg::kSmemBytes, stream, tmA, tmB, tmE, tmA2, tmB2, tmO, p);
@@ -412,20 +415,34 @@ static slope_status_t launch_skinny(const void* act, int ntok, const void* vals,
 }
 
 // Kernel choice for the sparse GEMMs.  Up to 256 tokens the GEMM is a weight stream from HBM and
-// runs on the few-token kernel.  Beyond that: the 512-row tile moves 31 % fewer L2 bytes per FLOP
-// but cannot overlap its epilogue with the next tile (tensor memory holds only one accumulator
-// set).  Measured at 16384 tokens it is 6 % faster per unit of work at a reduction length of
-// 4096 and 14-16 % at 11008, while at 768 the 256-row tile with its double-buffered accumulators
-// is up to 25 % faster.  The choice compares rounds of the machine (tiles / CTA pairs, rounded
-// up) times the relative cost of a tile, so that a shape whose 512-row tiles fill the last
-// round badly (4096 x 4096 with 4096 tokens: 152 tiles on 74 pairs) keeps the 256-row tile.
-static bool prefer_quad_tile(int M, int K, int ntok, int num_pairs) {
-    const int num_n = (ntok + kPairBlockN - 1) / kPairBlockN;
-    const int tiles_pair = ((M + 255) / 256) * num_n, tiles_quad = ((M + 511) / 512) * num_n;
+// runs on the few-token kernel.  Beyond that three tile shapes compete:
+//   512 x 224  moves 31 % fewer L2 bytes per FLOP but cannot overlap its epilogue with the next
+//              tile (tensor memory holds one accumulator set).  Measured at 16384 tokens it is
+//              6 % faster per unit of work at a reduction length of 4096 and 14-16 % at 11008,
+//              while at 768 the 256-row tile is up to 25 % faster.
+//   256 x 224  double-buffered accumulators.
+//   256 x 128  the same kernel with a narrower token tile: more, smaller tiles for shapes that
+//              would otherwise leave much of the last round of the machine empty (2048 x 2048
+//              with 2048 tokens: 80 tiles of 256 x 224 on 74 CTA pairs = 2 rounds for 1.08 rounds
+//              of work); it stages the weights for fewer tokens, which costs 12 % more time
+//              per unit of work at short reductions and 30-35 % at long ones (measured at 2048
+//              tokens).
+// The choice compares rounds of the machine (tiles / CTA pairs, rounded up) times the relative
+// cost of a tile.
+enum class SparseTile { kQuad224, kPair224, kPair128 };
+
+static SparseTile choose_sparse_tile(int M, int K, int ntok, int num_pairs) {
+    const auto rounds = [&](int rows, int block_n) {
+        const int tiles = ((M + rows - 1) / rows) * ((ntok + block_n - 1) / block_n);
+        return static_cast<double>((tiles + num_pairs - 1) / num_pairs);
+    };
     const double gain = K >= 8192 ? 0.14 : K >= 4096 ? 0.06 : K >= 2048 ? -0.05 : -0.25;
-    const double cost_pair = (tiles_pair + num_pairs - 1) / num_pairs;
-    const double cost_quad = 2.0 * (1.0 - gain) * ((tiles_quad + num_pairs - 1) / num_pairs);
-    return cost_quad < cost_pair;
+    const double cost_pair = rounds(256, kPairBlockN);
+    const double cost_quad = 2.0 * (1.0 - gain) * rounds(512, kPairBlockN);
+    const double narrow_penalty = K >= 8192 ? 1.35 : K >= 4096 ? 1.30 : K >= 2048 ? 1.20 : 1.12;
+    const double cost_narrow = narrow_penalty * kPairNarrowBlockN / kPairBlockN * rounds(256, kPairNarrowBlockN);
+    if (cost_quad < cost_pair && cost_quad <= cost_narrow) return SparseTile::kQuad224;
+    return cost_narrow < cost_pair ? SparseTile::kPair128 : SparseTile::kPair224;
 }
 
 static slope_status_t launch_sparse_gemm(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
@@ -433,9 +450,16 @@ static slope_status_t launch_sparse_gemm(const void* act, int ntok, const void* 
                                          cudaStream_t stream, const DeviceInfo& info) {
     if (ntok <= kSkinnyMaxTokens)
         return launch_skinny(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
-    return prefer_quad_tile(M, K, ntok, info.sm_count / 2)
-               ? launch_sparse_quad(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info)
-               : launch_sparse_pair(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
+    switch (choose_sparse_tile(M, K, ntok, info.sm_count / 2)) {
+        case SparseTile::kQuad224:
+            return launch_sparse_quad(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
+        case SparseTile::kPair128:
+            return launch_sparse_pair<kPairNarrowBlockN, kPairNarrowStages>(act, ntok, vals, meta, M, K, act2, fac2, r,
+                                                                            a2_mn, out, stream, info);
+        default:
+            return launch_sparse_pair<kPairBlockN, kPairStages>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out,
+                                                                stream, info);
+    }
 }
 
 template <bool A_MN, bool B_MN, int BLOCK_N, int EPI, int STAGES>
