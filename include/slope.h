@@ -88,8 +88,9 @@ slope_status_t slope_double_prune(const void* W, const void* mask1_bits, int d_o
  * Eq. (concat):  Y[b x d_out] = X[b x d_in] (W^R)^T  (+ T[b x r] R[r x d_out]).
  * Wc_vals / Wc_meta come from slope_prune_24.  T = X L is produced by
  * slope_adapter_fwd_bwd(phase 0).  r = 0 (T, R ignored) leaves the adapter out.
- * With b <= 256 (inference, decode: the paper's forward-only inference measurements) the
- * same call runs on a kernel that streams the compressed weight once from HBM and splits the
+ * With few tokens (inference, decode: the paper's forward-only inference measurements; always up
+ * to 16 tokens, up to 128 where it is estimated faster than the tile kernels) the same call
+ * runs on a kernel that streams the compressed weight once from HBM and splits the
  * reduction over a thread-block cluster; that launch is issued with programmatic stream
  * serialisation and synchronises on the device before it touches memory, so stream order
  * holds as for any other call.  Every compute call of this library can be captured in a CUDA

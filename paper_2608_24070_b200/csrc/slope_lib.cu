@@ -327,25 +327,50 @@ static slope_status_t launch_sparse_quad(const void* act, int ntok, const void* 
 constexpr double kSkinnySmUs = 0.23, kSkinnyHbmUs = 0.0028, kSkinnyWaveUs = 4.0, kSkinnyReduceUs = 0.5,
                  kSkinnyReducePerRankUs = 0.07;
 
-template <typename Capacity>
-static int skinny_splits(int slabs, int num_kb, Capacity capacity) {
+// A k-block costs an SM its weight tile (kSkinnySmUs) plus the activation tile's TMA row
+// requests (2 per token of the tile, ~2 ns each).
+constexpr double kSkinnyTokenUs = 0.004;
+
+static int skinny_splits(int slabs, int num_kb, int block_n, const int (&cap)[9], double* est_us = nullptr) {
     int best_s = 1;
     double best_cost = 1e30;
+    const double sm_us = kSkinnySmUs + kSkinnyTokenUs * block_n;
     for (int s = 1; s <= 8; ++s) {
         const int per = (num_kb + s - 1) / s;
         if ((num_kb + per - 1) / per != s) continue;                 // a rank would be left without a k-block
         if (s > 1 && per < 2) break;
-        const int cap = capacity(s);
-        if (cap <= 0) continue;
+        if (cap[s] <= 0) continue;
         double cost = s > 1 ? kSkinnyReduceUs + kSkinnyReducePerRankUs * s : 0.0;
-        for (int left = slabs; left > 0; left -= cap) {
-            const int active = (left < cap ? left : cap) * s;
-            const double per_kb = active * kSkinnyHbmUs > kSkinnySmUs ? active * kSkinnyHbmUs : kSkinnySmUs;
+        for (int left = slabs; left > 0; left -= cap[s]) {
+            const int active = (left < cap[s] ? left : cap[s]) * s;
+            const double per_kb = active * kSkinnyHbmUs > sm_us ? active * kSkinnyHbmUs : sm_us;
             cost += kSkinnyWaveUs + per * per_kb;
         }
         if (cost < best_cost - 1e-9) { best_cost = cost; best_s = s; }
     }
+    if (est_us) *est_us = best_cost;
     return best_s;
+}
+
+// Co-resident clusters of the few-token kernel per cluster size, asked of the driver once per
+// device and kernel variant.
+template <int BLOCK_N, int A_STAGES, int B_STAGES>
+static bool skinny_capacity(const DeviceInfo& info, int (&cap)[9]) {
+    using Cfg = SparseSkinnyCfg<BLOCK_N, A_STAGES, B_STAGES>;
+    static std::mutex mu;
+    static int capacity[64][9];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    auto kern = sparse_gemm_skinny_kernel<BLOCK_N, A_STAGES, B_STAGES>;
+    std::lock_guard<std::mutex> lock(mu);
+    if (capacity[dev][1] == 0) {
+        if (!set_smem(kern, Cfg::kSmemBytes)) return false;
+        for (int s = 1; s <= 8; ++s)
+            capacity[dev][s] = max_active_clusters(kern, s, kGemmThreads, Cfg::kSmemBytes, info.sm_count);
+    }
+    cap[0] = 0;
+    for (int s = 1; s <= 8; ++s) cap[s] = capacity[dev][s];
+    return cap[1] > 0;
 }
 
 template <int BLOCK_N, int A_STAGES, int B_STAGES>
@@ -379,22 +404,10 @@ static slope_status_t launch_sparse_skinny(const void* act, int ntok, const void
     auto kern = sparse_gemm_skinny_kernel<BLOCK_N, A_STAGES, B_STAGES>;
     if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
 
-    // co-resident clusters per cluster size, asked of the driver once per device
-    static std::mutex mu;
-    static int capacity[64][9];
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SLOPE_ERR_CUDA;
     int cap[9];
-    {
-        std::lock_guard<std::mutex> lock(mu);
-        if (capacity[dev][1] == 0)
-            for (int s = 1; s <= 8; ++s)
-                capacity[dev][s] = max_active_clusters(kern, s, kGemmThreads, Cfg::kSmemBytes, info.sm_count);
-        for (int s = 1; s <= 8; ++s) cap[s] = capacity[dev][s];
-    }
-    if (cap[1] <= 0) return SLOPE_ERR_CUDA;
+    if (!skinny_capacity<BLOCK_N, A_STAGES, B_STAGES>(info, cap)) return SLOPE_ERR_CUDA;
     const int slabs = (M + kBlockM - 1) / kBlockM, num_kb = K > 0 ? K / 128 : (r + 63) / 64;
-    const int splits = skinny_splits(slabs, num_kb, [&](int s) { return cap[s]; });
+    const int splits = skinny_splits(slabs, num_kb, BLOCK_N, cap);
     return launch_cluster_ex(kern, slabs * splits, splits, kGemmThreads, Cfg::kSmemBytes, true, stream, tmA, tmB,
                              tmE, tmA2, tmB2, p);
 }
@@ -445,10 +458,32 @@ static SparseTile choose_sparse_tile(int M, int K, int ntok, int num_pairs) {
     return cost_narrow < cost_pair ? SparseTile::kPair128 : SparseTile::kPair224;
 }
 
+// Few-token kernel or tile kernel?  Decode sizes (<= 16 tokens) always stream the weights through
+// the few-token kernel.  Up to 128 tokens the two are compared by estimate: the few-token kernel's
+// own cost model against a tile kernel that has one token tile, i.e. M / 256 tiles which each
+// walk the whole reduction (measured: ~4 us per launch plus 0.32 us per k-block and round of the
+// machine).  A tall weight (4096 -> 11008) then has enough tiles for the tile kernel, a long
+// reduction on few rows (11008 -> 4096) wants the K-split of the few-token kernel.  Beyond 128
+// tokens the 256-token variant of the few-token kernel pays 512 row requests per k-block for
+// its activations and loses almost everywhere (measured), so the tile kernels take over.
+static bool use_few_token_kernel(int M, int K, int ntok, int r, const DeviceInfo& info) {
+    if (ntok <= 16) return true;
+    if (ntok > 128) return false;
+    int cap[9];
+    const bool ok = ntok <= 64 ? skinny_capacity<64, 8, 4>(info, cap) : skinny_capacity<128, 7, 3>(info, cap);
+    if (!ok) return false;
+    double few_us = 0.0;
+    skinny_splits(M / kBlockM, K / 128, ntok <= 64 ? 64 : 128, cap, &few_us);
+    const int num_pairs = info.sm_count / 2;
+    const int tiles = (M + 255) / 256;
+    const double tile_us = 4.0 + ((tiles + num_pairs - 1) / num_pairs) * (K / 128 + (r + 63) / 64) * 0.32;
+    return few_us <= tile_us;
+}
+
 static slope_status_t launch_sparse_gemm(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                          const void* act2, const void* fac2, int r, bool a2_mn, void* out,
                                          cudaStream_t stream, const DeviceInfo& info) {
-    if (ntok <= kSkinnyMaxTokens)
+    if (use_few_token_kernel(M, K, ntok, r, info))
         return launch_skinny(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
     switch (choose_sparse_tile(M, K, ntok, info.sm_count / 2)) {
         case SparseTile::kQuad224:

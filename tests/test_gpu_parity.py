@@ -107,13 +107,13 @@ CASES = [
     (128, 128, 8, 16, 15),           # smallest legal problem
     (6144, 640, 264, 32, 16),        # long forward reduction (48 k-blocks) on the 256-row tile
     (640, 6144, 264, 0, 17),         # same for the input-gradient GEMM
-    (4096, 512, 40, 16, 18),         # few tokens: weight-streaming kernel (64-token tile), K split over a cluster
-    (1024, 384, 200, 0, 19),         # 200 tokens (256-token tile)
+    (4096, 512, 40, 16, 18),         # few tokens, long reduction on few rows: few-token kernel (64-token tile), K split over a cluster
+    (1024, 384, 200, 0, 19),         # 200 tokens: tile kernels with one narrow token tile
     (2048, 256, 64, 64, 20),         # exactly one 64-token tile with adapters
-    (256, 2048, 128, 32, 21),        # 128-token tile; dX has the long reduction
+    (256, 2048, 128, 32, 21),        # 128 tokens: forward and dX choose between few-token and tile kernel by estimate
     (1024, 512, 8, 64, 22),          # decode size: 16-token tile with adapters
     (512, 1536, 16, 128, 23),        # 16 tokens, two adapter K-steps
-    (1152, 384, 104, 128, 24),       # 128-token tile, ragged, two adapter K-steps, odd number of k-blocks
+    (1152, 384, 104, 128, 24),       # 104 tokens, ragged, two adapter K-steps, odd number of k-blocks
     (512, 768, 264, 256, 25),        # largest rank (6.25 % of a 4096-wide layer): two adapter column tiles
     (1024, 512, 16, 256, 26),        # largest rank at decode size
 ]
