@@ -402,7 +402,7 @@ def main():
     sp_fl = tot["linear_fwd"][0] + tot["linear_bwd_dx"][0]
     sp_s = tot["linear_fwd"][1] + tot["linear_bwd_dx"][1]
     sp_tflops = sp_fl / sp_s / 1e12 if sp_s else 0.0
-    roofline_sparse = {"kernel": "sparse_gemm_quad_kernel<224,3> (slope_linear_fwd, slope_linear_bwd_dx; sparse_gemm_pair_kernel<224,4> below a reduction length of 4096)", "bound": "tensor",
+    roofline_sparse = {"kernel": "sparse_gemm_quad_kernel<224,3> (slope_linear_fwd, slope_linear_bwd_dx; shapes with short reductions or few tiles run on sparse_gemm_pair_kernel<224,4> / <128,5>)", "bound": "tensor",
                        "achieved": round(sp_tflops, 1), "peak": round(sparse_peak, 1),
                        "unit": "TFLOP/s", "frac": round(sp_tflops / sparse_peak, 4), "traffic": None,
                        "ms_per_step": round(sp_s * 1e3, 4),
