@@ -7,13 +7,16 @@
 // loops, tensor memory is released and the kernel returns.
 //
 //   dense_gemm_kernel          1 CTA per 128 x N tile; the skinny adapter GEMMs and small dW
-//   dense_gemm_pair_kernel     CTA pair per 256 x 256 tile (cta_group::2); dW
-//   sparse_gemm_pair_kernel    CTA pair per 256 x 224 tile, tcgen05.mma.sp; forward / dX
+//   dense_gemm_pair_kernel     CTA pair per 256 x 256 tile (cta_group::2), the last round's tiles
+//                              halved; dW (masked epilogue) and the dense layer (store epilogue)
+//   sparse_gemm_pair_kernel    CTA pair per 256 x 224 (or 256 x 128) tile, tcgen05.mma.sp;
+//                              forward / dX with short reductions or few tiles
 //   sparse_gemm_quad_kernel    CTA pair per 512 x 224 tile (two MMA sub-tiles per activation
 //                              tile); forward / dX with long reductions
 //   sparse_gemm_skinny_kernel  one CTA per 128-row weight slab and K-slice, cluster reduction
-//                              through distributed shared memory; forward / dX with at most
-//                              256 tokens (inference, decode), not persistent
+//                              through distributed shared memory; forward / dX with few
+//                              tokens (inference, decode) and the adapter products at such
+//                              sizes, not persistent
 #pragma once
 #include "ptx.cuh"
 
