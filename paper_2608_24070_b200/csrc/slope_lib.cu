@@ -640,12 +640,18 @@ slope_status_t slope_linear_bwd_dw_masked(const void* dY, const void* X, int b, 
     if (!aligned16(dY) || !aligned16(X) || !aligned16(mask1_bits) || !aligned16(dWc_vals)) return SLOPE_ERR_ALIGNMENT;
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
-    // Small weight matrices do not have enough 256 x 256 tiles for the 74 CTA pairs; they run on
-    // 128 x 128 tiles, one CTA each, which fill the machine at the price of more L2 traffic per FLOP.
+    // Small weight matrices do not have enough 256 x 256 tiles for the 74 CTA pairs.  They run on
+    // 256 x 128 tiles of CTA pairs (each CTA stages half of the X tile: GPT-2-small 33 -> 29.5 us) or,
+    // when even those are few, on 128 x 128 tiles of one CTA each.
     const int pair_tiles = ((d_out + 255) / 256) * ((d_in + 255) / 256);
-    if (pair_tiles * 2 <= info.sm_count)
+    if (pair_tiles * 2 <= info.sm_count) {
+        const int narrow_tiles = ((d_out + 255) / 256) * ((d_in + 127) / 128);
+        if (narrow_tiles >= 24)
+            return launch_dense_pair<true, true, 128, kEpiMasked, 8>(dY, X, d_out, d_in, b, dWc_vals, mask1_bits,
+                                                                     static_cast<cudaStream_t>(stream), info);
         return launch_dense<true, true, 128, kEpiMasked, 6>(dY, X, d_out, d_in, b, 1, dWc_vals, mask1_bits,
                                                             static_cast<cudaStream_t>(stream), info);
+    }
     return launch_dense_pair<true, true, 256, kEpiMasked, 6>(dY, X, d_out, d_in, b, dWc_vals, mask1_bits,
                                                              static_cast<cudaStream_t>(stream), info);
 }
