@@ -1172,6 +1172,8 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 // in two separate rings with their own producer threads: a deep one for the weights, a
 // shallow one for the activations.
 // =====================================================================================
+constexpr int kSkinnyPrefetchBlocks = 6;   // k-blocks whose first-byte latency is otherwise exposed (6 x 0.23 us)
+
 template <int BLOCK_N, int A_STAGES, int B_STAGES>
 struct SparseSkinnyCfg {
     static constexpr int kABytes = kBlockM * 128;                    // compressed values of one k-block
@@ -1242,8 +1244,21 @@ sparse_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     // Everything above overlaps the tail of the previous kernel in the stream when the launch
-    // allows it; nothing below may touch global memory before that kernel has finished.
+    // allows it; nothing below may touch global memory before that kernel has finished.  One
+    // thing is safe earlier: asking L2 to fetch this CTA's first weight tiles.  A prefetch moves no
+    // data into the SM, and L2 is the point of coherence, so a line the previous kernel is still
+    // writing stays correct; the first loads after the wait then come at L2 instead of HBM latency.
     griddep_launch_dependents();
+    if (warp == 0 && elect_one()) {
+        // (a short K-slice gains nothing: its few tiles are requested at once after the wait, and the
+        // prefetch requests would only sit in front of them in the TMA queue)
+        const int n_pf = num_sb >= 8 ? kSkinnyPrefetchBlocks : 0;
+        for (int i = 0; i < n_pf; ++i) {
+            tma_prefetch_l2_2d(&tmA, (kb0 + i) * 64, m_blk * kBlockM);
+            tma_prefetch_l2_2d(&tmE, 0, m_blk * num_kb + kb0 + i);
+        }
+    }
+    __syncwarp();
     griddep_wait();
 
     if (warp == 0) {
