@@ -435,3 +435,57 @@ def test_seeded_shape_sweep_on_sampled_outputs(B, oracle, d_in, d_out, b, r):
 
     for t in (Y, dX, dWc):
         assert bool(torch.isfinite(t.float()).all())
+
+
+def test_two_host_threads_on_two_streams(B, oracle):
+    """Two host threads drive two layers on their own CUDA streams at the same time (the library keeps
+    per-device caches behind mutexes and per-launch state only): both results match the oracle."""
+    import threading
+
+    import torch
+
+    specs = [(1024, 512, 264, 32, 151), (512, 768, 16, 64, 161)]
+    results, errors = {}, []
+
+    def work(idx, d_in, d_out, b, r, seed):
+        try:
+            torch.cuda.set_device(0)
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                W = si.gaussian_bf16((d_out, d_in), 0.02, seed)
+                X = si.gaussian_bf16((b, d_in), 1.0, seed + 1)
+                dY = si.gaussian_bf16((b, d_out), 1.0, seed + 2)
+                L = si.gaussian_bf16((d_in, r), 0.01, seed + 3)
+                R = si.gaussian_bf16((r, d_out), 0.01, seed + 4)
+                layer = GpuLayer(W)
+                Xd, dYd, Ld, Rd = dev(B, X), dev(B, dY), dev(B, L), dev(B, R)
+                outs = None
+                for _ in range(10):
+                    T = layer.adapter_T(Xd, Ld)
+                    Y = layer.fwd(Xd, T, Rd)
+                    dT, dL, dR = layer.adapter_bwd(Xd, dYd, Ld, Rd, T)
+                    dX = layer.dx(dYd, dT, Ld)
+                    dWc = layer.dw(dYd, Xd)
+                    outs = (Y, dX, dWc)
+                stream.synchronize()
+                results[idx] = (W, X, dY, L, R, [B.bits_from_bf16(t) for t in outs], layer.mask1.cpu().numpy(),
+                                layer.mask2.cpu().numpy())
+        except Exception as ex:                         # noqa: BLE001
+            errors.append(ex)
+
+    threads = [threading.Thread(target=work, args=(i, *spec)) for i, spec in enumerate(specs)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    assert B.slope_poll_status() == 0
+    for idx, (d_in, d_out, b, r, seed) in enumerate(specs):
+        W, X, dY, L, R, (Y, dX, dWc), m1, m2 = results[idx]
+        _, _, mask1 = oracle.prune24(W)
+        _, _, mask2 = oracle.double_prune(W, mask1)
+        assert np.array_equal(m1, mask1) and np.array_equal(m2, mask2)
+        rows = np.arange(b)
+        assert rel_fro(to_f64(Y), oracle.fwd_rows(X, W, mask1, rows, L, R)) <= REL_TOL
+        assert rel_fro(to_f64(dX), oracle.dx_rows(dY, W, mask2, rows, L, R)) <= REL_TOL
+        assert rel_fro(to_f64(dWc), oracle.dw_rows(dY, X, mask1, np.arange(d_out))) <= REL_TOL
