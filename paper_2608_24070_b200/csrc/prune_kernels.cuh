@@ -244,70 +244,86 @@ __global__ void __launch_bounds__(256) sparse_add_kernel(const uint4* A, const u
 
 // "updateSparseMatrix" for the transposed copy: rebuild the values of the compressed
 // (W^{R,C})^T from new forward values Wc_new under the static masks.  Tile (rb, cb) of W
-// (128 x 128 elements = 128 x 64 compressed values) feeds tile (cb, rb) of the transposed copy:
-// its metadata block says which two rows of every 4-row group were kept by the second pass,
-// the first-pass mask says whether such an element exists at all and at which rank it sits
-// in its row's compressed group.
-constexpr int kDpOutPitch = 136;                // bytes per staged output row (128 + 8)
-constexpr int kUpdWcPitchW = 33;                 // 32-bit words per staged row of 64 bf16 (+1 pad)
-constexpr int kUpdSmemBytes = 128 * kUpdWcPitchW * 4 + 2048 + 2048 + 128 * kDpOutPitch;
+// (128 x 128 elements = 128 x 64 compressed values) feeds tile (cb, rb) of the transposed copy.
+// Same orientation trick as the second pruning pass: a thread owns 8 rows x 8 columns of W,
+// rebuilt from 8 bytes of compressed values and one first-pass mask byte per row (a pruned entry
+// is +0), so a 32-bit word is a pair of adjacent columns; the stored 2-bit codes of the
+// transposed copy's metadata say which two rows of every 4-row group go into its slots.  Only the
+// output is transposed, through the same XOR-swizzled staging tile.
+__device__ __forceinline__ void expand_compressed_row(uint2 cw, uint32_t mask_byte, uint32_t (&d)[4]) {
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+        const uint32_t pair = g == 0 ? cw.x : cw.y;
+        const uint32_t first = pair & 0xFFFFu, second = pair >> 16;
+        const uint32_t nib = (mask_byte >> (4 * g)) & 0xFu;
+        const uint32_t k0 = nib & 1u, k1 = (nib >> 1) & 1u, k2 = (nib >> 2) & 1u, k3 = (nib >> 3) & 1u;
+        const uint32_t v0 = k0 ? first : 0u;
+        const uint32_t v1 = k1 ? (k0 ? second : first) : 0u;
+        const uint32_t v2 = k2 ? ((k0 | k1) ? second : first) : 0u;
+        const uint32_t v3 = k3 ? second : 0u;                    // exactly two bits are set: the last is the second
+        d[2 * g] = v0 | (v1 << 16);
+        d[2 * g + 1] = v2 | (v3 << 16);
+    }
+}
 
-__global__ void __launch_bounds__(256) update_transposed_kernel(const uint4* __restrict__ Wc_new,
-                                                                const uint8_t* __restrict__ mask1,
-                                                                const uint4* __restrict__ metaT, int d_out, int d_in,
-                                                                uint4* __restrict__ valsT) {
-    extern __shared__ __align__(16) uint8_t up_smem[];
-    uint32_t* s_wc = reinterpret_cast<uint32_t*>(up_smem);
-    uint8_t* s_m1 = up_smem + 128 * kUpdWcPitchW * 4;
-    uint8_t* s_mt = s_m1 + 2048;
-    uint8_t* s_out = s_mt + 2048;
+__device__ __forceinline__ uint32_t pick_row(uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3, uint32_t q) {
+    const uint32_t lo = (q & 1u) ? r1 : r0, hi = (q & 1u) ? r3 : r2;
+    return (q & 2u) ? hi : lo;
+}
+
+__global__ void __launch_bounds__(256, 4) update_transposed_kernel(const uint2* __restrict__ Wc_new,
+                                                                   const uint8_t* __restrict__ mask1,
+                                                                   const uint4* __restrict__ metaT, int d_out, int d_in,
+                                                                   uint4* __restrict__ valsT) {
+    __shared__ __align__(16) uint8_t s_out[128 * 128];       // [column j][16 slots of 8 B], slot index XOR (j >> 3)
+    __shared__ __align__(16) uint8_t s_meta[2048];
 
     const int cb = blockIdx.x, rb = blockIdx.y;
     const int tid = threadIdx.x;
-    const size_t wc_row_u4 = static_cast<size_t>(d_in) >> 4;        // uint4 per compressed row (d_in/2 bf16)
-#pragma unroll
-    for (int pass = 0; pass < 4; ++pass) {
-        const int rr = pass * 32 + (tid >> 3), seg = tid & 7;
-        const uint4 v = __ldg(Wc_new + (static_cast<size_t>(rb) * 128 + rr) * wc_row_u4 + cb * 8 + seg);
-        uint32_t* dst = s_wc + rr * kUpdWcPitchW + seg * 4;
-        dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
-    }
+    const int c8 = tid & 15;                                 // 8-column slot of the tile
+    const int ig = tid >> 4;                                 // 8-row slot of the tile
+    const size_t row_u2 = static_cast<size_t>(d_in) >> 3;    // 8-byte units per compressed row = mask bytes per row
+
     if (tid < 128) {
-        const size_t row = static_cast<size_t>(rb) * 128 + tid;
-        reinterpret_cast<uint4*>(s_m1)[tid] = __ldg(reinterpret_cast<const uint4*>(mask1 + row * (d_in >> 3)) + cb);
-    } else {
         const size_t blk = static_cast<size_t>(cb) * (d_out >> 7) + rb;
-        reinterpret_cast<uint4*>(s_mt)[tid - 128] = __ldg(metaT + blk * 128 + (tid - 128));
+        reinterpret_cast<uint4*>(s_meta)[tid] = __ldg(metaT + blk * 128 + tid);
+    }
+    uint32_t d[8][4];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+        const size_t at = (static_cast<size_t>(rb) * 128 + ig * 8 + t) * row_u2 + cb * 16 + c8;
+        expand_compressed_row(__ldg(Wc_new + at), __ldg(mask1 + at), d[t]);
     }
     __syncthreads();
 
-    const int j = tid & 127;
-    const uint16_t* s_wc16 = reinterpret_cast<const uint16_t*>(s_wc);
-    auto fetch = [&](int i) -> uint32_t {
-        const uint32_t mbyte = s_m1[i * 16 + (j >> 3)];
-        const uint32_t kept = (mbyte >> (j & 7)) & 1u;
-        const uint32_t group = (mbyte >> (j & 4)) & 0xFu;
-        const int rank = __popc(group & ((1u << (j & 3)) - 1u));
-        return kept ? s_wc16[i * (kUpdWcPitchW * 2) + 2 * (j >> 2) + rank] : 0u;
-    };
-#pragma unroll 1
-    for (int it = 0; it < 8; ++it) {
-        const int ig = it * 2 + (tid >> 7);
-        const uint32_t code = s_mt[meta_byte_offset(j, ig)];
-        const int base = ig * 8;
-        uint2 out;
-        out.x = fetch(base + (code & 3)) | (fetch(base + ((code >> 2) & 3)) << 16);
-        out.y = fetch(base + 4 + ((code >> 4) & 3)) | (fetch(base + 4 + ((code >> 6) & 3)) << 16);
-        *reinterpret_cast<uint2*>(s_out + j * kDpOutPitch + ig * 8) = out;
+    const int meta_base = meta_byte_offset(c8 * 8, ig);      // + 16 per column inside the 8-column slot
+    const int slot = (ig ^ c8) * 8;
+#pragma unroll
+    for (int wi = 0; wi < 4; ++wi) {
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int k = 2 * wi + half;
+            const uint32_t code = s_meta[meta_base + 16 * k];   // rows 0..3: low nibble, rows 4..7: high nibble
+            uint32_t r[8];
+#pragma unroll
+            for (int t = 0; t < 8; ++t) r[t] = (d[t][wi] >> (16 * half)) & 0xFFFFu;
+            const uint32_t a = pick_row(r[0], r[1], r[2], r[3], code & 3u) |
+                               (pick_row(r[0], r[1], r[2], r[3], (code >> 2) & 3u) << 16);
+            const uint32_t b = pick_row(r[4], r[5], r[6], r[7], (code >> 4) & 3u) |
+                               (pick_row(r[4], r[5], r[6], r[7], (code >> 6) & 3u) << 16);
+            *reinterpret_cast<uint2*>(s_out + (c8 * 8 + k) * 128 + slot) = make_uint2(a, b);
+        }
     }
     __syncthreads();
-    const size_t vrow_u4 = static_cast<size_t>(d_out) >> 4;
+
+    const size_t vrow_u4 = static_cast<size_t>(d_out) >> 4;        // uint4 per row of valsT (d_out/2 bf16)
 #pragma unroll
     for (int pass = 0; pass < 4; ++pass) {
-        const int jr = pass * 32 + (tid >> 3), seg = tid & 7;
-        const uint2 a = *reinterpret_cast<const uint2*>(s_out + jr * kDpOutPitch + seg * 16);
-        const uint2 b = *reinterpret_cast<const uint2*>(s_out + jr * kDpOutPitch + seg * 16 + 8);
-        valsT[(static_cast<size_t>(cb) * 128 + jr) * vrow_u4 + rb * 8 + seg] = make_uint4(a.x, a.y, b.x, b.y);
+        const int jr = pass * 32 + (tid >> 3), seg = tid & 7;      // logical slots 2*seg, 2*seg+1
+        const int x = (jr >> 3) & 15;
+        const uint4 v = *reinterpret_cast<const uint4*>(s_out + jr * 128 + (((2 * seg) ^ x) >> 1) * 16);
+        const uint4 o = (x & 1) ? make_uint4(v.z, v.w, v.x, v.y) : v;
+        valsT[(static_cast<size_t>(cb) * 128 + jr) * vrow_u4 + rb * 8 + seg] = o;
     }
 }
 

@@ -771,10 +771,9 @@ slope_status_t slope_update_sparse_matrix(const void* Wc_vals, const void* mask1
         return SLOPE_ERR_ALIGNMENT;
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
-    if (!set_smem(update_transposed_kernel, kUpdSmemBytes)) return SLOPE_ERR_CUDA;
     dim3 grid(d_in / 128, d_out / 128);
-    update_transposed_kernel<<<grid, 256, kUpdSmemBytes, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const uint4*>(Wc_vals), static_cast<const uint8_t*>(mask1_bits),
+    update_transposed_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint2*>(Wc_vals), static_cast<const uint8_t*>(mask1_bits),
         static_cast<const uint4*>(WTc_meta), d_out, d_in, static_cast<uint4*>(WTc_vals));
     return launch_result();
 }
