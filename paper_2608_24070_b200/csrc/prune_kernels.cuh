@@ -250,25 +250,19 @@ __global__ void __launch_bounds__(256) sparse_add_kernel(const uint4* A, const u
 // is +0), so a 32-bit word is a pair of adjacent columns; the stored 2-bit codes of the
 // transposed copy's metadata say which two rows of every 4-row group go into its slots.  Only the
 // output is transposed, through the same XOR-swizzled staging tile.
-__device__ __forceinline__ void expand_compressed_row(uint2 cw, uint32_t mask_byte, uint32_t (&d)[4]) {
+// Byte-permute selectors that scatter the two kept values of a 4-column group (bytes 0-1 and
+// 2-3 of the compressed word; bytes 4-7 of the permute read zero) to their columns: low 16 bits
+// for columns 0-1, high 16 bits for columns 2-3.  One entry per 4-bit pattern of the first mask.
+__device__ __forceinline__ uint32_t expand_selector(uint32_t nib) {
+    uint32_t sel = 0, rank = 0;
 #pragma unroll
-    for (int g = 0; g < 2; ++g) {
-        const uint32_t pair = g == 0 ? cw.x : cw.y;
-        const uint32_t first = pair & 0xFFFFu, second = pair >> 16;
-        const uint32_t nib = (mask_byte >> (4 * g)) & 0xFu;
-        const uint32_t k0 = nib & 1u, k1 = (nib >> 1) & 1u, k2 = (nib >> 2) & 1u, k3 = (nib >> 3) & 1u;
-        const uint32_t v0 = k0 ? first : 0u;
-        const uint32_t v1 = k1 ? (k0 ? second : first) : 0u;
-        const uint32_t v2 = k2 ? ((k0 | k1) ? second : first) : 0u;
-        const uint32_t v3 = k3 ? second : 0u;                    // exactly two bits are set: the last is the second
-        d[2 * g] = v0 | (v1 << 16);
-        d[2 * g + 1] = v2 | (v3 << 16);
+    for (int k = 0; k < 4; ++k) {
+        const bool kept = (nib >> k) & 1u;
+        const uint32_t byte = kept ? 2u * min(rank, 1u) : 4u;
+        sel |= (byte | ((byte + 1u) << 4)) << (8 * k);
+        rank += kept ? 1u : 0u;
     }
-}
-
-__device__ __forceinline__ uint32_t pick_row(uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3, uint32_t q) {
-    const uint32_t lo = (q & 1u) ? r1 : r0, hi = (q & 1u) ? r3 : r2;
-    return (q & 2u) ? hi : lo;
+    return sel;
 }
 
 __global__ void __launch_bounds__(256, 4) update_transposed_kernel(const uint2* __restrict__ Wc_new,
@@ -277,6 +271,7 @@ __global__ void __launch_bounds__(256, 4) update_transposed_kernel(const uint2* 
                                                                    uint4* __restrict__ valsT) {
     __shared__ __align__(16) uint8_t s_out[128 * 128];       // [column j][16 slots of 8 B], slot index XOR (j >> 3)
     __shared__ __align__(16) uint8_t s_meta[2048];
+    __shared__ uint32_t s_expand[16];
 
     const int cb = blockIdx.x, rb = blockIdx.y;
     const int tid = threadIdx.x;
@@ -288,13 +283,25 @@ __global__ void __launch_bounds__(256, 4) update_transposed_kernel(const uint2* 
         const size_t blk = static_cast<size_t>(cb) * (d_out >> 7) + rb;
         reinterpret_cast<uint4*>(s_meta)[tid] = __ldg(metaT + blk * 128 + tid);
     }
-    uint32_t d[8][4];
+    if (tid >= 128 && tid < 144) s_expand[tid - 128] = expand_selector(tid - 128);
+    uint2 cw[8];
+    uint32_t mb[8];
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
         const size_t at = (static_cast<size_t>(rb) * 128 + ig * 8 + t) * row_u2 + cb * 16 + c8;
-        expand_compressed_row(__ldg(Wc_new + at), __ldg(mask1 + at), d[t]);
+        cw[t] = __ldg(Wc_new + at);
+        mb[t] = __ldg(mask1 + at);
     }
     __syncthreads();
+    uint32_t d[8][4];                                        // 8 rows x 4 column pairs of W^R
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+        const uint32_t s0 = s_expand[mb[t] & 15u], s1 = s_expand[mb[t] >> 4];
+        d[t][0] = __byte_perm(cw[t].x, 0u, s0);
+        d[t][1] = __byte_perm(cw[t].x, 0u, s0 >> 16);
+        d[t][2] = __byte_perm(cw[t].y, 0u, s1);
+        d[t][3] = __byte_perm(cw[t].y, 0u, s1 >> 16);
+    }
 
     const int meta_base = meta_byte_offset(c8 * 8, ig);      // + 16 per column inside the 8-column slot
     const int slot = (ig ^ c8) * 8;
@@ -304,13 +311,14 @@ __global__ void __launch_bounds__(256, 4) update_transposed_kernel(const uint2* 
         for (int half = 0; half < 2; ++half) {
             const int k = 2 * wi + half;
             const uint32_t code = s_meta[meta_base + 16 * k];   // rows 0..3: low nibble, rows 4..7: high nibble
-            uint32_t r[8];
-#pragma unroll
-            for (int t = 0; t < 8; ++t) r[t] = (d[t][wi] >> (16 * half)) & 0xFFFFu;
-            const uint32_t a = pick_row(r[0], r[1], r[2], r[3], code & 3u) |
-                               (pick_row(r[0], r[1], r[2], r[3], (code >> 2) & 3u) << 16);
-            const uint32_t b = pick_row(r[4], r[5], r[6], r[7], (code >> 4) & 3u) |
-                               (pick_row(r[4], r[5], r[6], r[7], (code >> 6) & 3u) << 16);
+            // column k of rows (0,1), (2,3), (4,5), (6,7) as four words, then one byte permute per
+            // row group picks rows q0 (low half) and q1 (high half): bytes 2q, 2q+1 of 8.
+            const uint32_t col = half ? 0x7632u : 0x5410u;
+            const uint32_t r01 = __byte_perm(d[0][wi], d[1][wi], col), r23 = __byte_perm(d[2][wi], d[3][wi], col);
+            const uint32_t r45 = __byte_perm(d[4][wi], d[5][wi], col), r67 = __byte_perm(d[6][wi], d[7][wi], col);
+            const uint32_t sel_a = 0x1010u + (code & 3u) * 0x22u + ((code >> 2) & 3u) * 0x2200u;
+            const uint32_t sel_b = 0x1010u + ((code >> 4) & 3u) * 0x22u + (code >> 6) * 0x2200u;
+            const uint32_t a = __byte_perm(r01, r23, sel_a), b = __byte_perm(r45, r67, sel_b);
             *reinterpret_cast<uint2*>(s_out + (c8 * 8 + k) * 128 + slot) = make_uint2(a, b);
         }
     }
