@@ -390,6 +390,14 @@ def main():
             bytes_ = d_in * d_out * (3.25 if op == "prune_24" else 3.25)   # double prune: 2 + 0.125 in, 1 + 0.125 out
             stage_rows.append({"layer": name, "d_in": d_in, "d_out": d_out, "op": op, "ms": round(ms, 4),
                                "gbs": round(bytes_ / (ms * 1e-3) / 1e9, 1)})
+        elif op in ("adapter_T", "adapter_bwd") and (d_in, d_out, op) not in seen:
+            # T = X L streams X once; the backward streams dY once for dT and X, dY once more for dL, dR
+            seen.add((d_in, d_out, op))
+            small = 2.0 * s.r * (s.b + d_in + d_out)
+            bytes_ = 2.0 * s.b * d_in + small if op == "adapter_T" else 2.0 * s.b * (d_in + 2 * d_out) + 3 * small
+            stage_rows.append({"layer": name, "d_in": d_in, "d_out": d_out, "op": op, "ms": round(ms, 4),
+                               "gbs": round(bytes_ / (ms * 1e-3) / 1e9, 1),
+                               "frac_of_hbm_peak": round(bytes_ / (ms * 1e-3) / 1e9 / pk["hbm_gbs"], 3)})
 
     # roofline of the two tensor-core kernels; the dominant one (by time inside the step) is "roofline"
     dw_fl, dw_s = tot["linear_bwd_dw_masked"]
@@ -453,6 +461,7 @@ def main():
         out["forward_speedup_by_shape"] = forward_shape_sweep(torch, B, stream)
         out["small_configs_hot_cold"] = small_config_probe(torch, B, stream, pk)
         out["dense_layer"] = dense_comparison(torch, B, layers, stream)
+        out["decoder_block_c5"] = decoder_block_probe(torch)
         if args.cusparselt_context:
             out["cusparselt_context"] = cusparselt_context(torch, B, layers, stream)
         out["e2e"] = e2e_run(torch, B, layers, de_flops, max(2, min(args.steps, 5)))
@@ -811,6 +820,54 @@ def dense_comparison(torch, B, layers, stream, reps=5):
             "dense_ms": round(totals["cublas"], 4), "inhouse_dense_ms": round(totals["inhouse"], 4),
             "slope_ms": round(totals["slope"], 4), "speedup": round(totals["cublas"] / totals["slope"], 3),
             "speedup_vs_inhouse_dense": round(totals["inhouse"] / totals["slope"], 3), "layers": rows}
+
+
+def decoder_block_probe(torch, reps=5):
+    """c5_llama13b_block as one decoder-block training step with real data flow (normalisation ->
+    q, k, v -> causal attention -> o -> residual -> normalisation -> gate, up -> SiLU * up -> down
+    -> residual; forward + backward, no optimizer).  The seven linears run through the library
+    (rank-128 adapters) or, for the all-dense arm, through torch (cuBLAS); normalisation,
+    attention, gate and residuals are torch in both arms.  Linear calls are bracketed by CUDA
+    events inside the step, so their sum is reported next to the whole-block time."""
+    from paper_2608_24070_b200 import block_harness as H
+
+    wl = si.WORKLOADS["c5_llama13b_block"]
+    batch, seq, heads, r = 4, 2048, 40, wl.rank
+    tokens, d = batch * seq, wl.layers[0].d_in
+    gen = torch.Generator(device="cuda").manual_seed(si.seed_for(5, 0, "W"))
+    mk = lambda shape, sigma: (torch.randn(shape, device="cuda", generator=gen) * sigma).bfloat16()
+    arms = {"slope": {}, "dense": {}}
+    for l in wl.layers:
+        W = mk((l.d_out, l.d_in), 0.02)
+        arms["slope"][l.name] = H.SlopeLinear(W, mk((l.d_in, r), 0.01), mk((r, l.d_out), 0.01), max_tokens=tokens)
+        arms["dense"][l.name] = H.DenseLinear(W)
+        del W
+    x, dout = mk((tokens, d), 1.0), mk((tokens, d), 1.0)
+    block_ms = {k: [] for k in arms}
+    linear_ms = {k: [] for k in arms}
+    for _ in range(reps + 2):
+        for k, layers in arms.items():
+            timers = []
+            for lay in layers.values():
+                lay.timers = timers
+                if k == "dense":
+                    lay.W.grad = None
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            H.block_step(x, dout, layers, batch, seq, heads)
+            e1.record()
+            torch.cuda.synchronize()
+            block_ms[k].append(e0.elapsed_time(e1))
+            linear_ms[k].append(H.elapsed_ms(timers))
+    med = lambda v: statistics.median(v[2:])
+    res = {k: {"linears_ms": round(med(linear_ms[k]), 4), "block_ms": round(med(block_ms[k]), 4)} for k in arms}
+    return {"what": "one decoder-block step (forward + backward) at LLaMA-13B width: 8192 tokens = 4 x 2048, 40 heads, "
+                    "seven linears through the library with rank-128 adapters vs the same block with dense torch "
+                    "(cuBLAS) linears and no adapters; non-linear glue is torch in both; seeded torch.randn inputs; "
+                    "median of %d steps after 2 warm-ups, arms interleaved" % reps,
+            **res,
+            "speedup_linears": round(res["dense"]["linears_ms"] / res["slope"]["linears_ms"], 3),
+            "speedup_block": round(res["dense"]["block_ms"] / res["slope"]["block_ms"], 3)}
 
 
 def cusparselt_context(torch, B, layers, stream, reps=10):
