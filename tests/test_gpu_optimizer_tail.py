@@ -26,7 +26,7 @@ def bf16_round(x64):
     return to_f64(si.f32_to_bf16_bits(x64.astype(np.float32)))
 
 
-@pytest.mark.parametrize("rows,cols", [(512, 512), (384, 1152)])
+@pytest.mark.parametrize("rows,cols", [(512, 512), (384, 1152), (11008, 4096)])
 def test_sparse_add(B, oracle, rows, cols):
     import torch
 
@@ -38,8 +38,9 @@ def test_sparse_add(B, oracle, rows, cols):
     assert B.slope_poll_status() == 0
     got = to_f64(B.bits_from_bf16(out))
     ref = oracle.sparse_add(A, Bv, np.float32(beta), np.float32(gamma))
-    # the kernel rounds twice (fp32 arithmetic, then bf16): allow one bf16 ulp on ties, nothing more
-    ulp = np.abs(ref) * 2.0 ** -7
+    # the kernel rounds twice (fp32 arithmetic, then bf16): allow one bf16 ulp on ties, plus the fp32
+    # rounding of gamma * b where the two terms cancel (seen among 22 million elements, not among thousands)
+    ulp = np.abs(ref) * 2.0 ** -7 + np.abs(np.float64(np.float32(gamma)) * to_f64(Bv)) * 2.0 ** -22
     assert (np.abs(got - ref) <= ulp).all()
     assert (got == bf16_round(ref)).mean() > 0.999
     # identity: 1*A + 0*B is a bit copy
@@ -47,7 +48,7 @@ def test_sparse_add(B, oracle, rows, cols):
     assert np.array_equal(B.bits_from_bf16(out), A)
 
 
-@pytest.mark.parametrize("d_out,d_in", [(512, 512), (384, 640), (1280, 128)])
+@pytest.mark.parametrize("d_out,d_in", [(512, 512), (384, 640), (1280, 128), (11008, 4096)])
 def test_update_sparse_matrix(B, oracle, d_out, d_in):
     import torch
 
