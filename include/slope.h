@@ -15,8 +15,8 @@
  *  - `stream` is a cudaStream_t (NULL = the legacy default stream).  Calls are
  *    asynchronous with respect to the host.
  *  - Argument, shape, alignment and architecture errors are returned before
- *    anything is launched.  d_out, d_in must be multiples of 128; tokens b a
- *    multiple of 8 (b >= 8); adapter rank r in {0, 16, 32, ..., 256}.
+ *    anything is launched.  d_out, d_in must be multiples of 128; any number of
+ *    tokens b >= 1; adapter rank r in {0, 16, 32, ..., 256}.
  *    There is no CPU fallback: on a device that is not sm_100 the calls return
  *    SLOPE_ERR_UNSUPPORTED_ARCH.
  *  - Device-side waits are bounded; a wait that runs out makes the kernel stop

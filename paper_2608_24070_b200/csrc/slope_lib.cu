@@ -609,7 +609,7 @@ slope_status_t slope_linear_fwd(const void* X, int b, const void* Wc_vals, const
                                 const void* T, const void* R, int r, void* Y, void* stream) {
     if (!X || !Wc_vals || !Wc_meta || !Y) return SLOPE_ERR_INVALID_ARG;
     if (r != 0 && (!T || !R)) return SLOPE_ERR_INVALID_ARG;
-    if (!dims_ok(d_out, d_in) || b < 8 || b % 8 != 0 || !rank_ok(r)) return SLOPE_ERR_SHAPE;
+    if (!dims_ok(d_out, d_in) || b < 1 || !rank_ok(r)) return SLOPE_ERR_SHAPE;
     if (!aligned16(X) || !aligned16(Wc_vals) || !aligned16(Wc_meta) || !aligned16(Y) ||
         (r != 0 && (!aligned16(T) || !aligned16(R))))
         return SLOPE_ERR_ALIGNMENT;
@@ -623,7 +623,7 @@ slope_status_t slope_linear_bwd_dx(const void* dY, int b, const void* WTc_vals, 
                                    int d_in, const void* dT, const void* L, int r, void* dX, void* stream) {
     if (!dY || !WTc_vals || !WTc_meta || !dX) return SLOPE_ERR_INVALID_ARG;
     if (r != 0 && (!dT || !L)) return SLOPE_ERR_INVALID_ARG;
-    if (!dims_ok(d_out, d_in) || b < 8 || b % 8 != 0 || !rank_ok(r)) return SLOPE_ERR_SHAPE;
+    if (!dims_ok(d_out, d_in) || b < 1 || !rank_ok(r)) return SLOPE_ERR_SHAPE;
     if (!aligned16(dY) || !aligned16(WTc_vals) || !aligned16(WTc_meta) || !aligned16(dX) ||
         (r != 0 && (!aligned16(dT) || !aligned16(L))))
         return SLOPE_ERR_ALIGNMENT;
@@ -636,7 +636,7 @@ slope_status_t slope_linear_bwd_dx(const void* dY, int b, const void* WTc_vals, 
 slope_status_t slope_linear_bwd_dw_masked(const void* dY, const void* X, int b, int d_out, int d_in,
                                           const void* mask1_bits, void* dWc_vals, void* stream) {
     if (!dY || !X || !mask1_bits || !dWc_vals) return SLOPE_ERR_INVALID_ARG;
-    if (!dims_ok(d_out, d_in) || b < 8 || b % 8 != 0) return SLOPE_ERR_SHAPE;
+    if (!dims_ok(d_out, d_in) || b < 1) return SLOPE_ERR_SHAPE;
     if (!aligned16(dY) || !aligned16(X) || !aligned16(mask1_bits) || !aligned16(dWc_vals)) return SLOPE_ERR_ALIGNMENT;
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
@@ -659,7 +659,7 @@ slope_status_t slope_linear_bwd_dw_masked(const void* dY, const void* X, int b, 
 // ------------------------------------------------------------------ dense layer on the same pipeline
 static slope_status_t dense_args(const void* a, const void* b_, const void* c, int b, int d_out, int d_in) {
     if (!a || !b_ || !c) return SLOPE_ERR_INVALID_ARG;
-    if (!dims_ok(d_out, d_in) || b < 8 || b % 8 != 0) return SLOPE_ERR_SHAPE;
+    if (!dims_ok(d_out, d_in) || b < 1) return SLOPE_ERR_SHAPE;
     if (!aligned16(a) || !aligned16(b_) || !aligned16(c)) return SLOPE_ERR_ALIGNMENT;
     return SLOPE_OK;
 }
@@ -707,7 +707,7 @@ slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY, c
                                      void* workspace, size_t workspace_bytes, void* stream_) {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (phase != 0 && phase != 1) return SLOPE_ERR_INVALID_ARG;
-    if (!dims_ok(d_out, d_in) || b < 8 || b % 8 != 0 || !rank_ok(r) || r == 0) return SLOPE_ERR_SHAPE;
+    if (!dims_ok(d_out, d_in) || b < 1 || !rank_ok(r) || r == 0) return SLOPE_ERR_SHAPE;
     DeviceInfo info;
     if (phase == 0) {
         if (!X || !L || !T) return SLOPE_ERR_INVALID_ARG;
@@ -915,7 +915,7 @@ slope_status_t slope_adapter_dl_noalloc(const void* X, const void* dT, int b, in
                                         void* stream_) {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (!X || !dT || !dL) return SLOPE_ERR_INVALID_ARG;
-    if (d_in <= 0 || d_in % 128 != 0 || b < 8 || b % 8 != 0 || !rank_ok(r) || r == 0) return SLOPE_ERR_SHAPE;
+    if (d_in <= 0 || d_in % 128 != 0 || b < 1 || !rank_ok(r) || r == 0) return SLOPE_ERR_SHAPE;
     if (!aligned16(X) || !aligned16(dT) || !aligned16(dL)) return SLOPE_ERR_ALIGNMENT;
     const int splits = adapter_splits(b, d_in);
     const size_t need = static_cast<size_t>(splits) * d_in * r * sizeof(float);

@@ -47,7 +47,7 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     buf = ctypes.create_string_buffer(64)
     p = ctypes.cast(buf, ctypes.c_void_p)
     assert lib.slope_prune_24(p, 100, 128, p, p, null, null) == 2                      # shape
-    assert lib.slope_linear_fwd(p, 12, p, p, 128, 128, null, null, 0, p, null) == 2    # tokens % 8
+    assert lib.slope_linear_fwd(p, 0, p, p, 128, 128, null, null, 0, p, null) == 2     # no tokens
     assert lib.slope_linear_fwd(p, 16, p, p, 128, 128, null, null, 24, p, null) == 1   # rank without factors
     assert lib.slope_adapter_fwd_bwd(7, p, p, p, p, 16, 128, 128, 16, p, p, p, p, p, 0, null) == 1
     assert lib.slope_status_string(6) == b"device-side wait timed out"

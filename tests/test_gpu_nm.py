@@ -136,7 +136,7 @@ def _dense_dw_from_oracle(oracle, dY, X, d_out, d_in):
     return np.concatenate([a, b], axis=-1).reshape(d_out, d_in)
 
 
-@pytest.mark.parametrize("d_in,d_out,b", [(384, 640, 776), (1024, 256, 264), (128, 128, 8)])
+@pytest.mark.parametrize("d_in,d_out,b", [(384, 640, 776), (1024, 256, 264), (128, 128, 8), (256, 384, 77), (384, 256, 1)])
 def test_dense_layer_against_oracle(B, oracle, d_in, d_out, b):
     import torch
     from helpers import REL_TOL, rel_fro, to_f64

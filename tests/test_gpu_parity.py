@@ -116,6 +116,14 @@ CASES = [
     (1152, 384, 104, 128, 24),       # 104 tokens, ragged, two adapter K-steps, odd number of k-blocks
     (512, 768, 264, 256, 25),        # largest rank (6.25 % of a 4096-wide layer): two adapter column tiles
     (1024, 512, 16, 256, 26),        # largest rank at decode size
+    (512, 384, 1, 16, 27),           # one token (decode of a single sequence)
+    (1024, 512, 3, 0, 28),           # token counts that are no multiple of 8, on every kernel family:
+    (384, 640, 7, 32, 29),
+    (512, 512, 17, 64, 30),          #   few-token kernel, 64-token tile
+    (640, 384, 100, 32, 31),
+    (256, 384, 130, 0, 32),          #   tile kernels
+    (384, 512, 250, 16, 33),         #   adapter products still on the few-token kernel
+    (512, 256, 1001, 32, 34),        #   one-CTA dense kernels for T / dT, 16 token k-blocks with a tail of 41
 ]
 
 
