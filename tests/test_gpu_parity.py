@@ -392,6 +392,10 @@ def _fuzz_shapes():
         b = 8 * int(rng.choice([1, 2, 5, 8, 13, 16, 27, 32, 33, 70, 129, 300]))
         r = int(rng.choice([0, 16, 48, 64, 112, 128, 256]))
         shapes.append((d_in, d_out, b, r))
+    ragged = np.random.Generator(np.random.PCG64(20260825))          # token counts around every tile boundary
+    for b in (1, 5, 9, 31, 63, 65, 127, 129, 255, 257, 999, 2047):
+        shapes.append((128 * int(ragged.integers(1, 17)), 128 * int(ragged.integers(1, 17)), b,
+                       int(ragged.choice([0, 16, 64, 128]))))
     shapes += [(2560, 5120, 2048, 0),      # dW: 10 x 20 = 200 tiles -> 2 rounds + 52 tiles (no halving: more than half the pairs)
                (2304, 2560, 1000, 16),     # dW: 90 tiles -> 1 round + 16 tiles, halved
                (4096, 1280, 3080, 64)]     # 512-row sparse tiles with a partial last row tile (1280 = 2.5 tiles)
@@ -497,3 +501,42 @@ def test_two_host_threads_on_two_streams(B, oracle):
         assert rel_fro(to_f64(Y), oracle.fwd_rows(X, W, mask1, rows, L, R)) <= REL_TOL
         assert rel_fro(to_f64(dX), oracle.dx_rows(dY, W, mask2, rows, L, R)) <= REL_TOL
         assert rel_fro(to_f64(dWc), oracle.dw_rows(dY, X, mask1, np.arange(d_out))) <= REL_TOL
+
+
+@pytest.mark.parametrize("b", [1, 7, 17, 130, 250, 1001])
+def test_rows_past_the_last_token_are_never_written(B, oracle, b):
+    """Outputs live at the start of larger buffers filled with a sentinel: whatever tile a kernel
+    works in, nothing behind row b - 1 may change (forward, input gradient, adapter T and dT)."""
+    import torch
+
+    d_in, d_out, r, guard = 384, 512, 32, 96
+    W = si.gaussian_bf16((d_out, d_in), 0.02, 9100 + b)
+    layer = GpuLayer(W)
+    Xd = dev(B, si.gaussian_bf16((b, d_in), 1.0, 9200 + b))
+    dYd = dev(B, si.gaussian_bf16((b, d_out), 1.0, 9300 + b))
+    Ld = dev(B, si.gaussian_bf16((d_in, r), 0.01, 9400 + b))
+    Rd = dev(B, si.gaussian_bf16((r, d_out), 0.01, 9500 + b))
+    sentinel = 0x7FC1                                              # a NaN pattern no kernel produces from finite inputs
+
+    def guarded(cols):
+        buf = torch.full(((b + guard) * cols,), sentinel, dtype=torch.int16, device="cuda").view(torch.bfloat16)
+        return buf, buf[: b * cols].view(b, cols)
+
+    bufs = {}
+    bufs["T"], T = guarded(r)
+    bufs["dT"], dT = guarded(r)
+    bufs["Y"], Y = guarded(d_out)
+    bufs["dX"], dX = guarded(d_in)
+    dL = torch.empty((d_in, r), dtype=torch.bfloat16, device="cuda")
+    dR = torch.empty((r, d_out), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(B.slope_adapter_workspace_bytes(b, d_out, d_in, r), dtype=torch.uint8, device="cuda")
+    B.slope_adapter_fwd_bwd(0, Xd, None, Ld, None, b, d_out, d_in, r, T=T)
+    B.slope_linear_fwd(Xd, layer.Wc_vals, layer.Wc_meta, d_out, Y, T, Rd)
+    B.slope_adapter_fwd_bwd(1, Xd, dYd, Ld, Rd, b, d_out, d_in, r, T=T, dT=dT, dL=dL, dR=dR, workspace=ws)
+    B.slope_linear_bwd_dx(dYd, layer.WTc_vals, layer.WTc_meta, d_in, dX, dT, Ld)
+    layer.poll()
+    for name, buf in bufs.items():
+        cols = {"T": r, "dT": r, "Y": d_out, "dX": d_in}[name]
+        tail = buf.view(torch.int16)[b * cols:]
+        assert bool((tail == sentinel).all()), name
+        assert bool(torch.isfinite(buf[: b * cols].float()).all()), name
