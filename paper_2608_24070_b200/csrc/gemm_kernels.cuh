@@ -127,6 +127,10 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Programmatic dependent launch: the set-up above may overlap the tail of the previous kernel in
+    // the stream; no thread touches global memory before that kernel has completed.
+    griddep_launch_dependents();
+    griddep_wait();
 
     // tile -> (problem, m block, n block, split): m fastest so that concurrently running CTAs share B
     auto decode = [&](int tile, int& m_blk, int& n_blk, int& kb0, int& kb1) {
@@ -406,6 +410,10 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     cluster_sync_all();                                      // peer barriers are initialised
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Programmatic dependent launch: the set-up above may overlap the tail of the previous kernel in
+    // the stream; no thread touches global memory before that kernel has completed.
+    griddep_launch_dependents();
+    griddep_wait();
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both CTAs)
@@ -647,6 +655,10 @@ dense_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     cluster_sync_all();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Programmatic dependent launch: the set-up above may overlap the tail of the previous kernel in
+    // the stream; no thread touches global memory before that kernel has completed.
+    griddep_launch_dependents();
+    griddep_wait();
 
     if (warp == 0) {
         if (elect_one()) {
@@ -880,6 +892,10 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     cluster_sync_all();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Programmatic dependent launch: the set-up above may overlap the tail of the previous kernel in
+    // the stream; no thread touches global memory before that kernel has completed.
+    griddep_launch_dependents();
+    griddep_wait();
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both CTAs)

@@ -154,7 +154,8 @@ static int max_active_clusters(Kernel kern, int cluster, int threads, int smem_b
 template <typename... KArgs, typename... Args>
 static slope_status_t launch_pairs(void (*kern)(KArgs...), int grid, int threads, int smem_bytes,
                                    cudaStream_t stream, Args&&... args) {
-    return launch_cluster(kern, grid, 2, threads, smem_bytes, stream, std::forward<Args>(args)...);
+    return launch_cluster_ex(kern, grid, 2, threads, smem_bytes, /*overlap_prologue=*/true, stream,
+                             std::forward<Args>(args)...);
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -214,8 +215,8 @@ static slope_status_t launch_dense2(const DenseProblem& q0, const DenseProblem& 
     auto kern = dense_gemm_kernel<A_MN, B_MN, BLOCK_N, EPI, STAGES>;
     if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
     const int grid = tiles < info.sm_count ? tiles : info.sm_count;
-    kern<<<grid, kGemmThreads, Cfg::kSmemBytes, stream>>>(tm[0], tm[1], p[0], tm[2], tm[3], p[1]);
-    return launch_result();
+    return launch_cluster_ex(kern, grid, 1, kGemmThreads, Cfg::kSmemBytes, /*overlap_prologue=*/true, stream, tm[0],
+                             tm[1], p[0], tm[2], tm[3], p[1]);
 }
 
 template <bool A_MN, bool B_MN, int BLOCK_N, int EPI, int STAGES>
