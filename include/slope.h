@@ -91,10 +91,11 @@ slope_status_t slope_double_prune(const void* W, const void* mask1_bits, int d_o
  * With few tokens (inference, decode: the paper's forward-only inference measurements; always up
  * to 16 tokens, up to 128 where it is estimated faster than the tile kernels) the same call
  * runs on a kernel that streams the compressed weight once from HBM and splits the
- * reduction over a thread-block cluster; that launch is issued with programmatic stream
- * serialisation and synchronises on the device before it touches memory, so stream order
- * holds as for any other call.  Every compute call of this library can be captured in a CUDA
- * graph (slope_poll_status synchronises the stream and cannot).
+ * reduction over a thread-block cluster.  All GEMM launches of this library are issued with
+ * programmatic stream serialisation (their set-up may overlap the previous kernel's tail) and
+ * synchronise on the device before they touch memory, so stream order holds as for any other
+ * launch.  Every compute call of this library can be captured in a CUDA graph
+ * (slope_poll_status synchronises the stream and cannot).
  */
 slope_status_t slope_linear_fwd(const void* X, int b, const void* Wc_vals, const void* Wc_meta,
                                 int d_out, int d_in, const void* T, const void* R, int r,
