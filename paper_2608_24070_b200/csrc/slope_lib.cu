@@ -703,6 +703,16 @@ size_t slope_adapter_workspace_bytes(int b, int d_out, int d_in, int r) {
     return adapter_partial_bytes(b, d_in, r) + adapter_partial_bytes(b, d_out, r);     // dL and dR partial sums
 }
 
+// Column tile of the adapter products T = X L and dT = dY R^T (128 token rows per CTA).  These
+// launches are bound by what one SM can pull in, so more CTAs beat fewer bytes per CTA: with
+// r > 64, 64-column tiles double the CTA count (the second read of the activation rows comes from
+// L2) and win as long as all of them still run in one wave.
+static bool adapter_narrow_tiles(int b, int r, const DeviceInfo& info) {
+    if (r <= 64) return true;
+    const int wide_tiles = ((b + kBlockM - 1) / kBlockM) * ((r + 127) / 128);
+    return 2 * wide_tiles <= info.sm_count;
+}
+
 slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY, const void* L, const void* R, int b,
                                      int d_out, int d_in, int r, void* T, void* dT, void* dL, void* dR,
                                      void* workspace, size_t workspace_bytes, void* stream_) {
@@ -717,8 +727,9 @@ slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY, c
         // T[b x r] = X[b x d_in] * L[d_in x r]   (A = X, K contiguous; B = L^T stored [K x N])
         if (b <= kSkinnyMaxTokens)            // few tokens: split d_in over a cluster instead of one CTA
             return launch_skinny(nullptr, b, nullptr, nullptr, r, 0, X, L, d_in, true, T, stream, info);
-        return r <= 64 ? launch_dense<false, true, 64, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info)
-                       : launch_dense<false, true, 128, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info);
+        return adapter_narrow_tiles(b, r, info)
+                   ? launch_dense<false, true, 64, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info)
+                   : launch_dense<false, true, 128, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info);
     }
     if (!X || !dY || !R || !T || !dT || !dL || !dR || !workspace) return SLOPE_ERR_INVALID_ARG;
     if (!aligned16(X) || !aligned16(dY) || !aligned16(R) || !aligned16(T) || !aligned16(dT) || !aligned16(dL) ||
@@ -730,8 +741,9 @@ slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY, c
     // dT[b x r] = dY[b x d_out] * R[r x d_out]^T   (both K contiguous)
     st = b <= kSkinnyMaxTokens
              ? launch_skinny(nullptr, b, nullptr, nullptr, r, 0, dY, R, d_out, false, dT, stream, info)
-         : r <= 64 ? launch_dense<false, false, 64, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info)
-                 : launch_dense<false, false, 128, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info);
+         : adapter_narrow_tiles(b, r, info)
+             ? launch_dense<false, false, 64, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info)
+             : launch_dense<false, false, 128, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info);
     if (st) return st;
     // dL[d_in x r] = X^T dT and dR^T[d_out x r] = dY^T T: operands stored [K x M] / [K x N] with
     // K = tokens, split into fixed slices; both problems share one launch, their fp32 partial
