@@ -56,6 +56,49 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
+// Encoding a tensor map is a pure function of (address, extents, box, kind) and costs the host
+// about a microsecond; a layer calls with the same buffers step after step.  Each host thread
+// keeps the last encodings in a small direct-mapped table (no locks, nothing shared).
+struct TmapKey {
+    const void* base;
+    long long rows;
+    int cols, box_rows, box_cols, kind;
+    bool operator==(const TmapKey& o) const {
+        return base == o.base && rows == o.rows && cols == o.cols && box_rows == o.box_rows && box_cols == o.box_cols &&
+               kind == o.kind;
+    }
+};
+struct TmapSlot {
+    TmapKey key;
+    CUtensorMap tm;
+    bool valid;
+};
+constexpr int kTmapSlots = 256;
+
+static TmapSlot& tmap_slot(const TmapKey& k) {
+    thread_local TmapSlot table[kTmapSlots] = {};
+    unsigned long long h = reinterpret_cast<uintptr_t>(k.base) >> 4;
+    h = h * 0x9E3779B97F4A7C15ull + static_cast<unsigned long long>(k.rows) * 0xC2B2AE3D27D4EB4Full;
+    h ^= (static_cast<unsigned long long>(k.cols) << 20) ^ (static_cast<unsigned long long>(k.box_rows) << 8) ^
+         (static_cast<unsigned long long>(k.box_cols) << 2) ^ static_cast<unsigned long long>(k.kind);
+    h ^= h >> 29;
+    return table[h % kTmapSlots];
+}
+
+template <typename Encode>
+static bool tmap_memo(CUtensorMap* tm, const TmapKey& key, Encode encode) {
+    TmapSlot& slot = tmap_slot(key);
+    if (slot.valid && slot.key == key) {
+        std::memcpy(tm, &slot.tm, sizeof(CUtensorMap));
+        return true;
+    }
+    if (!encode(tm)) return false;
+    slot.key = key;
+    std::memcpy(&slot.tm, tm, sizeof(CUtensorMap));
+    slot.valid = true;
+    return true;
+}
+
 // 2-D bf16 tensor map over a row-major [rows x cols] matrix, 128-byte swizzle,
 // box = box_cols (<= 64) x box_rows, out-of-bounds elements read as zero.
 static bool make_tmap(CUtensorMap* tm, const void* base, int rows, int cols, int box_rows, int box_cols) {
@@ -65,9 +108,11 @@ static bool make_tmap(CUtensorMap* tm, const void* base, int rows, int cols, int
     const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(cols) * 2};
     const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
     const cuuint32_t estr[2] = {1, 1};
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return tmap_memo(tm, TmapKey{base, rows, cols, box_rows, box_cols, 0}, [&](CUtensorMap* out) {
+        return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
 }
 
 // Metadata as a 2-D tensor of 8-byte words [blocks x 256]: one 2 KB block is ONE contiguous row,
@@ -79,9 +124,11 @@ static bool make_tmap_meta(CUtensorMap* tm, const void* base, size_t total_bytes
     const cuuint64_t gstride[1] = {2048};
     const cuuint32_t box[2] = {256, 1};
     const cuuint32_t estr[2] = {1, 1};
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(base), gdim, gstride, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return tmap_memo(tm, TmapKey{base, static_cast<long long>(total_bytes / 2048), 256, 1, 256, 1}, [&](CUtensorMap* out) {
+        return fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
 }
 
 // Plain (unswizzled) 2-D bf16 tensor map, used for TMA stores of output tiles.
@@ -92,9 +139,11 @@ static bool make_tmap_plain(CUtensorMap* tm, const void* base, int rows, int col
     const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(cols) * 2};
     const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
     const cuuint32_t estr[2] = {1, 1};
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return tmap_memo(tm, TmapKey{base, rows, cols, box_rows, box_cols, 2}, [&](CUtensorMap* out) {
+        return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
 }
 
 // Launch with thread-block clusters of `cluster` CTAs along x.
@@ -172,12 +221,26 @@ static slope_status_t launch_result() {
     return cudaGetLastError() == cudaSuccess ? SLOPE_OK : SLOPE_ERR_CUDA;
 }
 
-// Opt in to more than 48 KB of dynamic shared memory.  Set on every launch: the attribute
-// belongs to the current device's context, and a cached "already done" flag would be wrong
-// for a second device or a second host thread.
+// Opt in to more than 48 KB of dynamic shared memory.  The attribute belongs to the kernel in
+// the current device's context; every host thread remembers which (kernel, device) pairs it has
+// already set (a process-wide flag would be wrong for a second device).
 template <typename Kernel>
 static bool set_smem(Kernel k, int bytes) {
-    return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+    struct Done {
+        const void* fn;
+        int dev, bytes;
+    };
+    constexpr int kMax = 64;
+    thread_local Done done[kMax];
+    thread_local int n_done = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    const void* fn = reinterpret_cast<const void*>(k);
+    for (int i = 0; i < n_done; ++i)
+        if (done[i].fn == fn && done[i].dev == dev && done[i].bytes >= bytes) return true;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    if (n_done < kMax) done[n_done++] = Done{fn, dev, bytes};
+    return true;
 }
 
 // Grid of the grid-stride streaming kernels: many short blocks per SM keep the tail of the last
