@@ -7,7 +7,7 @@
 // loops, tensor memory is released and the kernel returns.
 //
 //   dense_gemm_kernel          1 CTA per 128 x N tile; the skinny adapter GEMMs and small dW
-//   dense_gemm_pair_kernel     CTA pair per 256 x 256 tile (cta_group::2), the last round's tiles
+//   dense_gemm_pair_kernel     CTA pair per 256 x 256 tile (cta_group::2), the last wave's tiles
 //                              halved; dW (masked epilogue) and the dense layer (store epilogue)
 //   sparse_gemm_pair_kernel    CTA pair per 256 x 224 (or 256 x 128) tile, tcgen05.mma.sp;
 //                              forward / dX with short reductions or few tiles
@@ -582,10 +582,10 @@ __device__ __forceinline__ void raster_tile(int tile, int num_m, int num_n, int&
 }
 
 // Work items of the persistent CTA-pair GEMM.  Items are tiles in raster order; when the tiles
-// left over after the last full round of the machine (num_tiles mod num_pairs) fill at most
-// half of the pairs, each of them is cut into two half-width items, so that the last round
+// left over after the last full wave of the machine (num_tiles mod num_pairs) fill at most
+// half of the pairs, each of them is cut into two half-width items, so that the last wave
 // takes half the time instead of a full tile time on a half-empty machine (4096 x 4096 weight
-// gradient: 256 tiles on 74 pairs = 3 rounds + 34 tiles -> 68 half items: 3.5 instead of 4 rounds).
+// gradient: 256 tiles on 74 pairs = 3 waves + 34 tiles -> 68 half items: 3.5 instead of 4 waves).
 struct PairWork {
     int m_pair, n0, width;
 };

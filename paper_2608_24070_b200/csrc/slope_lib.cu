@@ -330,9 +330,9 @@ constexpr int kQuadStages = 3;
 
 // Row tiles per raster group of the 512-row-tile kernel (see quad_tile).  All pairs that work on
 // one token block share its activations, so with every row tile in one group the activations
-// cross HBM once -- but a round of the machine then touches the whole compressed weight, and
+// cross HBM once -- but a wave of the machine then touches the whole compressed weight, and
 // when that is more than L2 keeps next to the streams (about 30 MB here) it is fetched again
-// every round.  Splitting the row tiles into g groups re-reads the activations g times and keeps
+// every wave.  Splitting the row tiles into g groups re-reads the activations g times and keeps
 // a group's weights resident.  Pick the g with the least estimated DRAM traffic
 // (measured at 16384 tokens: 4096 -> 11008 two groups +7 %, 5120 -> 13824 three groups +11 %,
 // square and long-reduction layers one group).
@@ -499,8 +499,8 @@ static slope_status_t launch_skinny(const void* act, int ntok, const void* vals,
 //              while at 768 the 256-row tile is up to 25 % faster.
 //   256 x 224  double-buffered accumulators.
 //   256 x 128  the same kernel with a narrower token tile: more, smaller tiles for shapes that
-//              would otherwise leave much of the last round of the machine empty (2048 x 2048
-//              with 2048 tokens: 80 tiles of 256 x 224 on 74 CTA pairs = 2 rounds for 1.08 rounds
+//              would otherwise leave much of the last wave of the machine empty (2048 x 2048
+//              with 2048 tokens: 80 tiles of 256 x 224 on 74 CTA pairs = 2 waves for 1.08 waves
 //              of work); it stages the weights for fewer tokens, which costs 12 % more time
 //              per unit of work at short reductions and 30-35 % at long ones (measured at 2048
 //              tokens).
@@ -525,7 +525,7 @@ static SparseTile choose_sparse_tile(int M, int K, int ntok, int num_pairs) {
 // Few-token kernel or tile kernel?  Decode sizes (<= 16 tokens) always stream the weights through
 // the few-token kernel.  Up to 128 tokens the two are compared by estimate: the few-token kernel's
 // own cost model against a tile kernel that has one token tile, i.e. M / 256 tiles which each
-// walk the whole reduction (measured: ~4 us per launch plus 0.32 us per k-block and round of the
+// walk the whole reduction (measured: ~4 us per launch plus 0.32 us per k-block and wave of the
 // machine).  A tall weight (4096 -> 11008) then has enough tiles for the tile kernel, a long
 // reduction on few rows (11008 -> 4096) wants the K-split of the few-token kernel.  Beyond 128
 // tokens the 256-token variant of the few-token kernel pays 512 row requests per k-block for

@@ -167,7 +167,7 @@ def test_layer_against_oracle(B, oracle, d_in, d_out, b, r, seed):
 
 @pytest.mark.parametrize("d_in,d_out,b,r", [(4096, 1024, 4104, 32), (1024, 4096, 4104, 0)])
 def test_512_row_tile_kernel_on_sampled_rows(B, oracle, d_in, d_out, b, r):
-    """Shapes for which the kernel choice takes the 512-row tile (38 tiles fill one round where 76
+    """Shapes for which the kernel choice takes the 512-row tile (38 tiles fill one wave where 76
     256-row tiles would need two), with a ragged token tail: sampled token rows against the oracle."""
     W = si.gaussian_bf16((d_out, d_in), 0.02, 131)
     X = si.gaussian_bf16((b, d_in), 1.0, 132)
@@ -383,7 +383,7 @@ def test_optional_masks_and_run_to_run_determinism(B, oracle):
 def _fuzz_shapes():
     """Seeded shapes that hit every branch of the kernel choice: few-token tiles of all four widths with
     one to eight K-splits, 256-row and 512-row sparse tiles, weight-gradient launches with and without
-    halved last-round tiles, one-CTA weight-gradient tiles, ranks from 16 to 256."""
+    halved last-wave tiles, one-CTA weight-gradient tiles, ranks from 16 to 256."""
     rng = np.random.Generator(np.random.PCG64(20260824))
     shapes = []
     for _ in range(20):
@@ -396,8 +396,8 @@ def _fuzz_shapes():
     for b in (1, 5, 9, 31, 63, 65, 127, 129, 255, 257, 999, 2047):
         shapes.append((128 * int(ragged.integers(1, 17)), 128 * int(ragged.integers(1, 17)), b,
                        int(ragged.choice([0, 16, 64, 128]))))
-    shapes += [(2560, 5120, 2048, 0),      # dW: 10 x 20 = 200 tiles -> 2 rounds + 52 tiles (no halving: more than half the pairs)
-               (2304, 2560, 1000, 16),     # dW: 90 tiles -> 1 round + 16 tiles, halved
+    shapes += [(2560, 5120, 2048, 0),      # dW: 10 x 20 = 200 tiles -> 2 waves + 52 tiles (no halving: more than half the pairs)
+               (2304, 2560, 1000, 16),     # dW: 90 tiles -> 1 wave + 16 tiles, halved
                (4096, 1280, 3080, 64)]     # 512-row sparse tiles with a partial last row tile (1280 = 2.5 tiles)
     return shapes
 
