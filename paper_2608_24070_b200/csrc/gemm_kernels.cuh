@@ -347,6 +347,16 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const SplitKReduce r
 // the barriers of both CTAs; the epilogues release an accumulator stage by arriving on the
 // leader's barrier through the cluster shared-memory window.
 // =====================================================================================
+// Token tiles are BLOCK_N wide except the last one of a ragged token count, which is only as wide
+// as the tokens that are left (rounded up to the 32-token block of the epilogue): the MMAs run
+// with that N, the second CTA's half of the activations starts at its middle, and the epilogue
+// stops there.  A 2048-token forward on 224-token tiles ends in a 32-token tile that costs a
+// fraction of a full one instead of a whole wave of the machine.
+__device__ __forceinline__ int token_tile_width(int ntok, int n0, int block_n) {
+    const int left = ntok - n0;
+    return left >= block_n ? block_n : ((left + 31) & ~31);
+}
+
 template <int BLOCK_N, int STAGES>
 struct SparsePairCfg {
     static constexpr int kHalfN = BLOCK_N / 2;
@@ -428,7 +438,8 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 const int m_pair = tile % num_m, n_blk = tile / num_m;
                 const int mb = m_pair * 2 + static_cast<int>(cta);           // this CTA's 128-row block
                 const int mb_e = mb < num_mb ? mb : num_mb - 1;              // rows past M: any valid metadata block
-                const int n_row0 = n_blk * BLOCK_N + static_cast<int>(cta) * Cfg::kHalfN;
+                const int width = token_tile_width(p.Ntok, n_blk * BLOCK_N, BLOCK_N);
+                const int n_row0 = n_blk * BLOCK_N + static_cast<int>(cta) * (width / 2);
                 for (int kb = 0; kb < total_kb; ++kb) {
                     if (!mbar_wait(&empty_bar[ps.stage], ps.phase ^ 1u, abort_flag)) { ok = false; break; }
                     uint8_t* sA = smem + ps.stage * Cfg::kStageBytes;
@@ -459,12 +470,13 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
         if (cta == 0 && elect_one()) {
-            constexpr uint32_t idesc_sp = make_idesc_bf16(2 * kBlockM, BLOCK_N, false, false, true);
-            const uint32_t idesc_ad = make_idesc_bf16(2 * kBlockM, BLOCK_N, p.a2_mn_major != 0, false, false);
             PipeState ps;
             bool ok = true;
             int it = 0;
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
+                const int width = token_tile_width(p.Ntok, (tile / num_m) * BLOCK_N, BLOCK_N);
+                const uint32_t idesc_sp = make_idesc_bf16(2 * kBlockM, width, false, false, true);
+                const uint32_t idesc_ad = make_idesc_bf16(2 * kBlockM, width, p.a2_mn_major != 0, false, false);
                 const int acc = it & 1;
                 const uint32_t acc_phase = static_cast<uint32_t>(it >> 1) & 1u;
                 if (!mbar_wait(&tempty_bar[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -525,8 +537,9 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             tc_fence_after_sync();
             const uint32_t t_row = tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
             const int m0 = (m_pair * 2 + static_cast<int>(cta)) * kBlockM + q * 32;
+            const int width = token_tile_width(p.Ntok, n_blk * BLOCK_N, BLOCK_N);
 #pragma unroll 1
-            for (int c0 = half * Cfg::kStoreRows; c0 < BLOCK_N; c0 += 2 * Cfg::kStoreRows) {
+            for (int c0 = half * Cfg::kStoreRows; c0 < width; c0 += 2 * Cfg::kStoreRows) {
                 uint32_t v0[16], v1[16];
                 tmem_ld_16(t_row + c0, v0);
                 tmem_ld_16(t_row + c0 + 16, v1);
@@ -911,13 +924,17 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 bool first, next_first = false;
                 quad_tile(tile, num_m, num_n, group_m, mt, n_blk, first);
                 const int nsub = (4 * mt + 2 < num_mb) ? 2 : 1;              // second sub-tile may lie past M
-                const int n_row0 = n_blk * BLOCK_N + static_cast<int>(cta) * Cfg::kHalfN;
+                const int width = token_tile_width(p.Ntok, n_blk * BLOCK_N, BLOCK_N);
+                const int n_row0 = n_blk * BLOCK_N + static_cast<int>(cta) * (width / 2);
                 // The pairs working on the same token block (same n_blk, different mt) run side by
                 // side and would all wait on the same first-touch DRAM fetch of an activation box.
                 // One of them (mt == 0) pulls the boxes into L2 kPrefetchAhead k-blocks early.
                 const int next_tile = tile + num_pairs;
                 if (next_tile < num_tiles) quad_tile(next_tile, num_m, num_n, group_m, next_mt, next_n_blk, next_first);
-                const int next_row0 = next_first ? next_n_blk * BLOCK_N + static_cast<int>(cta) * Cfg::kHalfN : 0;
+                const int next_row0 =
+                    next_first ? next_n_blk * BLOCK_N +
+                                     static_cast<int>(cta) * (token_tile_width(p.Ntok, next_n_blk * BLOCK_N, BLOCK_N) / 2)
+                               : 0;
                 for (int kb = 0; kb < total_kb; ++kb) {
                     if (kb < num_kb) {
                         const int pk = kb + kPrefetchAhead;
@@ -971,8 +988,7 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
         if (cta == 0 && elect_one()) {
-            constexpr uint32_t idesc_sp = make_idesc_bf16(2 * kBlockM, BLOCK_N, false, false, true);
-            const uint32_t idesc_ad = make_idesc_bf16(2 * kBlockM, BLOCK_N, p.a2_mn_major != 0, false, false);
+            uint32_t idesc_sp = 0, idesc_ad = 0;              // set per tile: N is the tile's width
             // the MMAs of sub-tile s for k-block kb out of pipeline stage `stage`
             auto issue = [&](int s, int kb, int stage) {
                 const uint32_t st = smem_u32(smem + stage * Cfg::kStageBytes);
@@ -1007,10 +1023,13 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             bool ok = true;
             int it = 0;
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
-                int mt, n_blk_unused;
+                int mt, n_blk;
                 bool first_unused;
-                quad_tile(tile, num_m, num_n, group_m, mt, n_blk_unused, first_unused);
+                quad_tile(tile, num_m, num_n, group_m, mt, n_blk, first_unused);
                 const int nsub = (4 * mt + 2 < num_mb) ? 2 : 1;
+                const int width = token_tile_width(p.Ntok, n_blk * BLOCK_N, BLOCK_N);
+                idesc_sp = make_idesc_bf16(2 * kBlockM, width, false, false, true);
+                idesc_ad = make_idesc_bf16(2 * kBlockM, width, p.a2_mn_major != 0, false, false);
                 const uint32_t acc_parity = (static_cast<uint32_t>(it) & 1u) ^ 1u;
                 if (!mbar_wait(&tempty_bar[0], acc_parity, abort_flag)) { ok = false; break; }
                 tc_fence_after_sync();
@@ -1077,6 +1096,7 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             bool first_unused;
             quad_tile(tile, num_m, num_n, group_m, mt, n_blk, first_unused);
             const int nsub = (4 * mt + 2 < num_mb) ? 2 : 1;
+            const int width = token_tile_width(p.Ntok, n_blk * BLOCK_N, BLOCK_N);
             uint32_t pk[2][kMyBlocks][16];
             // ---- first accumulator (its drain is what the next tile's first MMA waits for).  Two
             //      16-column loads in flight per wait: the warps of a 320-thread CTA are allocated
@@ -1089,7 +1109,7 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 #pragma unroll
                 for (int j = 0; j < kMyBlocks; ++j) {
                     const int c0 = (2 * j + half) * Cfg::kStoreRows;
-                    if (c0 < BLOCK_N) {
+                    if (c0 < width) {
                         uint32_t v0[16], v1[16];
                         tmem_ld_16(t_row + c0, v0);
                         tmem_ld_16(t_row + c0 + 16, v1);
@@ -1113,7 +1133,7 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 #pragma unroll
                 for (int j = 0; j < kMyBlocks; ++j) {
                     const int c0 = (2 * j + half) * Cfg::kStoreRows;
-                    if (c0 < BLOCK_N) {
+                    if (c0 < width) {
                         uint32_t v0[16], v1[16];
                         tmem_ld_16(t_row + c0, v0);
                         tmem_ld_16(t_row + c0 + 16, v1);
@@ -1136,7 +1156,7 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 #pragma unroll
                     for (int j = 0; j < kMyBlocks; ++j) {
                         const int c0 = (2 * j + half) * Cfg::kStoreRows;
-                        if (c0 < BLOCK_N) {
+                        if (c0 < width) {
                             // the staging buffer about to be overwritten must have been read by its TMA store
                             if (lane == 0) tma_store_wait_read<1>();
                             __syncwarp();

@@ -504,14 +504,27 @@ static slope_status_t launch_skinny(const void* act, int ntok, const void* vals,
 //              of work); it stages the weights for fewer tokens, which costs 12 % more time
 //              per unit of work at short reductions and 30-35 % at long ones (measured at 2048
 //              tokens).
-// The choice compares rounds of the machine (tiles / CTA pairs, rounded up) times the relative
+// The choice compares waves of the machine (tiles / CTA pairs, rounded up) times the relative
 // cost of a tile.
 enum class SparseTile { kQuad224, kPair224, kPair128 };
 
 static SparseTile choose_sparse_tile(int M, int K, int ntok, int num_pairs) {
+    // Waves of full tiles; the ragged last token tile of every row tile runs at its own width
+    // (its weight loads do not shrink, its epilogue does: measured, a 32-token tile costs 0.7-0.9
+    // of a 224-token one at reductions of 4096 and more, about 0.4 at 1024) and comes last in tile
+    // order, so it first fills the pairs that the last wave of full tiles leaves idle.
     const auto rounds = [&](int rows, int block_n) {
-        const int tiles = ((M + rows - 1) / rows) * ((ntok + block_n - 1) / block_n);
-        return static_cast<double>((tiles + num_pairs - 1) / num_pairs);
+        const int num_m = (M + rows - 1) / rows;
+        const int full = num_m * (ntok / block_n), ragged = ntok % block_n;
+        const int rem = full % num_pairs;
+        double t = full / num_pairs + (rem ? 1.0 : 0.0);
+        if (ragged) {
+            const double width = ((ragged + 31) & ~31) / static_cast<double>(block_n);
+            const int left = num_m - (rem ? num_pairs - rem : 0);
+            const double floor = K >= 4096 ? 0.8 : K >= 2048 ? 0.65 : 0.45;
+            if (left > 0) t += ((left + num_pairs - 1) / num_pairs) * (width > floor ? width : floor);
+        }
+        return t;
     };
     const double gain = K >= 8192 ? 0.14 : K >= 4096 ? 0.06 : K >= 2048 ? -0.05 : -0.25;
     const double cost_pair = rounds(256, kPairBlockN);
