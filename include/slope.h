@@ -8,8 +8,10 @@
  *
  * Common rules
  *  - Every pointer is DEVICE memory owned by the caller unless a comment says
- *    "host".  The library allocates no device memory.  Base pointers must be
- *    16-byte aligned.  Matrices are dense, row-major, contiguous.
+ *    "host".  The library allocates no device memory (on the host each calling
+ *    thread keeps a small table of tensor-map encodings it has already made).
+ *    Base pointers must be 16-byte aligned.  Matrices are dense, row-major,
+ *    contiguous.
  *  - bf16 = the upper 16 bits of an IEEE fp32.  GEMMs accumulate in fp32 and
  *    round once (nearest-even) to bf16.
  *  - `stream` is a cudaStream_t (NULL = the legacy default stream).  Calls are
