@@ -804,7 +804,7 @@ slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY, c
         if (b <= kSkinnyMaxTokens)            // few tokens: split d_in over a cluster instead of one CTA
             return launch_skinny(nullptr, b, nullptr, nullptr, r, 0, X, L, d_in, true, T, stream, info);
         return adapter_narrow_tiles(b, r, info)
-                   ? launch_dense<false, true, 64, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info)
+                   ? launch_dense<false, true, 64, kEpiStore, 9>(X, L, b, r, d_in, 1, T, nullptr, stream, info)
                    : launch_dense<false, true, 128, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info);
     }
     if (!X || !dY || !R || !T || !dT || !dL || !dR || !workspace) return SLOPE_ERR_INVALID_ARG;
@@ -818,7 +818,7 @@ slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY, c
     st = b <= kSkinnyMaxTokens
              ? launch_skinny(nullptr, b, nullptr, nullptr, r, 0, dY, R, d_out, false, dT, stream, info)
          : adapter_narrow_tiles(b, r, info)
-             ? launch_dense<false, false, 64, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info)
+             ? launch_dense<false, false, 64, kEpiStore, 9>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info)
              : launch_dense<false, false, 128, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info);
     if (st) return st;
     // dL[d_in x r] = X^T dT and dR^T[d_out x r] = dY^T T: operands stored [K x M] / [K x N] with
