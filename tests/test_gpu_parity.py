@@ -540,3 +540,47 @@ def test_rows_past_the_last_token_are_never_written(B, oracle, b):
         tail = buf.view(torch.int16)[b * cols:]
         assert bool((tail == sentinel).all()), name
         assert bool(torch.isfinite(buf[: b * cols].float()).all()), name
+
+
+def test_dependent_launches_back_to_back_equal_synchronised_launches_bitwise(B, oracle):
+    """Every GEMM launch may start its set-up under the previous kernel's tail (programmatic
+    dependent launch).  A chain in which each call consumes what the previous one wrote -- three
+    layers feeding one another forward, then backward, adapters included -- must give the same bits
+    whether the host synchronises after every call or never."""
+    import torch
+
+    dims = [384, 640, 256, 512]                      # layer i: dims[i] -> dims[i + 1]
+    b, r = 776, 32
+    layers, Ls, Rs = [], [], []
+    for i in range(3):
+        layers.append(GpuLayer(si.gaussian_bf16((dims[i + 1], dims[i]), 0.05, 9600 + i)))
+        Ls.append(dev(B, si.gaussian_bf16((dims[i], r), 0.05, 9610 + i)))
+        Rs.append(dev(B, si.gaussian_bf16((r, dims[i + 1]), 0.05, 9620 + i)))
+    X0 = dev(B, si.gaussian_bf16((b, dims[0]), 1.0, 9630))
+    dYlast = dev(B, si.gaussian_bf16((b, dims[3]), 1.0, 9631))
+
+    def run(sync):
+        def s():
+            if sync:
+                torch.cuda.synchronize()
+        acts, Ts = [X0], []
+        for i, lay in enumerate(layers):
+            T = lay.adapter_T(acts[-1], Ls[i]); s()
+            Ts.append(T)
+            acts.append(lay.fwd(acts[-1], T, Rs[i])); s()
+        grads, dY = [], dYlast
+        for i in reversed(range(3)):
+            dT, dL, dR = layers[i].adapter_bwd(acts[i], dY, Ls[i], Rs[i], Ts[i]); s()
+            dX = layers[i].dx(dY, dT, Ls[i]); s()
+            dWc = layers[i].dw(dY, acts[i]); s()
+            grads += [dL, dR, dWc]
+            dY = dX
+        torch.cuda.synchronize()
+        layers[0].poll()
+        return [t.clone() for t in acts[1:] + grads + [dY]]
+
+    ref = run(sync=True)
+    for _ in range(3):
+        got = run(sync=False)
+        for a, g in zip(ref, got):
+            assert torch.equal(a.view(torch.int16), g.view(torch.int16))
