@@ -172,30 +172,39 @@ def run_layer(B, s: LayerState, rec=None):
 
 
 def cpu_baseline_sample(wl, seconds_hint=15.0):
-    """Time the oracle, as it stands, on a bounded sample of the workload's first layer."""
+    """Time the oracle, as it stands, on the workload: in full where that takes about half a
+    minute at the oracle's ~0.02 TFLOP/s (the two small configurations), else on a bounded sample
+    of the first layer, with the flop-scaled extrapolation to a whole step as a separate key."""
     import oracle
 
     oracle.build()
-    lay = wl.layers[0]
-    b = wl.tokens
-    t = si.layer_tensors(wl, 0, tokens=b)
-    _, _, mask1 = oracle.prune24(t["W"])
-    _, _, mask2 = oracle.double_prune(t["W"], mask1)
-    n_rows = 1024
-    rows = si.sample_indices(b, n_rows, 1)
-    orows = si.sample_indices(lay.d_out, n_rows, 2)
-    t0 = time.perf_counter()
-    oracle.fwd_rows(t["X"], t["W"], mask1, rows, t.get("L"), t.get("R"))
-    oracle.dx_rows(t["dY"], t["W"], mask2, rows, t.get("L"), t.get("R"))
-    oracle.dw_rows(t["dY"], t["X"], mask1, orows)
-    dt = time.perf_counter() - t0
-    r = wl.rank
-    flops = (2 * len(rows) * (2.0 * lay.d_in * lay.d_out + 2.0 * r * (lay.d_in + lay.d_out))
-             + len(orows) * 2.0 * b * lay.d_in)
-    return {"value": flops / dt / 1e12, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
-            "seconds": round(dt, 2),
-            "sample": f"layer '{lay.name}' {lay.d_in}->{lay.d_out}, b={b}: fwd+dX on {len(rows)} token rows, "
-                      f"masked dW on {len(orows)} d_out rows (dense-equivalent FLOPs of the sample / wall time)"}
+    b, r = wl.tokens, wl.rank
+    step_flops = sum(6.0 * b * l.d_in * l.d_out + 6.0 * b * r * (l.d_in + l.d_out) for l in wl.layers)
+    full = step_flops / 0.02e12 <= 2.0 * seconds_hint
+    flops, dt, what = 0.0, 0.0, []
+    for li, lay in enumerate(wl.layers if full else wl.layers[:1]):
+        t = si.layer_tensors(wl, li, tokens=b)
+        _, _, mask1 = oracle.prune24(t["W"])
+        _, _, mask2 = oracle.double_prune(t["W"], mask1)
+        rows = np.arange(b) if full else si.sample_indices(b, 1024, 1)
+        orows = np.arange(lay.d_out) if full else si.sample_indices(lay.d_out, 1024, 2)
+        t0 = time.perf_counter()
+        oracle.fwd_rows(t["X"], t["W"], mask1, rows, t.get("L"), t.get("R"))
+        oracle.dx_rows(t["dY"], t["W"], mask2, rows, t.get("L"), t.get("R"))
+        oracle.dw_rows(t["dY"], t["X"], mask1, orows)
+        dt += time.perf_counter() - t0
+        flops += (2 * len(rows) * (2.0 * lay.d_in * lay.d_out + 2.0 * r * (lay.d_in + lay.d_out))
+                  + len(orows) * 2.0 * b * lay.d_in)
+        what.append(f"layer '{lay.name}' {lay.d_in}->{lay.d_out}, b={b}: fwd+dX on {len(rows)} token rows, "
+                    f"masked dW on {len(orows)} d_out rows")
+    value = flops / dt / 1e12
+    return {"value": value, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle", "seconds": round(dt, 2),
+            "sample": ("the whole workload: " if full else "bounded sample: ") + "; ".join(what) +
+                      " (dense-equivalent FLOPs of what was computed / wall time)",
+            "full_workload": full,
+            "extrapolated_step_seconds": round(step_flops / (value * 1e12), 1),
+            "extrapolation": "flop-scaled: dense-equivalent FLOPs of one step (fwd + dX + dW + adapter terms of every layer) "
+                             "/ the measured rate; equals the measured time when the whole workload was run"}
 
 
 def run_reference(args, rank):
