@@ -392,8 +392,12 @@ def main():
         if fl:
             tot[op][0] += fl
             tot[op][1] += ms * 1e-3
+            tf = fl / (ms * 1e-3) / 1e12
+            peak = pk["bf16_sustained"] if op == "linear_bwd_dw_masked" else sparse_peak
             stage_rows.append({"layer": name, "d_in": d_in, "d_out": d_out, "op": op, "ms": round(ms, 4),
-                               "tflops_dense_eq": round(fl / (ms * 1e-3) / 1e12, 1)})
+                               "tflops_dense_eq": round(tf, 1),
+                               "tflops_executed": round(tf if op == "linear_bwd_dw_masked" else tf / 2, 1),
+                               "frac_of_sustained_peak": round(tf / peak, 4)})
         elif op in ("prune_24", "double_prune") and (d_in, d_out, op) not in seen:
             seen.add((d_in, d_out, op))
             bytes_ = d_in * d_out * (3.25 if op == "prune_24" else 3.25)   # double prune: 2 + 0.125 in, 1 + 0.125 out
