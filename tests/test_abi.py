@@ -51,6 +51,18 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     assert lib.slope_linear_fwd(p, 16, p, p, 128, 128, null, null, 24, p, null) == 1   # rank without factors
     assert lib.slope_adapter_fwd_bwd(7, p, p, p, p, 16, 128, 128, 16, p, p, p, p, p, 0, null) == 1
     assert lib.slope_status_string(6) == b"device-side wait timed out"
+    # one of every kind of refusal, all before any CUDA call
+    a = (ctypes.addressof(buf) + 15) & ~15                                            # 16-byte aligned host address
+    assert lib.slope_linear_fwd(a, 16, a, a, 128, 128, a, a, 24, a, null) == 2         # rank not a multiple of 16
+    assert lib.slope_linear_fwd(a + 2, 16, a, a, 128, 128, null, null, 0, a, null) == 3  # misaligned pointer
+    assert lib.slope_linear_fwd(a, 16, a, a, 128, 100, null, null, 0, a, null) == 2    # d_in not a multiple of 128
+    assert lib.slope_adapter_fwd_bwd(1, a, a, a, a, 16, 128, 128, 16, a, a, a, a, a, 0, null) == 1   # workspace too small
+    assert lib.slope_adapter_fwd_bwd(0, a, a, a, a, 16, 128, 128, 0, a, a, a, a, a, 0, null) == 2    # adapter call without a rank
+    assert lib.slope_linear_bwd_dw_masked(a, a, 16, 128, 128, null, a, null) == 1      # mask is not optional
+    assert lib.slope_prune_nm(a, 128, 128, 2, 3, a, null, null) == 2                   # group size not 2, 4, 8, 16
+    assert lib.slope_prune_nm(a, 128, 128, 4, 4, a, null, null) == 2                   # n must be below m
+    assert lib.slope_sparse_add(a, a, 1.0, 1.0, 128, 100, a, null) == 2
+    assert lib.slope_update_sparse_matrix(a, a, a, 128, 128, null, null) == 1
 
 
 def test_binding_refuses_to_run_without_the_library(monkeypatch, tmp_path):
