@@ -72,3 +72,34 @@ def test_binding_refuses_to_run_without_the_library(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "_LIB_PATH", tmp_path / "libslope.so")
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         binding.lib()
+
+
+def test_format_sizes_against_the_papers_memory_accounting(lib):
+    """The size functions of the compressed format, per group of four weights, next to the bit counts the
+    paper prints: its sparse model holds 2 x (2 x 16 + 3) weight bits, 4 x 8 mask bits, 2 x 16 gradient bits
+    and 2 x 2 x 32 optimizer bits per group (ratio 0.68 of dense); inference 35 of 64 bits (0.54)."""
+    import math
+    import os
+
+    golden = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "memory_accounting.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].split()
+            if len(line) == 2:
+                golden[line[0]] = float(line[1])
+    # the paper's own arithmetic reproduces its printed ratios
+    assert golden["index_bits_per_group"] == math.ceil(math.log2(math.comb(4, 2)))
+    paper_sparse = 2 * (2 * 16 + 3) + 4 * 8 + 2 * 16 + 2 * 2 * 32
+    assert golden["dense_training_bits"] == 4 * 16 + 4 * 16 + 2 * 4 * 32
+    assert abs(paper_sparse / golden["dense_training_bits"] - golden["sparse_training_ratio"]) < 5e-3
+    assert golden["sparse_inference_bits"] == 2 * 16 + 3
+    assert abs(golden["sparse_inference_bits"] / golden["dense_inference_bits"] - golden["sparse_inference_ratio"]) < 1e-2
+    # this library's format: 4-bit codes (2 bits per kept value, what the tensor cores read) and 1-bit masks
+    rows, cols = 4096, 11008
+    groups = rows * cols // 4
+    copy_bits = 8 * (lib.slope_values_bytes(rows, cols) + lib.slope_meta_bytes(rows, cols)) / groups
+    mask_bits = 8 * lib.slope_mask_bytes(rows, cols) / groups
+    assert copy_bits == 2 * 16 + 4 and mask_bits == 4
+    ours_training = 2 * copy_bits + mask_bits + 2 * 16 + 2 * 2 * 32
+    assert ours_training == 236 and ours_training < paper_sparse
+    assert abs(copy_bits / golden["dense_inference_bits"] - 0.5625) < 1e-12          # one bit per group above the paper's count
