@@ -723,24 +723,33 @@ def inference_forward_probe(torch, B, wl, pk, copies=12, reps=5):
 
                     def run():
                         for v, m in Wc:
+                            B.slope_linear_fwd_adapter(X, v, m, d_out, L, R, T, Y)
+
+                    def run_two_calls():
+                        for v, m in Wc:
                             B.slope_adapter_fwd_bwd(0, X, None, L, None, b, d_out, d_in, r, T=T)
                             B.slope_linear_fwd(X, v, m, d_out, Y, T, R)
+                    us_two = time_graph(run_two_calls)
                 else:
                     def run():
                         for v, m in Wc:
                             B.slope_linear_fwd(X, v, m, d_out, Y)
+                    us_two = None
                 us = time_graph(run)
                 nbytes = d_in * d_out * 1.125 + 2.0 * b * (d_in + d_out) + 2.0 * r * (d_in + d_out) + 4.0 * b * r
                 gbs = nbytes / (us * 1e-6) / 1e9
                 rows.append({"d_in": d_in, "d_out": d_out, "tokens": b, "rank": r, "us": round(us, 2),
                              "algorithmic_bytes": int(nbytes), "gbs": round(gbs, 1),
                              "frac_of_hbm_peak": round(gbs / pk["hbm_gbs"], 4),
-                             "cublas_dense_us": round(us_dense, 2), "speedup_vs_cublas_dense": round(us_dense / us, 3)})
+                             "cublas_dense_us": round(us_dense, 2), "speedup_vs_cublas_dense": round(us_dense / us, 3),
+                             "separate_adapter_call_us": None if us_two is None else round(us_two, 2)})
         del Wc, Wd
     st = B.slope_poll_status()
     if st != 0:
         raise SystemExit(f"device status after the inference probe: {B.slope_status_string(st)}")
-    return {"what": f"forward only (adapter T = X L + fused sparse GEMM), CUDA graph of {copies} calls over distinct "
+    return {"what": f"forward only (with adapters: slope_linear_fwd_adapter, T = X L and the sparse GEMM with the fused "
+                    f"T R term as an overlapped pair of launches; separate_adapter_call_us = slope_adapter_fwd_bwd(0) "
+                    f"then slope_linear_fwd), CUDA graph of {copies} calls over distinct "
                     f"weight copies, best of {reps} replays, us per call; bytes: 1.125 B per weight element "
                     f"(values + metadata) + activations + adapter factors; HBM peak {pk['hbm_gbs']} GB/s "
                     f"({pk['src']}); cuBLAS reads the dense bf16 weight (2 B per element, no adapter)",

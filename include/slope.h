@@ -104,6 +104,22 @@ slope_status_t slope_linear_fwd(const void* X, int b, const void* Wc_vals, const
                                 void* Y, void* stream);
 
 /*
+ * The forward with its lazy adapter in one call, Eq. (concat):
+ *   T[b x r] = X L,   Y[b x d_out] = X (W^R)^T + T R      (L[d_in x r], R[r x d_out], r > 0).
+ * Same results, bit for bit, as slope_adapter_fwd_bwd(phase 0) followed by slope_linear_fwd.
+ * T is caller-owned scratch that holds X L afterwards.  At inference sizes (where the few-token
+ * kernel serves the forward) the two launches are issued as a fused pair: the forward streams
+ * its weights and runs its sparse reduction while T is still being computed and waits only for
+ * T itself, which takes the adapter's extra launch off the critical path (Sec. "Efficient
+ * inference": the adapter multiplications are what limits the inference speedup).  With more
+ * tokens it issues the same two launches as the separate calls.  The stream must not receive
+ * work from another host thread while the call runs.
+ */
+slope_status_t slope_linear_fwd_adapter(const void* X, int b, const void* Wc_vals, const void* Wc_meta,
+                                        int d_out, int d_in, const void* L, const void* R, int r,
+                                        void* T, void* Y, void* stream);
+
+/*
  * Input gradient, Eq. (sparse_backward_input), with the double-pruned weight:
  *   dX[b x d_in] = dY[b x d_out] W^{R,C}  (+ dT[b x r] L^T, L[d_in x r]).
  * WTc_vals / WTc_meta come from slope_double_prune.  dT = dY R^T is produced by

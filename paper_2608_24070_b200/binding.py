@@ -31,6 +31,7 @@ EXPORTS = (
     "slope_sparse_add", "slope_update_sparse_matrix", "slope_selftest_wait_timeout",
     "slope_prune_nm", "slope_double_prune_nm", "slope_apply_mask",
     "slope_dense_linear_fwd", "slope_dense_linear_bwd_dx", "slope_dense_linear_bwd_dw", "slope_mask_difference",
+    "slope_linear_fwd_adapter",
 )
 
 
@@ -56,6 +57,8 @@ def lib() -> ctypes.CDLL:
         L.slope_double_prune.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp]
         L.slope_linear_fwd.argtypes = [vp, ci, vp, vp, ci, ci, vp, vp, ci, vp, vp]
         L.slope_linear_bwd_dx.argtypes = [vp, ci, vp, vp, ci, ci, vp, vp, ci, vp, vp]
+        L.slope_linear_fwd_adapter.argtypes = [vp, ci, vp, vp, ci, ci, vp, vp, ci, vp, vp, vp]
+        L.slope_linear_fwd_adapter.restype = ci
         L.slope_linear_bwd_dw_masked.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp]
         L.slope_adapter_workspace_bytes.restype = sz
         L.slope_adapter_workspace_bytes.argtypes = [ci, ci, ci, ci]
@@ -149,6 +152,14 @@ def slope_linear_fwd(X, Wc_vals, Wc_meta, d_out, Y, T=None, R=None):
     r = 0 if T is None else T.shape[1]
     _check("slope_linear_fwd", lib().slope_linear_fwd(_ptr(X), b, _ptr(Wc_vals), _ptr(Wc_meta), d_out, d_in,
                                                       _ptr(T), _ptr(R), r, _ptr(Y), _stream()))
+
+
+def slope_linear_fwd_adapter(X, Wc_vals, Wc_meta, d_out, L, R, T, Y):
+    """T = X L and Y = X (W^R)^T + T R in one call (a fused pair of launches at inference sizes)."""
+    b, d_in = X.shape
+    _check("slope_linear_fwd_adapter", lib().slope_linear_fwd_adapter(
+        _ptr(X), b, _ptr(Wc_vals), _ptr(Wc_meta), d_out, d_in, _ptr(L), _ptr(R), L.shape[1], _ptr(T), _ptr(Y),
+        _stream()))
 
 
 def slope_linear_bwd_dx(dY, WTc_vals, WTc_meta, d_in, dX, dT=None, L=None):

@@ -55,6 +55,7 @@ struct SparseGemmParams {
     int M, K, Ntok, r;
     int a2_mn_major;              // 1: A2 is stored [r x M] (M contiguous)
     int group_m;                  // 512-row-tile kernel: row tiles per raster group (0: all in one group)
+    int pdl_mode;                 // few-token kernel: 0 plain, 1 producer / 2 consumer of a fused pair of launches
     const uint8_t* meta;          // metadata blocks of A
     uint16_t* out;                // [Ntok x M]
 };
@@ -1284,18 +1285,31 @@ sparse_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
     // thing is safe earlier: asking L2 to fetch this CTA's first weight tiles.  A prefetch moves no
     // data into the SM, and L2 is the point of coherence, so a line the previous kernel is still
     // writing stays correct; the first loads after the wait then come at L2 instead of HBM latency.
-    griddep_launch_dependents();
-    if (warp == 0 && elect_one()) {
-        // (a short K-slice gains nothing: its few tiles are requested at once after the wait, and the
-        // prefetch requests would only sit in front of them in the TMA queue)
-        const int n_pf = num_sb >= 8 ? kSkinnyPrefetchBlocks : 0;
-        for (int i = 0; i < n_pf; ++i) {
-            tma_prefetch_l2_2d(&tmA, (kb0 + i) * 64, m_blk * kBlockM);
-            tma_prefetch_l2_2d(&tmE, 0, m_blk * num_kb + kb0 + i);
+    //
+    // Two launches issued together by one call (T = X L, then the forward that adds T R) use the
+    // dependency more finely.  The producer (pdl_mode 1) waits first and releases its dependents
+    // afterwards: when the consumer starts, everything that preceded the pair in the stream is
+    // complete.  The consumer (pdl_mode 2) therefore streams its weights and activations and runs
+    // its whole sparse reduction without waiting; only the thread that loads the producer's
+    // output T waits, right before the first such load.  Everything that follows in the consumer
+    // (the adapter MMAs, the cluster reduction, the stores) is ordered behind that load.
+    if (p.pdl_mode == 1) {
+        griddep_wait();
+        griddep_launch_dependents();
+    } else {
+        griddep_launch_dependents();
+        if (warp == 0 && elect_one()) {
+            // (a short K-slice gains nothing: its few tiles are requested at once after the wait, and the
+            // prefetch requests would only sit in front of them in the TMA queue)
+            const int n_pf = num_sb >= 8 && p.pdl_mode == 0 ? kSkinnyPrefetchBlocks : 0;
+            for (int i = 0; i < n_pf; ++i) {
+                tma_prefetch_l2_2d(&tmA, (kb0 + i) * 64, m_blk * kBlockM);
+                tma_prefetch_l2_2d(&tmE, 0, m_blk * num_kb + kb0 + i);
+            }
         }
+        __syncwarp();
+        if (p.pdl_mode != 2) griddep_wait();
     }
-    __syncwarp();
-    griddep_wait();
 
     if (warp == 0) {
         // ---------------------------------------------------------- weight ring (values + metadata)
@@ -1378,6 +1392,7 @@ sparse_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_
                     tma_load_2d(sB, &tmB, bar, kb * 128, 0);
                     tma_load_2d(sB + BLOCK_N * 128, &tmB, bar, kb * 128 + 64, 0);
                 } else {
+                    if (p.pdl_mode == 2 && i == num_sb) griddep_wait();      // T comes from the launch before this one
                     mbar_expect_tx(bar, BLOCK_N * 128);
                     tma_load_2d(sB, &tmB2, bar, (ab0 + i - num_sb) * 64, 0);
                 }

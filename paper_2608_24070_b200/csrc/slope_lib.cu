@@ -440,7 +440,7 @@ static bool skinny_capacity(const DeviceInfo& info, int (&cap)[9]) {
 template <int BLOCK_N, int A_STAGES, int B_STAGES>
 static slope_status_t launch_sparse_skinny(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                            const void* act2, const void* fac2, int r, bool a2_mn, void* out,
-                                           cudaStream_t stream, const DeviceInfo& info) {
+                                           cudaStream_t stream, const DeviceInfo& info, int pdl_mode) {
     using Cfg = SparseSkinnyCfg<BLOCK_N, A_STAGES, B_STAGES>;
     CUtensorMap tmA, tmB, tmE, tmA2, tmB2;
     if (r > 0) {
@@ -463,6 +463,7 @@ static slope_status_t launch_sparse_skinny(const void* act, int ntok, const void
     }
     SparseGemmParams p = {};
     p.M = M; p.K = K; p.Ntok = ntok; p.r = r; p.a2_mn_major = a2_mn ? 1 : 0;
+    p.pdl_mode = pdl_mode;
     p.meta = static_cast<const uint8_t*>(meta);
     p.out = static_cast<uint16_t*>(out);
     auto kern = sparse_gemm_skinny_kernel<BLOCK_N, A_STAGES, B_STAGES>;
@@ -470,6 +471,17 @@ static slope_status_t launch_sparse_skinny(const void* act, int ntok, const void
 
     int cap[9];
     if (!skinny_capacity<BLOCK_N, A_STAGES, B_STAGES>(info, cap)) return SLOPE_ERR_CUDA;
+    if (pdl_mode == 2) {
+        // The consumer of a fused pair has to be resident next to its producer (one cluster of up to 8
+        // CTAs per 128 adapter columns), or its last clusters would wait for the producer to finish
+        // and the overlap would be lost: count only the clusters that fit beside it.
+        const int reserved = 8 * ((r + kBlockM - 1) / kBlockM);
+        for (int sz = 1; sz <= 8; ++sz) {
+            cap[sz] -= (reserved + sz - 1) / sz + (sz > 1 ? 1 : 0);
+            if (cap[sz] < 0) cap[sz] = 0;
+        }
+        if (cap[1] <= 0) return SLOPE_ERR_CUDA;
+    }
     const int slabs = (M + kBlockM - 1) / kBlockM, num_kb = K > 0 ? K / 128 : (r + 63) / 64;
     const int splits = skinny_splits(slabs, num_kb, BLOCK_N, cap);
     return launch_cluster_ex(kern, slabs * splits, splits, kGemmThreads, Cfg::kSmemBytes, true, stream, tmA, tmB,
@@ -484,11 +496,14 @@ constexpr int kSkinnyMaxTokens = 256;
 
 static slope_status_t launch_skinny(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                     const void* act2, const void* fac2, int r, bool a2_mn, void* out,
-                                    cudaStream_t stream, const DeviceInfo& info) {
-    if (ntok <= 16) return launch_sparse_skinny<16, 10, 4>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
-    if (ntok <= 64) return launch_sparse_skinny<64, 8, 4>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
-    if (ntok <= 128) return launch_sparse_skinny<128, 7, 3>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
-    return launch_sparse_skinny<256, 5, 2>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
+                                    cudaStream_t stream, const DeviceInfo& info, int pdl_mode = 0) {
+    if (ntok <= 16)
+        return launch_sparse_skinny<16, 10, 4>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info, pdl_mode);
+    if (ntok <= 64)
+        return launch_sparse_skinny<64, 8, 4>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info, pdl_mode);
+    if (ntok <= 128)
+        return launch_sparse_skinny<128, 7, 3>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info, pdl_mode);
+    return launch_sparse_skinny<256, 5, 2>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info, pdl_mode);
 }
 
 // Kernel choice for the sparse GEMMs.  Up to 256 tokens the GEMM is a weight stream from HBM and
@@ -694,6 +709,38 @@ slope_status_t slope_linear_fwd(const void* X, int b, const void* Wc_vals, const
     if (slope_status_t st = check_arch(info)) return st;
     return launch_sparse_gemm(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R, r, /*a2_mn=*/true, Y,
                               static_cast<cudaStream_t>(stream), info);
+}
+
+static bool adapter_narrow_tiles(int b, int r, const DeviceInfo& info);
+
+slope_status_t slope_linear_fwd_adapter(const void* X, int b, const void* Wc_vals, const void* Wc_meta, int d_out,
+                                        int d_in, const void* L, const void* R, int r, void* T, void* Y,
+                                        void* stream_) {
+    if (!X || !Wc_vals || !Wc_meta || !L || !R || !T || !Y) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(d_out, d_in) || b < 1 || !rank_ok(r) || r == 0) return SLOPE_ERR_SHAPE;
+    if (!aligned16(X) || !aligned16(Wc_vals) || !aligned16(Wc_meta) || !aligned16(L) || !aligned16(R) ||
+        !aligned16(T) || !aligned16(Y))
+        return SLOPE_ERR_ALIGNMENT;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (use_few_token_kernel(d_out, d_in, b, r, info)) {
+        // Two launches of the few-token kernel as a fused pair: T = X L releases its dependent only
+        // once everything before it in the stream is complete, so the forward streams its weights
+        // and runs its sparse reduction while T is still being computed, and waits only for T.
+        if (slope_status_t st = launch_skinny(nullptr, b, nullptr, nullptr, r, 0, X, L, d_in, true, T, stream, info, 1))
+            return st;
+        return launch_skinny(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R, r, true, Y, stream, info, 2);
+    }
+    slope_status_t st;
+    if (b <= kSkinnyMaxTokens)
+        st = launch_skinny(nullptr, b, nullptr, nullptr, r, 0, X, L, d_in, true, T, stream, info);
+    else
+        st = adapter_narrow_tiles(b, r, info)
+                 ? launch_dense<false, true, 64, kEpiStore, 9>(X, L, b, r, d_in, 1, T, nullptr, stream, info)
+                 : launch_dense<false, true, 128, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info);
+    if (st) return st;
+    return launch_sparse_gemm(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R, r, /*a2_mn=*/true, Y, stream, info);
 }
 
 slope_status_t slope_linear_bwd_dx(const void* dY, int b, const void* WTc_vals, const void* WTc_meta, int d_out,

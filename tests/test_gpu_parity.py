@@ -584,3 +584,76 @@ def test_dependent_launches_back_to_back_equal_synchronised_launches_bitwise(B, 
         got = run(sync=False)
         for a, g in zip(ref, got):
             assert torch.equal(a.view(torch.int16), g.view(torch.int16))
+
+
+@pytest.mark.parametrize("d_in,d_out,b,r", [(1024, 512, 1, 16), (4096, 512, 8, 64), (512, 1536, 16, 128),
+                                            (2048, 256, 40, 64), (1152, 384, 104, 256), (1024, 512, 16, 256),
+                                            (384, 640, 776, 32)])
+def test_forward_with_adapter_in_one_call_equals_the_two_calls_bitwise(B, oracle, d_in, d_out, b, r):
+    """slope_linear_fwd_adapter: at inference sizes a fused pair of launches (the forward runs its
+    sparse reduction while T is still being computed), with many tokens the plain two launches.
+    Same kernels, same order of additions: the same bits as the separate calls, and the oracle's values."""
+    import torch
+
+    seed = 9700 + b + r
+    W = si.gaussian_bf16((d_out, d_in), 0.02, seed)
+    X = si.gaussian_bf16((b, d_in), 1.0, seed + 1)
+    L = si.gaussian_bf16((d_in, r), 0.01, seed + 2)
+    R = si.gaussian_bf16((r, d_out), 0.01, seed + 3)
+    layer = GpuLayer(W)
+    Xd, Ld, Rd = dev(B, X), dev(B, L), dev(B, R)
+    T_ref = layer.adapter_T(Xd, Ld)
+    Y_ref = layer.fwd(Xd, T_ref, Rd)
+    layer.poll()
+    for _ in range(3):                                            # repeated: a race would not repeat its bits
+        T = torch.full((b, r), float("nan"), dtype=torch.bfloat16, device="cuda")
+        Y = torch.full((b, d_out), float("nan"), dtype=torch.bfloat16, device="cuda")
+        B.slope_linear_fwd_adapter(Xd, layer.Wc_vals, layer.Wc_meta, d_out, Ld, Rd, T, Y)
+        layer.poll()
+        assert torch.equal(T.view(torch.int16), T_ref.view(torch.int16))
+        assert torch.equal(Y.view(torch.int16), Y_ref.view(torch.int16))
+    _, _, mask1 = oracle.prune24(W)
+    err = rel_fro(to_f64(B.bits_from_bf16(Y)), oracle.fwd_rows(X, W, mask1, np.arange(b), L, R))
+    assert err <= REL_TOL, err
+
+
+def test_chain_of_fused_adapter_forwards_in_a_cuda_graph(B, oracle):
+    """Four decode-size layers, each through the one-call forward, each fed by the previous one's
+    output (so every pair's first launch really has to wait for the pair before it): eager result,
+    captured graph and its replays agree bitwise with the chain of separate calls."""
+    import torch
+
+    dims, b, r = [512, 1024, 384, 640, 512], 8, 64
+    layers, Ls, Rs = [], [], []
+    for i in range(4):
+        layers.append(GpuLayer(si.gaussian_bf16((dims[i + 1], dims[i]), 0.05, 9800 + i)))
+        Ls.append(dev(B, si.gaussian_bf16((dims[i], r), 0.05, 9810 + i)))
+        Rs.append(dev(B, si.gaussian_bf16((r, dims[i + 1]), 0.05, 9820 + i)))
+    X0 = dev(B, si.gaussian_bf16((b, dims[0]), 1.0, 9830))
+    ref = X0
+    for i, lay in enumerate(layers):
+        ref = lay.fwd(ref, lay.adapter_T(ref, Ls[i]), Rs[i])
+    layers[0].poll()
+    Ts = [torch.empty((b, r), dtype=torch.bfloat16, device="cuda") for _ in range(4)]
+    acts = [X0] + [torch.empty((b, dims[i + 1]), dtype=torch.bfloat16, device="cuda") for i in range(4)]
+
+    def chain():
+        for i, lay in enumerate(layers):
+            B.slope_linear_fwd_adapter(acts[i], lay.Wc_vals, lay.Wc_meta, dims[i + 1], Ls[i], Rs[i], Ts[i], acts[i + 1])
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        chain()                                                    # eager, also warms up before capture
+        side.synchronize()
+        assert torch.equal(acts[4].view(torch.int16), ref.view(torch.int16))
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            chain()
+        for _ in range(3):
+            acts[4].zero_()
+            graph.replay()
+            side.synchronize()
+            assert torch.equal(acts[4].view(torch.int16), ref.view(torch.int16))
+    torch.cuda.current_stream().wait_stream(side)
+    layers[0].poll()
