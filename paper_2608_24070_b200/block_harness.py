@@ -80,8 +80,9 @@ class _SlopeLinearFn(torch.autograd.Function):
             nonlocal T
             if layer.r:
                 T = torch.empty(b, layer.r, dtype=torch.bfloat16, device=X.device)
-                B.slope_adapter_fwd_bwd(0, X, None, layer.L, None, b, layer.d_out, layer.d_in, layer.r, T=T)
-            B.slope_linear_fwd(X, layer.Wc_vals, layer.Wc_meta, layer.d_out, Y, T, layer.R)
+                B.slope_linear_fwd_adapter(X, layer.Wc_vals, layer.Wc_meta, layer.d_out, layer.L, layer.R, T, Y)
+            else:
+                B.slope_linear_fwd(X, layer.Wc_vals, layer.Wc_meta, layer.d_out, Y)
 
         _timed(layer.timers, run)
         ctx.layer = layer
