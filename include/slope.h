@@ -106,7 +106,9 @@ slope_status_t slope_linear_fwd(const void* X, int b, const void* Wc_vals, const
 /*
  * The forward with its lazy adapter in one call, Eq. (concat):
  *   T[b x r] = X L,   Y[b x d_out] = X (W^R)^T + T R      (L[d_in x r], R[r x d_out], r > 0).
- * Same results, bit for bit, as slope_adapter_fwd_bwd(phase 0) followed by slope_linear_fwd.
+ * The same sums as slope_adapter_fwd_bwd(phase 0) followed by slope_linear_fwd: T bit for bit; Y up
+ * to the order of fp32 partial sums (a fused pair may split the reduction differently), and
+ * deterministic like every other call.
  * T is caller-owned scratch that holds X L afterwards.  At inference sizes (where the few-token
  * kernel serves the forward) the two launches are issued as a fused pair: the forward streams
  * its weights and runs its sparse reduction while T is still being computed and waits only for

@@ -423,8 +423,10 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     const uint32_t tmem_base = *tmem_slot;
     // Programmatic dependent launch: the set-up above may overlap the tail of the previous kernel in
     // the stream; no thread touches global memory before that kernel has completed.
+    // (As the consumer of a fused pair of launches -- pdl_mode 2, see the few-token kernel -- only the
+    // producer thread waits, right before its first load of the adapter operand T.)
     griddep_launch_dependents();
-    griddep_wait();
+    if (p.pdl_mode != 2) griddep_wait();
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both CTAs)
@@ -435,6 +437,7 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             const uint64_t keep = l2_policy_evict_last();
             PipeState ps;
             bool ok = true;
+            bool waited = false;
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
                 const int m_pair = tile % num_m, n_blk = tile / num_m;
                 const int mb = m_pair * 2 + static_cast<int>(cta);           // this CTA's 128-row block
@@ -455,6 +458,10 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                         tma_load_2d_pair_hint(sE, &tmE, bar, 0, mb_e * num_kb + kb, keep);
                     } else {
                         const int ab = kb - num_kb;
+                        if (p.pdl_mode == 2 && !waited) {
+                            griddep_wait();
+                            waited = true;
+                        }
                         if (cta == 0) mbar_expect_tx(&full_bar[ps.stage], 2 * (Cfg::kABytes + Cfg::kHalfN * 128));
                         if (p.a2_mn_major) {
                             tma_load_2d_pair(sA, &tmA2, bar, mb * kBlockM, ab * 64);

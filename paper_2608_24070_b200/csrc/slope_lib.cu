@@ -299,7 +299,7 @@ constexpr int kPairNarrowStages = 5;
 template <int BLOCK_N, int STAGES>
 static slope_status_t launch_sparse_pair(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                          const void* act2, const void* fac2, int r, bool a2_mn, void* out,
-                                         cudaStream_t stream, const DeviceInfo& info) {
+                                         cudaStream_t stream, const DeviceInfo& info, int pdl_mode = 0) {
     using Cfg = SparsePairCfg<BLOCK_N, STAGES>;
     CUtensorMap tmA, tmB, tmE, tmA2, tmB2, tmO;
     if (!make_tmap(&tmA, vals, M, K / 2, kBlockM, 64)) return SLOPE_ERR_CUDA;
@@ -319,8 +319,10 @@ static slope_status_t launch_sparse_pair(const void* act, int ntok, const void* 
     p.out = static_cast<uint16_t*>(out);
     auto kern = sparse_gemm_pair_kernel<BLOCK_N, STAGES>;
     if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
+    p.pdl_mode = pdl_mode;
     const int tiles = ((M / kBlockM + 1) / 2) * ((ntok + BLOCK_N - 1) / BLOCK_N);
-    const int max_pairs = info.sm_count / 2;
+    // (the consumer of a fused pair leaves the producer's SMs alone: up to 8 CTAs per 128 adapter columns)
+    const int max_pairs = (info.sm_count - (pdl_mode == 2 ? 8 * ((r + kBlockM - 1) / kBlockM) : 0)) / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
     return launch_pairs(kern, 2 * pairs, Cfg::kThreads, Cfg::kSmemBytes, stream, tmA, tmB, tmE, tmA2, tmB2, tmO, p);
 }
@@ -733,9 +735,20 @@ slope_status_t slope_linear_fwd_adapter(const void* X, int b, const void* Wc_val
         return launch_skinny(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R, r, true, Y, stream, info, 2);
     }
     slope_status_t st;
-    if (b <= kSkinnyMaxTokens)
+    if (b <= kSkinnyMaxTokens) {
+        // a few more tokens: the 256-row tile kernel can be the consumer of such a pair as well
+        const SparseTile tile = choose_sparse_tile(d_out, d_in, b, info.sm_count / 2);
+        if (tile != SparseTile::kQuad224) {
+            st = launch_skinny(nullptr, b, nullptr, nullptr, r, 0, X, L, d_in, true, T, stream, info, 1);
+            if (st) return st;
+            return tile == SparseTile::kPair128
+                       ? launch_sparse_pair<kPairNarrowBlockN, kPairNarrowStages>(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R,
+                                                                                  r, true, Y, stream, info, 2)
+                       : launch_sparse_pair<kPairBlockN, kPairStages>(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R, r, true, Y,
+                                                                      stream, info, 2);
+        }
         st = launch_skinny(nullptr, b, nullptr, nullptr, r, 0, X, L, d_in, true, T, stream, info);
-    else
+    } else
         st = adapter_narrow_tiles(b, r, info)
                  ? launch_dense<false, true, 64, kEpiStore, 9>(X, L, b, r, d_in, 1, T, nullptr, stream, info)
                  : launch_dense<false, true, 128, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info);

@@ -588,11 +588,15 @@ def test_dependent_launches_back_to_back_equal_synchronised_launches_bitwise(B, 
 
 @pytest.mark.parametrize("d_in,d_out,b,r", [(1024, 512, 1, 16), (4096, 512, 8, 64), (512, 1536, 16, 128),
                                             (2048, 256, 40, 64), (1152, 384, 104, 256), (1024, 512, 16, 256),
-                                            (384, 640, 776, 32)])
-def test_forward_with_adapter_in_one_call_equals_the_two_calls_bitwise(B, oracle, d_in, d_out, b, r):
+                                            (1024, 2816, 64, 64), (256, 2048, 128, 32), (1024, 384, 200, 64),
+                                            (512, 5632, 250, 256), (384, 640, 776, 32)])
+def test_forward_with_adapter_in_one_call_against_the_two_calls(B, oracle, d_in, d_out, b, r):
     """slope_linear_fwd_adapter: at inference sizes a fused pair of launches (the forward runs its
     sparse reduction while T is still being computed), with many tokens the plain two launches.
-    Same kernels, same order of additions: the same bits as the separate calls, and the oracle's values."""
+    T is the same launch as in the separate call: same bits.  Y is the same sum, but the forward of
+    a fused pair picks its K-split among the clusters that fit beside the T launch, so fp32 partial
+    sums may be grouped differently: a few outputs can land on the neighbouring bf16 value.  The
+    call itself is deterministic, and a race with the T launch would not repeat its bits."""
     import torch
 
     seed = 9700 + b + r
@@ -605,13 +609,20 @@ def test_forward_with_adapter_in_one_call_equals_the_two_calls_bitwise(B, oracle
     T_ref = layer.adapter_T(Xd, Ld)
     Y_ref = layer.fwd(Xd, T_ref, Rd)
     layer.poll()
-    for _ in range(3):                                            # repeated: a race would not repeat its bits
+    first = None
+    for _ in range(3):
         T = torch.full((b, r), float("nan"), dtype=torch.bfloat16, device="cuda")
         Y = torch.full((b, d_out), float("nan"), dtype=torch.bfloat16, device="cuda")
         B.slope_linear_fwd_adapter(Xd, layer.Wc_vals, layer.Wc_meta, d_out, Ld, Rd, T, Y)
         layer.poll()
         assert torch.equal(T.view(torch.int16), T_ref.view(torch.int16))
-        assert torch.equal(Y.view(torch.int16), Y_ref.view(torch.int16))
+        if first is None:
+            first = Y
+        assert torch.equal(Y.view(torch.int16), first.view(torch.int16))
+    differ = Y.view(torch.int16) != Y_ref.view(torch.int16)
+    assert int(differ.sum()) <= max(1, Y.numel() // 500)
+    gap = (Y.float() - Y_ref.float()).abs()
+    assert bool((gap <= Y_ref.float().abs() * 2.0 ** -6 + 1e-30).all())      # at most the neighbouring bf16 value
     _, _, mask1 = oracle.prune24(W)
     err = rel_fro(to_f64(B.bits_from_bf16(Y)), oracle.fwd_rows(X, W, mask1, np.arange(b), L, R))
     assert err <= REL_TOL, err
@@ -619,8 +630,9 @@ def test_forward_with_adapter_in_one_call_equals_the_two_calls_bitwise(B, oracle
 
 def test_chain_of_fused_adapter_forwards_in_a_cuda_graph(B, oracle):
     """Four decode-size layers, each through the one-call forward, each fed by the previous one's
-    output (so every pair's first launch really has to wait for the pair before it): eager result,
-    captured graph and its replays agree bitwise with the chain of separate calls."""
+    output (so every pair's first launch really has to wait for the pair before it): the eager
+    result agrees with the chain of separate calls up to the summation order of the K-split, and
+    the captured graph and its replays reproduce the eager bits."""
     import torch
 
     dims, b, r = [512, 1024, 384, 640, 512], 8, 64
@@ -646,7 +658,8 @@ def test_chain_of_fused_adapter_forwards_in_a_cuda_graph(B, oracle):
     with torch.cuda.stream(side):
         chain()                                                    # eager, also warms up before capture
         side.synchronize()
-        assert torch.equal(acts[4].view(torch.int16), ref.view(torch.int16))
+        eager = acts[4].clone()
+        assert rel_fro(eager.double().cpu().numpy(), ref.double().cpu().numpy()) <= 2e-3
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=side):
             chain()
@@ -654,6 +667,6 @@ def test_chain_of_fused_adapter_forwards_in_a_cuda_graph(B, oracle):
             acts[4].zero_()
             graph.replay()
             side.synchronize()
-            assert torch.equal(acts[4].view(torch.int16), ref.view(torch.int16))
+            assert torch.equal(acts[4].view(torch.int16), eager.view(torch.int16))
     torch.cuda.current_stream().wait_stream(side)
     layers[0].poll()
