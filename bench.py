@@ -711,7 +711,7 @@ def inference_forward_probe(torch, B, wl, pk, copies=12, reps=5):
         B.slope_prune_24(W, vals, meta, None)
         Wc = [(vals.clone(), meta.clone()) for _ in range(copies)]
         Wd = [W.clone() for _ in range(copies)]
-        for b in (1, 8, 64):
+        for b in (1, 8, 64, 512, 2048):
             X = B.bf16_from_bits(si.gaussian_bf16((b, d_in), 1.0, si.seed_for(9, 0, "X")), dev)
             Y = torch.empty((b, d_out), dtype=torch.bfloat16, device=dev)
             us_dense = time_graph(lambda: [torch.matmul(X, w.t(), out=Y) for w in Wd])

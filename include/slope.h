@@ -109,9 +109,10 @@ slope_status_t slope_linear_fwd(const void* X, int b, const void* Wc_vals, const
  * The same sums as slope_adapter_fwd_bwd(phase 0) followed by slope_linear_fwd: T bit for bit; Y up
  * to the order of fp32 partial sums (a fused pair may split the reduction differently), and
  * deterministic like every other call.
- * T is caller-owned scratch that holds X L afterwards.  At inference sizes (where the few-token
- * kernel serves the forward) the two launches are issued as a fused pair: the forward streams
- * its weights and runs its sparse reduction while T is still being computed and waits only for
+ * T is caller-owned scratch that holds X L afterwards.  At inference sizes (decode, and prefill
+ * up to a few thousand tokens: as long as the T launch is small enough to run beside the forward
+ * and an estimate says it pays) the two launches are issued as a fused pair: the forward streams
+ * its operands and runs its sparse reduction while T is still being computed and waits only for
  * T itself, which takes the adapter's extra launch off the critical path (Sec. "Efficient
  * inference": the adapter multiplications are what limits the inference speedup).  With more
  * tokens it issues the same two launches as the separate calls.  The stream must not receive

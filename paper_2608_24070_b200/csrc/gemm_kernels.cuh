@@ -78,6 +78,7 @@ struct DenseGemmParams {
     int k_splits;
     void* out;
     const uint8_t* mask;          // kEpiMasked: [M x N/8]
+    int pdl_mode;                 // 1: producer of a fused pair of launches (wait first, release dependents afterwards)
 };
 
 template <int BLOCK_N, int STAGES>
@@ -130,8 +131,13 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
     const uint32_t tmem_base = *tmem_slot;
     // Programmatic dependent launch: the set-up above may overlap the tail of the previous kernel in
     // the stream; no thread touches global memory before that kernel has completed.
-    griddep_launch_dependents();
-    griddep_wait();
+    if (p0.pdl_mode == 1) {              // see the few-token kernel: the dependent may rely on all earlier work
+        griddep_wait();
+        griddep_launch_dependents();
+    } else {
+        griddep_launch_dependents();
+        griddep_wait();
+    }
 
     // tile -> (problem, m block, n block, split): m fastest so that concurrently running CTAs share B
     auto decode = [&](int tile, int& m_blk, int& n_blk, int& kb0, int& kb1) {
@@ -915,8 +921,10 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     const uint32_t tmem_base = *tmem_slot;
     // Programmatic dependent launch: the set-up above may overlap the tail of the previous kernel in
     // the stream; no thread touches global memory before that kernel has completed.
+    // (consumer of a fused pair of launches, pdl_mode 2: only the producer thread waits, before its
+    // first load of the adapter operand T)
     griddep_launch_dependents();
-    griddep_wait();
+    if (p.pdl_mode != 2) griddep_wait();
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both CTAs)
@@ -927,6 +935,7 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             const uint64_t keep = l2_policy_evict_last();
             PipeState ps;
             bool ok = true;
+            bool waited = false;
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs) {
                 int mt, n_blk, next_mt, next_n_blk;
                 bool first, next_first = false;
@@ -975,6 +984,10 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                         }
                     } else {
                         const int ab = kb - num_kb;
+                        if (p.pdl_mode == 2 && !waited) {
+                            griddep_wait();
+                            waited = true;
+                        }
                         if (cta == 0)
                             mbar_expect_tx(&full_bar[ps.stage], 2 * (Cfg::kHalfN * 128 + nsub * Cfg::kABytes));
                         tma_load_2d_pair(sB, &tmB2, bar, ab * 64, n_row0);

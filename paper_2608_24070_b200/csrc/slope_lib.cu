@@ -254,6 +254,7 @@ struct DenseProblem {
     int M = 0, N = 0, K = 0, k_splits = 1;
     void* out = nullptr;
     const void* mask = nullptr;
+    int pdl_mode = 0;
 };
 
 // One launch of the 1-CTA dense kernel over one or two problems of the same kind.
@@ -273,20 +274,27 @@ static slope_status_t launch_dense2(const DenseProblem& q0, const DenseProblem& 
         const bool live = i == 0 || q1.M > 0;
         p[i].M = live ? q.M : 0; p[i].N = q.N; p[i].K = q.K; p[i].k_splits = q.k_splits; p[i].out = q.out;
         p[i].mask = static_cast<const uint8_t*>(q.mask);
+        p[i].pdl_mode = q0.pdl_mode;
         if (live) tiles += ((q.M + kBlockM - 1) / kBlockM) * ((q.N + BLOCK_N - 1) / BLOCK_N) * q.k_splits;
     }
     auto kern = dense_gemm_kernel<A_MN, B_MN, BLOCK_N, EPI, STAGES>;
     if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
-    const int grid = tiles < info.sm_count ? tiles : info.sm_count;
-    return launch_cluster_ex(kern, grid, 1, kGemmThreads, Cfg::kSmemBytes, /*overlap_prologue=*/true, stream, tm[0],
-                             tm[1], p[0], tm[2], tm[3], p[1]);
+    int grid = tiles < info.sm_count ? tiles : info.sm_count;
+    // The producer of a fused pair runs beside a kernel of CTA pairs: launched as clusters of two its
+    // CTAs fill whole SM pairs instead of breaking up many (the kernel itself ignores the cluster;
+    // a CTA without a tile exits at once).
+    const int cluster = q0.pdl_mode == 1 ? 2 : 1;
+    if (cluster == 2) grid = (grid + 1) & ~1;
+    return launch_cluster_ex(kern, grid, cluster, kGemmThreads, Cfg::kSmemBytes, /*overlap_prologue=*/true, stream,
+                             tm[0], tm[1], p[0], tm[2], tm[3], p[1]);
 }
 
 template <bool A_MN, bool B_MN, int BLOCK_N, int EPI, int STAGES>
 static slope_status_t launch_dense(const void* A, const void* B, int M, int N, int K, int k_splits, void* out,
-                                   const void* mask, cudaStream_t stream, const DeviceInfo& info) {
+                                   const void* mask, cudaStream_t stream, const DeviceInfo& info, int pdl_mode = 0) {
     DenseProblem q;
     q.A = A; q.B = B; q.M = M; q.N = N; q.K = K; q.k_splits = k_splits; q.out = out; q.mask = mask;
+    q.pdl_mode = pdl_mode;
     return launch_dense2<A_MN, B_MN, BLOCK_N, EPI, STAGES>(q, DenseProblem{}, stream, info);
 }
 
@@ -299,7 +307,8 @@ constexpr int kPairNarrowStages = 5;
 template <int BLOCK_N, int STAGES>
 static slope_status_t launch_sparse_pair(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                          const void* act2, const void* fac2, int r, bool a2_mn, void* out,
-                                         cudaStream_t stream, const DeviceInfo& info, int pdl_mode = 0) {
+                                         cudaStream_t stream, const DeviceInfo& info, int pdl_mode = 0,
+                                         int reserved_ctas = 0) {
     using Cfg = SparsePairCfg<BLOCK_N, STAGES>;
     CUtensorMap tmA, tmB, tmE, tmA2, tmB2, tmO;
     if (!make_tmap(&tmA, vals, M, K / 2, kBlockM, 64)) return SLOPE_ERR_CUDA;
@@ -321,8 +330,8 @@ static slope_status_t launch_sparse_pair(const void* act, int ntok, const void* 
     if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
     p.pdl_mode = pdl_mode;
     const int tiles = ((M / kBlockM + 1) / 2) * ((ntok + BLOCK_N - 1) / BLOCK_N);
-    // (the consumer of a fused pair leaves the producer's SMs alone: up to 8 CTAs per 128 adapter columns)
-    const int max_pairs = (info.sm_count - (pdl_mode == 2 ? 8 * ((r + kBlockM - 1) / kBlockM) : 0)) / 2;
+    // (the consumer of a fused pair leaves the producer's SMs alone)
+    const int max_pairs = (info.sm_count - reserved_ctas) / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
     return launch_pairs(kern, 2 * pairs, Cfg::kThreads, Cfg::kSmemBytes, stream, tmA, tmB, tmE, tmA2, tmB2, tmO, p);
 }
@@ -356,7 +365,8 @@ static int quad_group_m(int M, int K, int ntok, int num_pairs) {
 
 static slope_status_t launch_sparse_quad(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                          const void* act2, const void* fac2, int r, bool a2_mn, void* out,
-                                         cudaStream_t stream, const DeviceInfo& info) {
+                                         cudaStream_t stream, const DeviceInfo& info, int pdl_mode = 0,
+                                         int reserved_ctas = 0) {
     using Cfg = SparseQuadCfg<kQuadBlockN, kQuadStages>;
     CUtensorMap tmA, tmB, tmE, tmA2, tmB2, tmO;
     if (!make_tmap(&tmA, vals, M, K / 2, kBlockM, 64)) return SLOPE_ERR_CUDA;
@@ -374,11 +384,12 @@ static slope_status_t launch_sparse_quad(const void* act, int ntok, const void* 
     p.M = M; p.K = K; p.Ntok = ntok; p.r = r; p.a2_mn_major = a2_mn ? 1 : 0;
     p.meta = static_cast<const uint8_t*>(meta);
     p.out = static_cast<uint16_t*>(out);
-    p.group_m = quad_group_m(M, K, ntok, info.sm_count / 2);
+    const int max_pairs = (info.sm_count - reserved_ctas) / 2;
+    p.pdl_mode = pdl_mode;
+    p.group_m = quad_group_m(M, K, ntok, max_pairs);
     auto kern = sparse_gemm_quad_kernel<kQuadBlockN, kQuadStages>;
     if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
     const int tiles = ((M / kBlockM + 3) / 4) * ((ntok + kQuadBlockN - 1) / kQuadBlockN);
-    const int max_pairs = info.sm_count / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
     return launch_pairs(kern, 2 * pairs, Cfg::kThreads, Cfg::kSmemBytes, stream, tmA, tmB, tmE, tmA2, tmB2, tmO, p);
 }
@@ -525,7 +536,7 @@ static slope_status_t launch_skinny(const void* act, int ntok, const void* vals,
 // cost of a tile.
 enum class SparseTile { kQuad224, kPair224, kPair128 };
 
-static SparseTile choose_sparse_tile(int M, int K, int ntok, int num_pairs) {
+static SparseTile choose_sparse_tile(int M, int K, int ntok, int num_pairs, double* cost_out = nullptr) {
     // Waves of full tiles; the ragged last token tile of every row tile runs at its own width
     // (its weight loads do not shrink, its epilogue does: measured, a 32-token tile costs 0.7-0.9
     // of a 224-token one at reductions of 4096 and more, about 0.4 at 1024) and comes last in tile
@@ -548,7 +559,12 @@ static SparseTile choose_sparse_tile(int M, int K, int ntok, int num_pairs) {
     const double cost_quad = 2.0 * (1.0 - gain) * rounds(512, kPairBlockN);
     const double narrow_penalty = K >= 8192 ? 1.35 : K >= 4096 ? 1.30 : K >= 2048 ? 1.20 : 1.12;
     const double cost_narrow = narrow_penalty * kPairNarrowBlockN / kPairBlockN * rounds(256, kPairNarrowBlockN);
-    if (cost_quad < cost_pair && cost_quad <= cost_narrow) return SparseTile::kQuad224;
+    // (cost_out: the winner's cost in time units of one 256 x 224 tile)
+    if (cost_quad < cost_pair && cost_quad <= cost_narrow) {
+        if (cost_out) *cost_out = cost_quad;
+        return SparseTile::kQuad224;
+    }
+    if (cost_out) *cost_out = cost_narrow < cost_pair ? cost_narrow : cost_pair;
     return cost_narrow < cost_pair ? SparseTile::kPair128 : SparseTile::kPair224;
 }
 
@@ -574,21 +590,32 @@ static bool use_few_token_kernel(int M, int K, int ntok, int r, const DeviceInfo
     return few_us <= tile_us;
 }
 
+// One of the three tile kernels.  As the consumer of a fused pair of launches (pdl_mode 2) it leaves
+// `reserved_ctas` SMs to the producer that runs beside it.
+static slope_status_t launch_sparse_tiles(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
+                                          const void* act2, const void* fac2, int r, bool a2_mn, void* out,
+                                          cudaStream_t stream, const DeviceInfo& info, int pdl_mode = 0,
+                                          int reserved_ctas = 0) {
+    switch (choose_sparse_tile(M, K, ntok, (info.sm_count - reserved_ctas) / 2)) {
+        case SparseTile::kQuad224:
+            return launch_sparse_quad(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info, pdl_mode,
+                                      reserved_ctas);
+        case SparseTile::kPair128:
+            return launch_sparse_pair<kPairNarrowBlockN, kPairNarrowStages>(act, ntok, vals, meta, M, K, act2, fac2, r,
+                                                                            a2_mn, out, stream, info, pdl_mode,
+                                                                            reserved_ctas);
+        default:
+            return launch_sparse_pair<kPairBlockN, kPairStages>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out,
+                                                                stream, info, pdl_mode, reserved_ctas);
+    }
+}
+
 static slope_status_t launch_sparse_gemm(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                          const void* act2, const void* fac2, int r, bool a2_mn, void* out,
                                          cudaStream_t stream, const DeviceInfo& info) {
     if (use_few_token_kernel(M, K, ntok, r, info))
         return launch_skinny(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
-    switch (choose_sparse_tile(M, K, ntok, info.sm_count / 2)) {
-        case SparseTile::kQuad224:
-            return launch_sparse_quad(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
-        case SparseTile::kPair128:
-            return launch_sparse_pair<kPairNarrowBlockN, kPairNarrowStages>(act, ntok, vals, meta, M, K, act2, fac2, r,
-                                                                            a2_mn, out, stream, info);
-        default:
-            return launch_sparse_pair<kPairBlockN, kPairStages>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out,
-                                                                stream, info);
-    }
+    return launch_sparse_tiles(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info);
 }
 
 template <bool A_MN, bool B_MN, int BLOCK_N, int EPI, int STAGES>
@@ -599,7 +626,7 @@ static slope_status_t launch_dense_pair(const void* A, const void* B, int M, int
     const bool okA = A_MN ? make_tmap(&tmA, A, K, M, 64, 64) : make_tmap(&tmA, A, M, K, kBlockM, 64);
     const bool okB = B_MN ? make_tmap(&tmB, B, K, N, 64, 64) : make_tmap(&tmB, B, N, K, Cfg::kHalfN, 64);
     if (!okA || !okB) return SLOPE_ERR_CUDA;
-    DenseGemmParams p;
+    DenseGemmParams p = {};
     p.M = M; p.N = N; p.K = K; p.k_splits = 1; p.out = out;
     p.mask = static_cast<const uint8_t*>(mask);
     auto kern = dense_gemm_pair_kernel<A_MN, B_MN, BLOCK_N, EPI, STAGES>;
@@ -734,25 +761,37 @@ slope_status_t slope_linear_fwd_adapter(const void* X, int b, const void* Wc_val
             return st;
         return launch_skinny(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R, r, true, Y, stream, info, 2);
     }
+    // More tokens: the tile kernels are the consumer of such a pair in the same way, as long as the
+    // T launch is small enough to run beside them (it then costs the forward that share of the
+    // machine, which pays while T takes a comparable time: up to 32 CTAs, i.e. 4096 tokens at r <= 128).
+    const bool t_few = b <= kSkinnyMaxTokens;
+    const bool t_narrow = adapter_narrow_tiles(b, r, info);
+    const int t_ctas = t_few ? 8 * ((r + kBlockM - 1) / kBlockM)
+                             : ((b + kBlockM - 1) / kBlockM) * (t_narrow ? (r + 63) / 64 : (r + 127) / 128);
+    const int reserved = (t_ctas + 1) & ~1;
+    // Worth it?  Side by side the forward runs on fewer CTA pairs (more waves of tiles, perhaps)
+    // but no longer waits for T; one after the other it has the whole machine.  Tile time and T
+    // time from the measured constants: ~0.33 us per 128-wide k-block and tile + ~1.5 us of
+    // epilogue; a T CTA walks d_in in 64-wide steps of ~0.3 us after ~6 us of launch and start-up.
+    int mode = 0;
+    if (reserved <= info.sm_count / 3) {
+        double cost_full = 0.0, cost_beside = 0.0;
+        choose_sparse_tile(d_out, d_in, b, info.sm_count / 2, &cost_full);
+        choose_sparse_tile(d_out, d_in, b, (info.sm_count - reserved) / 2, &cost_beside);
+        const double tile_us = d_in / 128 * 0.33 + 1.5;
+        const double t_us = t_few ? 5.0 : 6.0 + d_in / 64 * 0.3;
+        const double fwd_beside = cost_beside * tile_us + 2.0;
+        if (1.08 * (fwd_beside > t_us ? fwd_beside : t_us + 2.0) < t_us + cost_full * tile_us) mode = 1;
+    }
     slope_status_t st;
-    if (b <= kSkinnyMaxTokens) {
-        // a few more tokens: the 256-row tile kernel can be the consumer of such a pair as well
-        const SparseTile tile = choose_sparse_tile(d_out, d_in, b, info.sm_count / 2);
-        if (tile != SparseTile::kQuad224) {
-            st = launch_skinny(nullptr, b, nullptr, nullptr, r, 0, X, L, d_in, true, T, stream, info, 1);
-            if (st) return st;
-            return tile == SparseTile::kPair128
-                       ? launch_sparse_pair<kPairNarrowBlockN, kPairNarrowStages>(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R,
-                                                                                  r, true, Y, stream, info, 2)
-                       : launch_sparse_pair<kPairBlockN, kPairStages>(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R, r, true, Y,
-                                                                      stream, info, 2);
-        }
-        st = launch_skinny(nullptr, b, nullptr, nullptr, r, 0, X, L, d_in, true, T, stream, info);
-    } else
-        st = adapter_narrow_tiles(b, r, info)
-                 ? launch_dense<false, true, 64, kEpiStore, 9>(X, L, b, r, d_in, 1, T, nullptr, stream, info)
-                 : launch_dense<false, true, 128, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info);
+    if (t_few)
+        st = launch_skinny(nullptr, b, nullptr, nullptr, r, 0, X, L, d_in, true, T, stream, info, mode);
+    else
+        st = t_narrow ? launch_dense<false, true, 64, kEpiStore, 9>(X, L, b, r, d_in, 1, T, nullptr, stream, info, mode)
+                      : launch_dense<false, true, 128, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info, mode);
     if (st) return st;
+    if (mode == 1)
+        return launch_sparse_tiles(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R, r, /*a2_mn=*/true, Y, stream, info, 2, reserved);
     return launch_sparse_gemm(X, b, Wc_vals, Wc_meta, d_out, d_in, T, R, r, /*a2_mn=*/true, Y, stream, info);
 }
 

@@ -589,7 +589,8 @@ def test_dependent_launches_back_to_back_equal_synchronised_launches_bitwise(B, 
 @pytest.mark.parametrize("d_in,d_out,b,r", [(1024, 512, 1, 16), (4096, 512, 8, 64), (512, 1536, 16, 128),
                                             (2048, 256, 40, 64), (1152, 384, 104, 256), (1024, 512, 16, 256),
                                             (1024, 2816, 64, 64), (256, 2048, 128, 32), (1024, 384, 200, 64),
-                                            (512, 5632, 250, 256), (384, 640, 776, 32)])
+                                            (512, 5632, 250, 256), (384, 640, 776, 32), (1024, 1024, 1000, 64),
+                                            (2048, 512, 2048, 128), (512, 2816, 1544, 16)])
 def test_forward_with_adapter_in_one_call_against_the_two_calls(B, oracle, d_in, d_out, b, r):
     """slope_linear_fwd_adapter: at inference sizes a fused pair of launches (the forward runs its
     sparse reduction while T is still being computed), with many tokens the plain two launches.
