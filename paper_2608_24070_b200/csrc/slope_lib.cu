@@ -781,7 +781,7 @@ slope_status_t slope_linear_fwd_adapter(const void* X, int b, const void* Wc_val
         const double tile_us = d_in / 128 * 0.33 + 1.5;
         const double t_us = t_few ? 5.0 : 6.0 + d_in / 64 * 0.3;
         const double fwd_beside = cost_beside * tile_us + 2.0;
-        if (1.08 * (fwd_beside > t_us ? fwd_beside : t_us + 2.0) < t_us + cost_full * tile_us) mode = 1;
+        if (1.15 * (fwd_beside > t_us ? fwd_beside : t_us + 2.0) < t_us + cost_full * tile_us) mode = 1;
     }
     slope_status_t st;
     if (t_few)
