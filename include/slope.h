@@ -95,8 +95,10 @@ slope_status_t slope_double_prune(const void* W, const void* mask1_bits, int d_o
  * runs on a kernel that streams the compressed weight once from HBM and splits the
  * reduction over a thread-block cluster.  All GEMM launches of this library are issued with
  * programmatic stream serialisation (their set-up may overlap the previous kernel's tail) and
- * synchronise on the device before they touch memory, so stream order holds as for any other
- * launch.  Every compute call of this library can be captured in a CUDA graph
+ * synchronise on the device before they touch memory (the second launch of
+ * slope_linear_fwd_adapter relies on its first one having done so and waits only for that one's
+ * output), so stream order holds as for any other launch.  Every compute call of this library
+ * can be captured in a CUDA graph
  * (slope_poll_status synchronises the stream and cannot).
  */
 slope_status_t slope_linear_fwd(const void* X, int b, const void* Wc_vals, const void* Wc_meta,
