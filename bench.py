@@ -470,6 +470,7 @@ def main():
         out["optimizer_tail"] = optimizer_tail_probe(torch, B, layers, stream, pk)
         out["burst"] = burst_probe(torch, B, layers, stream, pk)
         out["inference_forward"] = inference_forward_probe(torch, B, wl, pk)
+        out["decode_block"] = decode_block_probe(torch, B)
         out["nm_masked_dense"] = nm_probe(torch, B, layers, stream, pk)
         out["forward_speedup_by_shape"] = forward_shape_sweep(torch, B, stream)
         out["small_configs_hot_cold"] = small_config_probe(torch, B, stream, pk)
@@ -753,6 +754,92 @@ def inference_forward_probe(torch, B, wl, pk, copies=12, reps=5):
                     f"weight copies, best of {reps} replays, us per call; bytes: 1.125 B per weight element "
                     f"(values + metadata) + activations + adapter factors; HBM peak {pk['hbm_gbs']} GB/s "
                     f"({pk['src']}); cuBLAS reads the dense bf16 weight (2 B per element, no adapter)",
+            "rows": rows}
+
+
+def decode_block_probe(torch, B, blocks=4, reps=5):
+    """The linears of a LLaMA-7B decoder block at decode sizes, in the order a block runs them and
+    each fed by a real predecessor in the stream: q, k, v stacked along d_out (4096 -> 12288), o,
+    gate and up stacked (4096 -> 22016), down; `blocks` blocks with their own weights (> L2
+    together) in one CUDA graph.  Stacking is exact for both pruning passes.  The activations between
+    the linears are stand-ins of the right shape (attention and the gate are not part of this
+    library).  With adapters every linear is one slope_linear_fwd_adapter call; cuBLAS runs the
+    dense bf16 weights without adapters."""
+    dev = torch.device("cuda")
+    shapes = [("qkv", 4096, 12288), ("o", 4096, 4096), ("gate_up", 4096, 22016), ("down", 11008, 4096)]
+    gen = torch.Generator(device="cuda").manual_seed(si.seed_for(8, 0, "W"))
+    mk = lambda shape, sigma: (torch.randn(shape, device="cuda", generator=gen) * sigma).bfloat16()
+    dense, sparse, adapters = [], [], {64: [], 256: []}
+    for _ in range(blocks):
+        dl, sl = [], []
+        for name, d_in, d_out in shapes:
+            W = mk((d_out, d_in), 0.02)
+            vals, meta, _ = B.alloc_compressed(d_out, d_in, dev)
+            B.slope_prune_24(W, vals, meta, None)
+            dl.append(W)
+            sl.append((vals, meta, d_out))
+        dense.append(dl)
+        sparse.append(sl)
+    for r in adapters:
+        adapters[r] = [(mk((d_in, r), 0.01), mk((r, d_out), 0.01)) for _, d_in, d_out in shapes]
+
+    def time_graph(fn):
+        side = torch.cuda.Stream()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            fn(); fn()
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                fn()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); graph.replay(); e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        return best * 1e3 / blocks                          # microseconds per block
+
+    rows = []
+    for b in (1, 8):
+        X = {d: mk((b, d), 1.0) for d in (4096, 11008)}
+        Y = {n: torch.empty((b, d_out), dtype=torch.bfloat16, device=dev) for n, _, d_out in shapes}
+
+        def run_dense():
+            for dl in dense:
+                for (name, d_in, d_out), W in zip(shapes, dl):
+                    torch.matmul(X[d_in], W.t(), out=Y[name])
+
+        def run_sparse():
+            for sl in sparse:
+                for (name, d_in, d_out), (vals, meta, _) in zip(shapes, sl):
+                    B.slope_linear_fwd(X[d_in], vals, meta, d_out, Y[name])
+
+        us_dense, us_sparse = time_graph(run_dense), time_graph(run_sparse)
+        row = {"tokens": b, "cublas_dense_us_per_block": round(us_dense, 1), "slope_us_per_block": round(us_sparse, 1),
+               "speedup": round(us_dense / us_sparse, 3)}
+        for r, facs in adapters.items():
+            T = torch.empty((b, r), dtype=torch.bfloat16, device=dev)
+
+            def run_adapter():
+                for sl in sparse:
+                    for (name, d_in, d_out), (vals, meta, _), (L, R) in zip(shapes, sl, facs):
+                        B.slope_linear_fwd_adapter(X[d_in], vals, meta, d_out, L, R, T, Y[name])
+
+            us = time_graph(run_adapter)
+            row[f"slope_rank{r}_us_per_block"] = round(us, 1)
+            row[f"speedup_rank{r}"] = round(us_dense / us, 3)
+        rows.append(row)
+    st = B.slope_poll_status()
+    if st != 0:
+        raise SystemExit(f"device status after the decode block probe: {B.slope_status_string(st)}")
+    weight_bytes = sum(d_in * d_out for _, d_in, d_out in shapes)
+    return {"what": f"the four linears of a LLaMA-7B decoder block at decode sizes (q, k, v stacked; gate, up stacked), "
+                    f"{blocks} blocks with their own weights in one CUDA graph, us per block, best of {reps} replays; "
+                    f"compressed weights {weight_bytes * 1.125 / 1e6:.0f} MB per block against {weight_bytes * 2 / 1e6:.0f} MB dense",
             "rows": rows}
 
 

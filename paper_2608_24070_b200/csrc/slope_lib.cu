@@ -181,7 +181,7 @@ static slope_status_t launch_cluster(void (*kern)(KArgs...), int grid, int clust
 template <typename Kernel>
 static int max_active_clusters(Kernel kern, int cluster, int threads, int smem_bytes, int sm_count) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(cluster * sm_count, 1, 1);
+    cfg.gridDim = dim3(cluster * sm_count * 8, 1, 1);      // (the answer is capped by the grid of the query)
     cfg.blockDim = dim3(threads, 1, 1);
     cfg.dynamicSmemBytes = smem_bytes;
     cudaLaunchAttribute attr;
@@ -239,6 +239,11 @@ static bool set_smem(Kernel k, int bytes) {
     for (int i = 0; i < n_done; ++i)
         if (done[i].fn == fn && done[i].dev == dev && done[i].bytes >= bytes) return true;
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    // all of the SM's L1 / shared memory as shared memory: a kernel that asks for under half of it
+    // would otherwise get a carve-out that holds only one of its CTAs
+    if (cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) !=
+        cudaSuccess)
+        return false;
     if (n_done < kMax) done[n_done++] = Done{fn, dev, bytes};
     return true;
 }
@@ -445,8 +450,14 @@ static bool skinny_capacity(const DeviceInfo& info, int (&cap)[9]) {
         for (int s = 1; s <= 8; ++s)
             capacity[dev][s] = max_active_clusters(kern, s, kGemmThreads, Cfg::kSmemBytes, info.sm_count);
     }
+    // The occupancy query answers one CTA per SM for every kernel that allocates tensor memory,
+    // whatever its shared memory (it cannot know how many columns a CTA will ask for).  The CTA
+    // scheduler itself goes by registers, warps and shared memory: two CTAs of a variant that
+    // needs under half of the shared memory do run side by side (measured: a launch of 172 CTAs
+    // takes one wave, not two), and their 32- or 128-column allocations fit together.
+    const int per_sm = 2 * (Cfg::kSmemBytes + 1024) <= 232448 ? 2 : 1;
     cap[0] = 0;
-    for (int s = 1; s <= 8; ++s) cap[s] = capacity[dev][s];
+    for (int s = 1; s <= 8; ++s) cap[s] = capacity[dev][s] * per_sm;
     return cap[1] > 0;
 }
 
@@ -507,12 +518,32 @@ static slope_status_t launch_sparse_skinny(const void* act, int ntok, const void
 // dT = dY R^T at inference sizes.
 constexpr int kSkinnyMaxTokens = 256;
 
+// A variant of the few-token kernel with a half as deep weight ring fits two CTAs on an SM (the
+// same bytes in flight per SM).  It pays when the slabs times K-slices of a launch exceed what the
+// machine holds at one CTA per SM (stacked projections, d_out beyond ~19000 rows): one wave
+// instead of two.  Decided by the same cost model over both variants' capacities.
+template <int BLOCK_N, int A_DEEP, int B_DEEP, int A_FLAT, int B_FLAT>
+static bool prefer_two_ctas_per_sm(int M, int K, const DeviceInfo& info) {
+    if (K <= 0) return false;
+    int cap_deep[9], cap_flat[9];
+    if (!skinny_capacity<BLOCK_N, A_DEEP, B_DEEP>(info, cap_deep)) return false;
+    if (!skinny_capacity<BLOCK_N, A_FLAT, B_FLAT>(info, cap_flat)) return false;
+    double est_deep = 0.0, est_flat = 0.0;
+    const int slabs = (M + kBlockM - 1) / kBlockM;
+    skinny_splits(slabs, K / 128, BLOCK_N, cap_deep, &est_deep);
+    skinny_splits(slabs, K / 128, BLOCK_N, cap_flat, &est_flat);
+    return est_flat < 0.93 * est_deep;
+}
+
 static slope_status_t launch_skinny(const void* act, int ntok, const void* vals, const void* meta, int M, int K,
                                     const void* act2, const void* fac2, int r, bool a2_mn, void* out,
                                     cudaStream_t stream, const DeviceInfo& info, int pdl_mode = 0) {
-    if (ntok <= 16)
+    if (ntok <= 16) {
+        if (prefer_two_ctas_per_sm<16, 10, 4, 5, 2>(M, K, info))
+            return launch_sparse_skinny<16, 5, 2>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info, pdl_mode);
         return launch_sparse_skinny<16, 10, 4>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info, pdl_mode);
-    if (ntok <= 64)
+    }
+    if (ntok <= 64)      // (a two-per-SM variant of this tile, <64, 4, 2>, measured slower: its activation ring is too shallow)
         return launch_sparse_skinny<64, 8, 4>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info, pdl_mode);
     if (ntok <= 128)
         return launch_sparse_skinny<128, 7, 3>(act, ntok, vals, meta, M, K, act2, fac2, r, a2_mn, out, stream, info, pdl_mode);
