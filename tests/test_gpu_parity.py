@@ -124,6 +124,8 @@ CASES = [
     (256, 384, 130, 0, 32),          #   tile kernels
     (384, 512, 250, 16, 33),         #   adapter products still on the few-token kernel
     (512, 256, 1001, 32, 34),        #   one-CTA dense kernels for T / dT, 16 token k-blocks with a tail of 41
+    (512, 22016, 8, 16, 35),         # more weight slabs (172) than SMs: few-token kernel with two CTAs per SM
+    (256, 19200, 1, 0, 36),          #   same, one token, 150 slabs
 ]
 
 
