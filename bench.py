@@ -758,15 +758,21 @@ def inference_forward_probe(torch, B, wl, pk, copies=12, reps=5):
 
 
 def decode_block_probe(torch, B, blocks=4, reps=5):
-    """The linears of a LLaMA-7B decoder block at decode sizes, in the order a block runs them and
-    each fed by a real predecessor in the stream: q, k, v stacked along d_out (4096 -> 12288), o,
-    gate and up stacked (4096 -> 22016), down; `blocks` blocks with their own weights (> L2
+    """decode_block_width for LLaMA-7B and LLaMA-13B widths."""
+    return {"llama7b": decode_block_width(torch, B, 4096, 11008, blocks, reps),
+            "llama13b": decode_block_width(torch, B, 5120, 13824, blocks, reps)}
+
+
+def decode_block_width(torch, B, d, ffn, blocks=4, reps=5):
+    """The linears of a LLaMA-style decoder block (width d, hidden ffn) at decode sizes, in the order
+    a block runs them and each fed by a real predecessor in the stream: q, k, v stacked along d_out
+    (d -> 3d), o, gate and up stacked (d -> 2 ffn), down; `blocks` blocks with their own weights (> L2
     together) in one CUDA graph.  Stacking is exact for both pruning passes.  The activations between
     the linears are stand-ins of the right shape (attention and the gate are not part of this
     library).  With adapters every linear is one slope_linear_fwd_adapter call; cuBLAS runs the
     dense bf16 weights without adapters."""
     dev = torch.device("cuda")
-    shapes = [("qkv", 4096, 12288), ("o", 4096, 4096), ("gate_up", 4096, 22016), ("down", 11008, 4096)]
+    shapes = [("qkv", d, 3 * d), ("o", d, d), ("gate_up", d, 2 * ffn), ("down", ffn, d)]
     gen = torch.Generator(device="cuda").manual_seed(si.seed_for(8, 0, "W"))
     mk = lambda shape, sigma: (torch.randn(shape, device="cuda", generator=gen) * sigma).bfloat16()
     dense, sparse, adapters = [], [], {64: [], 256: []}
@@ -805,7 +811,7 @@ def decode_block_probe(torch, B, blocks=4, reps=5):
 
     rows = []
     for b in (1, 8):
-        X = {d: mk((b, d), 1.0) for d in (4096, 11008)}
+        X = {w: mk((b, w), 1.0) for w in (d, ffn)}
         Y = {n: torch.empty((b, d_out), dtype=torch.bfloat16, device=dev) for n, _, d_out in shapes}
 
         def run_dense():
@@ -837,7 +843,7 @@ def decode_block_probe(torch, B, blocks=4, reps=5):
     if st != 0:
         raise SystemExit(f"device status after the decode block probe: {B.slope_status_string(st)}")
     weight_bytes = sum(d_in * d_out for _, d_in, d_out in shapes)
-    return {"what": f"the four linears of a LLaMA-7B decoder block at decode sizes (q, k, v stacked; gate, up stacked), "
+    return {"what": f"the four linears of a LLaMA-style decoder block of width {d} / {ffn} at decode sizes (q, k, v stacked; gate, up stacked), "
                     f"{blocks} blocks with their own weights in one CUDA graph, us per block, best of {reps} replays; "
                     f"compressed weights {weight_bytes * 1.125 / 1e6:.0f} MB per block against {weight_bytes * 2 / 1e6:.0f} MB dense",
             "rows": rows}
