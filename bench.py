@@ -4,9 +4,11 @@
 A step = one pass of the whole hot path over one batch of synthetic input, for every
 linear layer of the workload: first-pass prune + compress, double prune, [adapter T = X L],
 forward, [adapter backward], input gradient, masked weight gradient -- every stage a
-hand-written kernel behind the C ABI.  Prints ONE JSON line (rank 0).
+hand-written kernel behind the C ABI.  The LAST line of stdout (rank 0) is one compact JSON
+object (at most 2000 characters: headline, clocks, roofline, dense comparison, e2e, CPU baseline); the
+per-stage table and, with --extras, the probe suite go to a side file.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload KEY] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload KEY] [--impl reference] [--extras]
 
 N > 1 (under torchrun) runs N independent replicas (the path has no exchange step).
 """
@@ -195,12 +197,10 @@ def cpu_baseline_sample(wl, seconds_hint=15.0):
         dt += time.perf_counter() - t0
         flops += (2 * len(rows) * (2.0 * lay.d_in * lay.d_out + 2.0 * r * (lay.d_in + lay.d_out))
                   + len(orows) * 2.0 * b * lay.d_in)
-        what.append(f"layer '{lay.name}' {lay.d_in}->{lay.d_out}, b={b}: fwd+dX on {len(rows)} token rows, "
-                    f"masked dW on {len(orows)} d_out rows")
+        what.append(f"{lay.name} {lay.d_in}->{lay.d_out} b={b}: fwd+dX {len(rows)} token rows, dW {len(orows)} rows")
     value = flops / dt / 1e12
-    return {"value": value, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle", "seconds": round(dt, 2),
-            "sample": ("the whole workload: " if full else "bounded sample: ") + "; ".join(what) +
-                      " (dense-equivalent FLOPs of what was computed / wall time)",
+    return {"value": round(value, 6), "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle", "seconds": round(dt, 2),
+            "sample": ("whole workload: " if full else "bounded sample: ") + "; ".join(what),
             "full_workload": full,
             "extrapolated_step_seconds": round(step_flops / (value * 1e12), 1),
             "extrapolation": "flop-scaled: dense-equivalent FLOPs of one step (fwd + dX + dW + adapter terms of every layer) "
@@ -266,6 +266,106 @@ def replica_throughput(world, flops_per_replica, ms_step):
     return world * flops_per_replica / (ms_step * 1e-3) / 1e12
 
 
+def kernel_sources_sha256():
+    """Hash of the CUDA sources the library is built from: the ncu-recorded DRAM traffic below is
+    reported only while it describes the kernels that actually ran."""
+    import hashlib
+
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2608_24070_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        if name.endswith((".cu", ".cuh")):
+            with open(os.path.join(csrc, name), "rb") as f:
+                h.update(name.encode() + b"\0" + f.read())
+    return h.hexdigest()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from an ncu capture of the two tensor-core
+# kernels at 4096 tokens (one pass, --clock-control none), scaled by tokens to the bench's launch.
+# `sources` is kernel_sources_sha256() of the build that was captured; a build with other sources
+# reports traffic = null (tests/test_bench_line.py fails until the capture is refreshed or cleared).
+NCU_TRAFFIC = {
+    "sources": None,
+    "captured_tokens": 4096,
+    "sparse_bytes_per_launch": None,      # mean over the 14 sparse GEMM launches of one step
+    "dense_bytes_per_launch": None,       # mean over the 7 weight-gradient launches of one step
+}
+
+
+def recorded_traffic(kind, wl_key, tokens):
+    if NCU_TRAFFIC["sources"] is None or wl_key not in ("c3_llama7b", "c4_llama7b_adapter"):
+        return None, "no ncu capture recorded for this workload"
+    if NCU_TRAFFIC["sources"] != kernel_sources_sha256():
+        return None, "stale: the kernels changed since the recorded ncu capture"
+    v = NCU_TRAFFIC[f"{kind}_bytes_per_launch"]
+    if v is None:
+        return None, "no ncu capture recorded for this kernel"
+    scale = tokens / NCU_TRAFFIC["captured_tokens"]
+    return round(v * scale), f"ncu at {NCU_TRAFFIC['captured_tokens']} tokens x{scale:g}, sources {NCU_TRAFFIC['sources'][:12]}"
+
+
+SM_COUNT = 148
+DENSE_FLOP_PER_CLK_SM = 8192            # dense bf16 tcgen05: 2 * 4096 MAC per clock and SM
+DATASHEET_SPARSE_TFLOPS = 4500.0
+DATASHEET_DENSE_TFLOPS = 2250.0
+
+
+def algorithmic_bytes(op, b, d_in, d_out, r):
+    """Minimum HBM bytes of one launch (activations in and out, compressed weight, adapter operands)."""
+    w = 1.125 * d_in * d_out
+    if op == "linear_fwd":
+        return 2.0 * b * d_in + w + 2.0 * b * d_out + (2.0 * b * r + 2.0 * r * d_out if r else 0.0)
+    if op == "linear_bwd_dx":
+        return 2.0 * b * d_out + w + 2.0 * b * d_in + (2.0 * b * r + 2.0 * r * d_in if r else 0.0)
+    if op == "linear_bwd_dw_masked":
+        return 2.0 * b * (d_in + d_out) + w
+    return 0.0
+
+
+def compact_line(out):
+    """The one line the driver parses: short enough to survive a few-KB tail of stdout."""
+    line = json.dumps(out, separators=(",", ":"))
+    if len(line) > 2000:
+        raise SystemExit(f"bench line grew to {len(line)} characters; move detail to the side file")
+    return line
+
+
+def headline(args, wl, b, world, value, ms_step, executed_tflops, launches, clocks_full, roofline, other,
+             ms_step_staged, stage_ms):
+    """The compact record (pure function of measured numbers: also exercised without a GPU)."""
+    clocks = None
+    if clocks_full is not None:
+        clocks = {k: clocks_full.get(k) for k in ("sm_mhz", "sm_mhz_min", "sm_max_mhz", "power_w_max", "reasons")}
+    adapter_ms = stage_ms.get("adapter_T", 0.0) + stage_ms.get("adapter_bwd", 0.0)
+    return {
+        "impl": "slope", "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.key, "tokens": b, "rank": wl.rank, "parallelism": "replicas" if world > 1 else "1 GPU",
+                   "l2": "inputs larger than L2",
+                   "step": f"prune, double prune, adapters, fwd, dX, masked dW x {len(wl.layers)} layers"},
+        "executed_tflops": round(executed_tflops, 2),
+        "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
+        "roofline_other": None if other is None else {k: other[k] for k in (
+            "kernel", "achieved", "peak", "frac", "frac_sustained", "frac_clock", "kernel_ms_per_step")},
+        "ms_per_step_staged": round(ms_step_staged, 4),
+        "stage_ms": stage_ms,
+        "adapter_share": round(adapter_ms / sum(stage_ms.values()), 4) if stage_ms else None,
+    }
+
+
+def attach_extras(out, dl, e2e, cb):
+    """Dense comparison, end-to-end run and CPU baseline, cut down to what the line carries."""
+    if dl is not None:
+        out["dense_layer"] = {"cublas_ms": dl["dense_ms"], "inhouse_ms": dl["inhouse_dense_ms"], "slope_ms": dl["slope_ms"],
+                              "speedup": dl["speedup"], "speedup_vs_inhouse": dl["speedup_vs_inhouse_dense"]}
+    out["e2e"] = None if e2e is None else {k: e2e[k] for k in ("value", "unit", "ms_per_step", "h2d_bytes_per_step",
+                                                                 "d2h_bytes_per_step")}
+    out["cpu_baseline"] = None if cb is None else {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample",
+                                                                       "full_workload", "seconds")}
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -274,10 +374,17 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(si.WORKLOADS))
     ap.add_argument("--impl", default="slope", choices=["slope", "reference"])
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling only)")
-    ap.add_argument("--no-extras", action="store_true", help="skip dense comparison, e2e and CPU baseline")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="only the timed step: skip the per-stage pass' side file, dense comparison, e2e and CPU baseline")
+    ap.add_argument("--extras", action="store_true",
+                    help="also run the probe suite (per-op medians over 200 launches, burst, optimizer tail, N:M, "
+                         "inference forward, decode block, shape sweep, small configurations, decoder block) and "
+                         "write it to the side file")
+    ap.add_argument("--side-file", default=os.path.join(ROOT, "gpurun_out", "bench_extras.json"),
+                    help="where the per-stage table and the probe results go (not printed)")
     ap.add_argument("--cusparselt-context", action="store_true",
-                    help="also time the forward GEMMs through torch's semi-structured sparse matmul (cuSPARSELt, "
-                         "the library the paper builds on); context only, off by default")
+                    help="with --extras: also time the forward GEMMs through torch's semi-structured sparse matmul "
+                         "(cuSPARSELt, the library the paper builds on); context only")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "slope" and not args.tokens else args.warmup
 
@@ -323,23 +430,19 @@ def main():
         if dist is not None:
             dist.barrier()
 
+    def check_status(where):
+        st = B.slope_poll_status()
+        if st != 0:
+            raise SystemExit(f"device status after {where}: {B.slope_status_string(st)}")
+
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
-    st = B.slope_poll_status()
-    if st != 0:
-        raise SystemExit(f"device status after warm-up: {B.slope_status_string(st)}")
+    check_status("warm-up")
 
-    # ---------------- timed region: exactly K steps, device time, max over ranks
-    events = []
-
-    def rec(op, s, fn):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        fn()
-        e1.record(stream)
-        events.append((op, s, e0, e1))
-
+    # ---------------- timed region: exactly K steps, nothing but the library's launches between the
+    # two events (per-stage events would sit between the programmatic dependent launches), device
+    # time, max over ranks
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
@@ -351,142 +454,193 @@ def main():
     t_begin = time.time()
     ev0.record(stream)
     for _ in range(args.steps):
-        step(rec)
+        step()
     ev1.record(stream)
     torch.cuda.synchronize()
     t_end = time.time()
     barrier()
     launches = B.slope_launch_count() - launches0
-    if rank == 0:
-        time.sleep(0.1)
-    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     ms_total = replica_max_ms(torch, dist, ev0.elapsed_time(ev1), dev)
-    st = B.slope_poll_status()
-    if st != 0:
-        raise SystemExit(f"device status after the timed region: {B.slope_status_string(st)}")
+    check_status("the timed region")
     ms_step = ms_total / args.steps
     value = replica_throughput(world, de_flops, ms_step)
 
-    # ---------------- per-stage times from the same timed region
-    per_op = {op: 0.0 for op in OPS}
+    # ---------------- stage pass: the same K steps again, every call bracketed by CUDA events on the
+    # launching stream; per (layer, op) the MEDIAN over the K launches.  The clock sampler keeps
+    # running, so the clocks below cover both passes (same load).
+    events = []
+
+    def rec(op, s, fn):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        fn()
+        e1.record(stream)
+        events.append((op, s, e0, e1))
+
+    ev2, ev3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev2.record(stream)
+    for _ in range(args.steps):
+        step(rec)
+    ev3.record(stream)
+    torch.cuda.synchronize()
+    t_end_stage = time.time()
+    ms_step_staged = ev2.elapsed_time(ev3) / args.steps
+    check_status("the stage pass")
+    if rank == 0:
+        time.sleep(0.1)
+    clocks_full = sampler.stop(t_begin, t_end_stage) if rank == 0 else None
+
     per_layer_op = {}
     for op, s, e0, e1 in events:
-        ms = e0.elapsed_time(e1)
-        per_op[op] += ms
-        per_layer_op.setdefault((s.name, s.d_in, s.d_out, op), []).append(ms)
-    per_op_ms_step = {op: v / args.steps for op, v in per_op.items() if v > 0}
+        per_layer_op.setdefault((s.name, op), []).append(e0.elapsed_time(e1))
+    by_name = {s.name: s for s in layers}
 
     def op_flops(op, s):
         m = 2.0 * s.b * s.d_in * s.d_out
         return {"linear_fwd": m + 2.0 * s.b * s.r * s.d_out, "linear_bwd_dx": m + 2.0 * s.b * s.r * s.d_in,
                 "linear_bwd_dw_masked": m}.get(op, 0.0)
 
-    sparse_peak = 2.0 * pk["bf16_sustained"]
-    stage_rows = []
-    tot = {"linear_fwd": [0.0, 0.0], "linear_bwd_dx": [0.0, 0.0], "linear_bwd_dw_masked": [0.0, 0.0]}
-    seen = set()
-    for (name, d_in, d_out, op), lst in per_layer_op.items():
-        ms = statistics.mean(lst)
-        s = next(x for x in layers if x.name == name)
+    sm_mhz = (clocks_full or {}).get("sm_mhz")
+    stage_rows, per_op_ms = [], {op: 0.0 for op in OPS}
+    tot = {"sparse": [0.0, 0.0, 0.0, 0], "dense": [0.0, 0.0, 0.0, 0]}        # flops, seconds, bytes, launches
+    for (name, op), lst in per_layer_op.items():
+        s = by_name[name]
+        ms = statistics.median(lst)
+        per_op_ms[op] += ms
+        row = {"layer": name, "d_in": s.d_in, "d_out": s.d_out, "op": op, "ms_median": round(ms, 4),
+               "ms_mean": round(statistics.mean(lst), 4), "launches": len(lst)}
         fl = op_flops(op, s)
+        n_el = s.d_in * s.d_out
         if fl:
-            tot[op][0] += fl
-            tot[op][1] += ms * 1e-3
+            kind = "dense" if op == "linear_bwd_dw_masked" else "sparse"
+            nbytes = algorithmic_bytes(op, s.b, s.d_in, s.d_out, s.r)
+            t = tot[kind]
+            t[0] += fl; t[1] += ms * 1e-3; t[2] += nbytes; t[3] += 1
             tf = fl / (ms * 1e-3) / 1e12
-            peak = pk["bf16_sustained"] if op == "linear_bwd_dw_masked" else sparse_peak
-            stage_rows.append({"layer": name, "d_in": d_in, "d_out": d_out, "op": op, "ms": round(ms, 4),
-                               "tflops_dense_eq": round(tf, 1),
-                               "tflops_executed": round(tf if op == "linear_bwd_dw_masked" else tf / 2, 1),
-                               "frac_of_sustained_peak": round(tf / peak, 4)})
-        elif op in ("prune_24", "double_prune") and (d_in, d_out, op) not in seen:
-            seen.add((d_in, d_out, op))
-            bytes_ = d_in * d_out * (3.25 if op == "prune_24" else 3.25)   # double prune: 2 + 0.125 in, 1 + 0.125 out
-            stage_rows.append({"layer": name, "d_in": d_in, "d_out": d_out, "op": op, "ms": round(ms, 4),
-                               "gbs": round(bytes_ / (ms * 1e-3) / 1e9, 1)})
-        elif op in ("adapter_T", "adapter_bwd") and (d_in, d_out, op) not in seen:
-            # T = X L streams X once; the backward streams dY once for dT and X, dY once more for dL, dR
-            seen.add((d_in, d_out, op))
-            small = 2.0 * s.r * (s.b + d_in + d_out)
-            bytes_ = 2.0 * s.b * d_in + small if op == "adapter_T" else 2.0 * s.b * (d_in + 2 * d_out) + 3 * small
-            stage_rows.append({"layer": name, "d_in": d_in, "d_out": d_out, "op": op, "ms": round(ms, 4),
-                               "gbs": round(bytes_ / (ms * 1e-3) / 1e9, 1),
-                               "frac_of_hbm_peak": round(bytes_ / (ms * 1e-3) / 1e9 / pk["hbm_gbs"], 3)})
+            burst = pk["bf16"] * (1.0 if kind == "dense" else 2.0)
+            t_star = max(fl / (burst * 1e12), nbytes / (pk["hbm_gbs"] * 1e9))
+            row.update({"tflops_dense_eq": round(tf, 1), "tflops_executed": round(tf if kind == "dense" else tf / 2, 1),
+                        "frac_of_burst_peak": round(tf / burst, 4), "roofline_frac_t_star": round(t_star / (ms * 1e-3), 4)})
+        elif op in ("prune_24", "double_prune"):
+            gbs = 3.25 * n_el / (ms * 1e-3) / 1e9
+            row.update({"gbs": round(gbs, 1), "frac_of_hbm_peak": round(gbs / pk["hbm_gbs"], 4)})
+        elif op in ("adapter_T", "adapter_bwd"):
+            # T = X L streams X once; the backward streams dY once for dT (X and dY for dL, dR ride in the dW launch
+            # when the library fuses them)
+            small = 2.0 * s.r * (s.b + s.d_in + s.d_out)
+            nbytes = 2.0 * s.b * s.d_in + small if op == "adapter_T" else 2.0 * s.b * (s.d_in + 2 * s.d_out) + 3 * small
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            row.update({"gbs": round(gbs, 1), "frac_of_hbm_peak": round(gbs / pk["hbm_gbs"], 4)})
+        stage_rows.append(row)
 
-    # roofline of the two tensor-core kernels; the dominant one (by time inside the step) is "roofline"
-    dw_fl, dw_s = tot["linear_bwd_dw_masked"]
-    dw_tflops = dw_fl / dw_s / 1e12 if dw_s else 0.0
-    roofline_dense = {"kernel": "dense_gemm_pair_kernel<MN,MN,256,masked,6> (slope_linear_bwd_dw_masked)",
-                      "bound": "tensor", "achieved": round(dw_tflops, 1), "peak": pk["bf16_sustained"],
-                      "unit": "TFLOP/s", "frac": round(dw_tflops / pk["bf16_sustained"], 4), "traffic": None,
-                      "ms_per_step": round(dw_s * 1e3, 4),
-                      "peak_source": f"{pk['src']} sustained dense bf16 (cuBLAS)"}
-    sp_fl = tot["linear_fwd"][0] + tot["linear_bwd_dx"][0]
-    sp_s = tot["linear_fwd"][1] + tot["linear_bwd_dx"][1]
-    sp_tflops = sp_fl / sp_s / 1e12 if sp_s else 0.0
-    roofline_sparse = {"kernel": "sparse_gemm_quad_kernel<224,3> (slope_linear_fwd, slope_linear_bwd_dx; shapes with short reductions or few tiles run on sparse_gemm_pair_kernel<224,4> / <128,5>)", "bound": "tensor",
-                       "achieved": round(sp_tflops, 1), "peak": round(sparse_peak, 1),
-                       "unit": "TFLOP/s", "frac": round(sp_tflops / sparse_peak, 4), "traffic": None,
-                       "ms_per_step": round(sp_s * 1e3, 4),
-                       "flops": "dense-equivalent (2*b*d_in*d_out per launch; half of them executed)",
-                       "frac_of_2x_burst_3386": round(sp_tflops / (2.0 * pk["bf16"]), 4),
-                       "frac_of_datasheet_4500": round(sp_tflops / 4500.0, 4),
-                       "peak_source": f"2 x {pk['src']} sustained dense bf16 (sparse bf16 peak := 2 x dense)"}
-    # dram__bytes_read + write per launch from the 1-pass ncu capture at these sizes
-    # (profiles/dram_traffic_full_size_c3_llama7b.md), averaged over the launches of a step.
-    if wl.key in ("c3_llama7b", "c4_llama7b_adapter") and b == 16384:
-        sp_reads = (154.9 + 154.5 + 155.4 + 155.6 + 154.6 + 165.5 + 154.7 + 154.6) + (374.3 + 792.3) + (376.9 + 792.6) \
-            + (792.5 + 361.9)
-        sp_writes = (109.0 + 105.8 + 107.5 + 106.2 + 106.5 + 106.0 + 105.2 + 105.8) + (356.7 + 146.5) + (358.2 + 146.8) \
-            + (146.5 + 356.3)
-        roofline_sparse["traffic"] = round((sp_reads + sp_writes) / 14 * 1e6)
-        roofline_sparse["traffic_note"] = "mean DRAM bytes per launch over the 14 sparse GEMM launches of a step (ncu, no adapter operands)"
-        roofline_sparse["algorithmic_bytes"] = round((4 * 2 * (153.1 + 134.2) + 2 * (184.9 + 360.7 + 411.4 + 134.2) + (411.4 + 134.2 + 184.9 + 360.7)) / 14 * 1e6)
-        dw_traffic = (630.4 + 14.2) + (630.6 + 14.2) + (630.4 + 14.5) + (630.4 + 14.2) + (1948.5 + 42.8) \
-            + (1990.3 + 42.6) + (1648.1 + 42.5)
-        roofline_dense["traffic"] = round(dw_traffic / 7 * 1e6)
-        roofline_dense["algorithmic_bytes"] = round((4 * (270.5 + 16.8) + 3 * (500.5 + 45.1)) / 7 * 1e6)
-    sparse_dominant = sp_s >= dw_s
+    def roofline_of(kind, kernel, peak_burst, peak_sustained, datasheet, flop_per_clk_sm):
+        fl, sec, nbytes, n = tot[kind]
+        if not sec:
+            return None
+        tf = fl / sec / 1e12
+        traffic, source = recorded_traffic(kind, wl.key, b)
+        r = {"kernel": kernel, "bound": "tensor", "achieved": round(tf, 1), "peak": round(peak_burst, 1),
+             "unit": "TFLOP/s", "frac": round(tf / peak_burst, 4), "traffic": traffic,
+             "algorithmic_bytes": round(nbytes / n), "traffic_source": source,
+             "peak_source": ("2 x " if kind == "sparse" else "") + f"{pk['src']} burst cuBLAS bf16",
+             "frac_sustained": round(tf / peak_sustained, 4), "frac_datasheet": round(tf / datasheet, 4),
+             "frac_clock": round(fl / sec / (sm_mhz * 1e6 * SM_COUNT * flop_per_clk_sm), 4) if sm_mhz else None,
+             "tflop_per_step": round(fl / 1e12, 4), "kernel_ms_per_step": round(sec * 1e3, 4), "launches_per_step": n}
+        return r
+
+    roofline_sparse = roofline_of(
+        "sparse", "sparse_gemm_quad/pair_kernel (fwd, dX)",
+        2.0 * pk["bf16"], 2.0 * pk["bf16_sustained"], DATASHEET_SPARSE_TFLOPS, 2 * DENSE_FLOP_PER_CLK_SM)
+    roofline_dense = roofline_of(
+        "dense", "dense_gemm_pair_kernel (masked dW)",
+        pk["bf16"], pk["bf16_sustained"], DATASHEET_DENSE_TFLOPS, DENSE_FLOP_PER_CLK_SM)
+    sparse_dominant = tot["sparse"][1] >= tot["dense"][1]
     roofline = roofline_sparse if sparse_dominant else roofline_dense
-    roofline_other = roofline_dense if sparse_dominant else roofline_sparse
+    other = roofline_dense if sparse_dominant else roofline_sparse
+    stage_ms = {k: round(v, 3) for k, v in per_op_ms.items() if v > 0}
 
-    out = {
-        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": wl.key, "tokens": b, "rank": wl.rank, "layers": [f"{l.name}:{l.d_in}->{l.d_out}" for l in wl.layers],
-                   "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "l2": "inputs larger than L2 (each layer streams > 126 MB of activations)",
-                   "step": "prune_24 + double_prune + adapter + fwd + dX + masked dW for every layer"},
-        "executed_tflops": round(world * ex_flops / (ms_step * 1e-3) / 1e12, 2),
-        "gpu_launches": int(launches),
-        "clocks": clocks,
-        "roofline": roofline,
-        "roofline_second_kernel": roofline_other,
-        "stage_ms_per_step": {k: round(v, 4) for k, v in per_op_ms_step.items()},
-        "stages": stage_rows,
-    }
+    out = headline(args, wl, b, world, value, ms_step, world * ex_flops / (ms_step * 1e-3) / 1e12, launches,
+                   clocks_full, roofline, other, ms_step_staged, stage_ms)
 
+    side = {"headline": dict(out), "clocks": clocks_full, "roofline_sparse": roofline_sparse,
+            "roofline_dense": roofline_dense, "stages": stage_rows}
     if rank == 0 and not args.no_extras and world == 1:
-        out["optimizer_tail"] = optimizer_tail_probe(torch, B, layers, stream, pk)
-        out["burst"] = burst_probe(torch, B, layers, stream, pk)
-        out["inference_forward"] = inference_forward_probe(torch, B, wl, pk)
-        out["decode_block"] = decode_block_probe(torch, B)
-        out["nm_masked_dense"] = nm_probe(torch, B, layers, stream, pk)
-        out["forward_speedup_by_shape"] = forward_shape_sweep(torch, B, stream)
-        out["small_configs_hot_cold"] = small_config_probe(torch, B, stream, pk)
-        out["dense_layer"] = dense_comparison(torch, B, layers, stream)
-        out["decoder_block_c5"] = decoder_block_probe(torch)
-        if args.cusparselt_context:
-            out["cusparselt_context"] = cusparselt_context(torch, B, layers, stream)
-        out["e2e"] = e2e_run(torch, B, layers, de_flops, max(2, min(args.steps, 5)))
-        out["cpu_baseline"] = cpu_baseline_sample(wl)
+        dl = dense_comparison(torch, B, layers, stream)
+        side["dense_layer"] = dl
+        if args.extras:
+            side["per_op_200"] = per_op_probe(torch, B, layers, stream, pk)
+            side["optimizer_tail"] = optimizer_tail_probe(torch, B, layers, stream, pk)
+            side["burst"] = burst_probe(torch, B, layers, stream, pk)
+            side["inference_forward"] = inference_forward_probe(torch, B, wl, pk)
+            side["decode_block"] = decode_block_probe(torch, B)
+            side["nm_masked_dense"] = nm_probe(torch, B, layers, stream, pk)
+            side["forward_speedup_by_shape"] = forward_shape_sweep(torch, B, stream)
+            side["small_configs_hot_cold"] = small_config_probe(torch, B, stream, pk)
+            side["decoder_block_c5"] = decoder_block_probe(torch)
+            if args.cusparselt_context:
+                side["cusparselt_context"] = cusparselt_context(torch, B, layers, stream)
+        e2e = e2e_run(torch, B, layers, de_flops, max(2, min(args.steps, 5)))
+        side["e2e"] = e2e
+        cb = cpu_baseline_sample(wl)
+        side["cpu_baseline"] = cb
+        attach_extras(out, dl, e2e, cb)
     elif rank == 0:
-        out["e2e"] = None
-        out["cpu_baseline"] = None
+        attach_extras(out, None, None, None)
     if rank == 0:
-        print(json.dumps(out), flush=True)
+        if not args.no_extras:
+            try:
+                os.makedirs(os.path.dirname(args.side_file), exist_ok=True)
+                with open(args.side_file, "w") as f:
+                    json.dump(side, f, indent=1)
+            except OSError as ex:
+                print(f"side file not written: {ex}", file=sys.stderr)
+        print(compact_line(out), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def per_op_probe(torch, B, layers, stream, pk, launches=200, warm=20):
+    """Every op of every distinct layer shape timed alone: `warm` untimed launches, then `launches`
+    launches each bracketed by its own pair of CUDA events; median per op (the activations of one
+    launch are larger than L2, so consecutive launches do not find them there)."""
+    rows, seen = [], set()
+    for s in layers:
+        if (s.d_in, s.d_out) in seen:
+            continue
+        seen.add((s.d_in, s.d_out))
+        calls = {"prune_24": lambda s=s: B.slope_prune_24(s.W, s.Wc_vals, s.Wc_meta, s.mask1),
+                 "double_prune": lambda s=s: B.slope_double_prune(s.W, s.mask1, s.WTc_vals, s.WTc_meta, None),
+                 "linear_bwd_dw_masked": lambda s=s: B.slope_linear_bwd_dw_masked(s.dY, s.X, s.mask1, s.dWc)}
+        if s.r:
+            calls["adapter_T"] = lambda s=s: B.slope_adapter_fwd_bwd(0, s.X, None, s.L, None, s.b, s.d_out, s.d_in, s.r, T=s.T)
+            calls["linear_fwd"] = lambda s=s: B.slope_linear_fwd(s.X, s.Wc_vals, s.Wc_meta, s.d_out, s.Y, s.T, s.R)
+            calls["adapter_bwd"] = lambda s=s: B.slope_adapter_fwd_bwd(1, s.X, s.dY, s.L, s.R, s.b, s.d_out, s.d_in, s.r,
+                                                                      T=s.T, dT=s.dT, dL=s.dL, dR=s.dR, workspace=s.ws)
+            calls["linear_bwd_dx"] = lambda s=s: B.slope_linear_bwd_dx(s.dY, s.WTc_vals, s.WTc_meta, s.d_in, s.dX, s.dT, s.L)
+        else:
+            calls["linear_fwd"] = lambda s=s: B.slope_linear_fwd(s.X, s.Wc_vals, s.Wc_meta, s.d_out, s.Y)
+            calls["linear_bwd_dx"] = lambda s=s: B.slope_linear_bwd_dx(s.dY, s.WTc_vals, s.WTc_meta, s.d_in, s.dX)
+        for op, fn in calls.items():
+            for _ in range(warm):
+                fn()
+            evs = []
+            for _ in range(launches):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream); fn(); e1.record(stream)
+                evs.append((e0, e1))
+            torch.cuda.synchronize()
+            ms = statistics.median(e0.elapsed_time(e1) for e0, e1 in evs)
+            row = {"d_in": s.d_in, "d_out": s.d_out, "tokens": s.b, "op": op, "ms_median": round(ms, 4)}
+            if op.startswith("linear"):
+                fl = 2.0 * s.b * s.d_in * s.d_out
+                peak = pk["bf16"] * (1.0 if op == "linear_bwd_dw_masked" else 2.0)
+                nbytes = algorithmic_bytes(op, s.b, s.d_in, s.d_out, s.r)
+                t_star = max(fl / (peak * 1e12), nbytes / (pk["hbm_gbs"] * 1e9))
+                row.update({"tflops_dense_eq": round(fl / ms / 1e9, 1), "frac_of_burst_peak": round(fl / ms / 1e9 / peak, 4),
+                            "roofline_frac_t_star": round(t_star / (ms * 1e-3), 4)})
+            rows.append(row)
+    return {"what": f"median of {launches} launches after {warm} warm-ups, each launch between its own CUDA events; "
+                    f"peaks: dense {pk['bf16']} TFLOP/s burst ({pk['src']}), sparse := 2 x dense", "rows": rows}
 
 
 def optimizer_tail_probe(torch, B, layers, stream, pk, reps=20):
@@ -1046,11 +1200,13 @@ def e2e_run(torch, B, layers, de_flops, steps):
             key = (nm, tuple(t.shape))
             if key not in host:
                 host[key] = t.cpu().pin_memory()
-        key = ("dWc", tuple(s.dWc.shape))
-        if key not in host:
-            host[key] = torch.empty(s.dWc.shape, dtype=s.dWc.dtype).pin_memory()
+        for nm in ("dWc", "dL", "dR") if s.r else ("dWc",):
+            t = getattr(s, nm)
+            key = (nm, tuple(t.shape))
+            if key not in host:
+                host[key] = torch.empty(t.shape, dtype=t.dtype).pin_memory()
     h2d = sum(2 * (s.X.numel() + s.dY.numel()) for s in layers)
-    d2h = sum(2 * s.dWc.numel() for s in layers)
+    d2h = sum(2 * (s.dWc.numel() + (s.dL.numel() + s.dR.numel() if s.r else 0)) for s in layers)
     n = len(layers)
     arrived = [torch.cuda.Event() for _ in range(n)]       # inputs of layer i are on the device
     consumed = [torch.cuda.Event() for _ in range(n)]      # layer i's kernels are done with its inputs
@@ -1072,7 +1228,9 @@ def e2e_run(torch, B, layers, de_flops, steps):
             consumed[i].record(compute)
             with torch.cuda.stream(d2h_stream):
                 d2h_stream.wait_event(consumed[i])
-                host[("dWc", tuple(s.dWc.shape))].copy_(s.dWc, non_blocking=True)
+                for nm in ("dWc", "dL", "dR") if s.r else ("dWc",):
+                    t = getattr(s, nm)
+                    host[(nm, tuple(t.shape))].copy_(t, non_blocking=True)
                 read_back[i].record(d2h_stream)
 
     def drain():
@@ -1093,7 +1251,8 @@ def e2e_run(torch, B, layers, de_flops, steps):
     return {"value": round(de_flops / (ms * 1e-3) / 1e12, 2), "unit": UNIT, "ms_per_step": round(ms, 3),
             "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": steps,
             "note": "pinned host X, dY -> device per layer (copy stream, overlapped with compute), C-ABI kernels, "
-                    "compressed dW -> pinned host"}
+                    "the layer's parameter gradients (compressed dW, dL, dR) -> pinned host; Y and dX stay on the "
+                    "device on purpose: they are the next / previous layer's input, not a result the host reads"}
 
 
 if __name__ == "__main__":

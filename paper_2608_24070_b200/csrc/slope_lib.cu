@@ -673,12 +673,15 @@ static int adapter_splits(int b, int rows) {
     // rounds(s) = ceil(tiles * s / SMs) passes over the machine, each 1/s of a tile long; take
     // the s that minimises rounds(s) / s (with a small charge per split for the fp32 partials),
     // keeping at least 4 k-blocks (256 tokens) per split and no split without a k-block.
+    // The split count sizes the caller's workspace (slope_adapter_workspace_bytes, which is asked
+    // with no device at hand), so it is a function of the shape alone: the SM count is the B200's.
+    constexpr int kSms = 148;
     const int tiles = (rows + kBlockM - 1) / kBlockM;
     const int num_kb = (b + 63) / 64;
     int best_s = 1;
     double best_cost = 1e30;
     for (int s = 1; s <= 16 && s * 4 <= num_kb; ++s) {
-        const int rounds = (tiles * s + 147) / 148;
+        const int rounds = (tiles * s + kSms - 1) / kSms;
         const double cost = static_cast<double>(rounds) / s + 0.004 * s;
         if (cost < best_cost - 1e-12) { best_cost = cost; best_s = s; }
     }

@@ -41,17 +41,17 @@ def _reference_dl(B, torch, X, dY, L, R, d_out):
 
 
 @pytest.mark.parametrize("shapes", [((2048, 640, 256, 64), (1024, 384, 128, 32))])
-def test_noalloc_dl_matches_workspace_path_on_two_calls_in_a_row(B, shapes):
+def test_noalloc_dl_matches_workspace_path_on_two_calls_in_a_row(B, oracle, shapes):
     """Two different problems back to back: the second call finds the first call's partial
-    sums in the shared fixed array and must not be disturbed by them."""
+    sums in the shared fixed array and must not be disturbed by them.  Each result is checked
+    against the workspace-based entry point and against the CPU oracle."""
     import torch
 
     for call, (b, d_in, d_out, r) in enumerate(shapes):
         seed = 900 + 10 * call
-        X = B.bf16_from_bits(si.gaussian_bf16((b, d_in), 1.0, seed))
-        dY = B.bf16_from_bits(si.gaussian_bf16((b, d_out), 1.0, seed + 1))
-        L = B.bf16_from_bits(si.gaussian_bf16((d_in, r), 0.01, seed + 2))
-        R = B.bf16_from_bits(si.gaussian_bf16((r, d_out), 0.01, seed + 3))
+        Xb, dYb = si.gaussian_bf16((b, d_in), 1.0, seed), si.gaussian_bf16((b, d_out), 1.0, seed + 1)
+        Lb, Rb = si.gaussian_bf16((d_in, r), 0.01, seed + 2), si.gaussian_bf16((r, d_out), 0.01, seed + 3)
+        X, dY, L, R = (B.bf16_from_bits(a) for a in (Xb, dYb, Lb, Rb))
         dT, dL_ref = _reference_dl(B, torch, X, dY, L, R, d_out)
         dL = torch.full((d_in, r), float("nan"), dtype=torch.bfloat16, device="cuda")
         B.slope_adapter_dl_noalloc(X, dT, dL)
@@ -62,6 +62,9 @@ def test_noalloc_dl_matches_workspace_path_on_two_calls_in_a_row(B, shapes):
         assert err <= REL_TOL, (call, err)
         # same kernels, same split order: in fact bit-identical
         assert np.array_equal(B.bits_from_bf16(dL), B.bits_from_bf16(dL_ref))
+        # and against the oracle's dL = X^T (dY R^T) (dT kept in fp64 there, bf16 here: two roundings)
+        err_o = rel_fro(got, oracle.adapter_dL_rows(Xb, dYb, Rb, np.arange(d_in)))
+        assert err_o <= REL_TOL, (call, err_o)
 
 
 def test_noalloc_rejects_sizes_beyond_its_fixed_scratch(B):
@@ -71,7 +74,10 @@ def test_noalloc_rejects_sizes_beyond_its_fixed_scratch(B):
     assert limit == 16 << 20
     buf = torch.zeros(4096, dtype=torch.uint8, device="cuda")
     p = ctypes.c_void_p(buf.data_ptr())
-    # 2 splits x 16512 x 128 x 4 bytes > 16 MiB: refused before any launch (pointers are never read)
-    assert B.lib().slope_adapter_dl_noalloc(p, p, 16384, 16512, 128, p, None) == 2
+    launches = B.slope_launch_count()
+    # 16512 x 256 x 4 bytes = 16.9 MB > 16 MiB already for a single split, whatever the split
+    # heuristic says: refused before any launch (the pointers are never read)
+    assert B.lib().slope_adapter_dl_noalloc(p, p, 16384, 16512, 256, p, None) == 2
     assert B.lib().slope_adapter_dl_noalloc(None, p, 1024, 128, 64, p, None) == 1
+    assert B.slope_launch_count() == launches
     assert B.slope_poll_status() == 0
