@@ -10,6 +10,35 @@ def rel_fro(gpu_f64: np.ndarray, ref: np.ndarray) -> float:
     return float(np.linalg.norm(gpu_f64 - ref) / (den if den > 0 else 1.0))
 
 
+# Elementwise bound beside the per-tensor norm.  One fp32 -> bf16 rounding moves an element by at
+# most half a unit in the last place, i.e. 2^-8 of its magnitude; what the fp32 accumulation and a
+# bf16-rounded adapter operand add is independent of the element's own size, so it is allowed
+# relative to the tensor's root mean square: 2^-9 for outputs rounded once (measured: fp32
+# accumulation ~1e-6, the adapter term's bf16 T ~1e-4 of the rms), 2^-6 for the gradients that are
+# sums over a bf16-rounded intermediate (dL over dT, dR over T: a Gaussian error of ~1.7e-3 rms per
+# element, whose largest value over a million elements is ~5 sigma).  A single wrong element (a
+# dropped k-block, a wrong metadata code) is off by a large fraction of the rms and fails this
+# where the Frobenius norm of a big tensor would hide it.
+ELEM_REL = 2.0 ** -8
+ELEM_RMS = {1: 2.0 ** -9, 2: 2.0 ** -6}
+
+
+def parity_error(gpu_f64: np.ndarray, ref: np.ndarray, roundings: int = 1) -> float:
+    """Relative Frobenius error of a GPU output against the oracle; raises when any single
+    element is further off than bf16 rounding (plus the slack above) explains."""
+    gpu_f64, ref = np.asarray(gpu_f64, dtype=np.float64), np.asarray(ref, dtype=np.float64)
+    assert gpu_f64.shape == ref.shape, (gpu_f64.shape, ref.shape)
+    rms = float(np.sqrt(np.mean(ref * ref))) if ref.size else 0.0
+    bound = ELEM_REL * np.abs(ref) + ELEM_RMS[roundings] * rms
+    excess = np.abs(gpu_f64 - ref) - bound
+    bad = int(np.count_nonzero(~(excess <= 0)))          # NaN counts as bad
+    if bad:
+        worst = np.unravel_index(int(np.nanargmax(np.where(np.isnan(excess), np.inf, excess))), ref.shape)
+        raise AssertionError(f"{bad} of {ref.size} elements outside the elementwise bound; worst at {worst}: "
+                             f"gpu {gpu_f64[worst]!r} oracle {ref[worst]!r} bound {bound[worst]!r} (rms {rms!r})")
+    return rel_fro(gpu_f64, ref)
+
+
 def to_f64(bits: np.ndarray) -> np.ndarray:
     return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
 

@@ -139,7 +139,7 @@ def _dense_dw_from_oracle(oracle, dY, X, d_out, d_in):
 @pytest.mark.parametrize("d_in,d_out,b", [(384, 640, 776), (1024, 256, 264), (128, 128, 8), (256, 384, 77), (384, 256, 1)])
 def test_dense_layer_against_oracle(B, oracle, d_in, d_out, b):
     import torch
-    from helpers import REL_TOL, rel_fro, to_f64
+    from helpers import REL_TOL, parity_error, to_f64
 
     W = si.gaussian_bf16((d_out, d_in), 0.02, 501)
     X = si.gaussian_bf16((b, d_in), 1.0, 502)
@@ -155,9 +155,9 @@ def test_dense_layer_against_oracle(B, oracle, d_in, d_out, b):
     full = np.full((d_out, d_in // 8), 0xFF, np.uint8)        # every entry kept: the dense layer
     rows = np.arange(b)
     errs = {
-        "Y": rel_fro(to_f64(B.bits_from_bf16(Y)), oracle.fwd_rows(X, W, full, rows)),
-        "dX": rel_fro(to_f64(B.bits_from_bf16(dX)), oracle.dx_rows(dY, W, full, rows)),
-        "dW": rel_fro(to_f64(B.bits_from_bf16(dW)), _dense_dw_from_oracle(oracle, dY, X, d_out, d_in)),
+        "Y": parity_error(to_f64(B.bits_from_bf16(Y)), oracle.fwd_rows(X, W, full, rows)),
+        "dX": parity_error(to_f64(B.bits_from_bf16(dX)), oracle.dx_rows(dY, W, full, rows)),
+        "dW": parity_error(to_f64(B.bits_from_bf16(dW)), _dense_dw_from_oracle(oracle, dY, X, d_out, d_in)),
     }
     print(errs)
     for k, v in errs.items():
@@ -168,7 +168,7 @@ def test_emulated_2_8_layer_matches_oracle_on_the_masks(B, oracle):
     """An N:M-emulated layer (2:8): prune, double prune, dense GEMMs on the masked-dense matrices and the
     masked weight gradient, against the oracle evaluated with the same (oracle-made) masks."""
     import torch
-    from helpers import REL_TOL, rel_fro, to_f64
+    from helpers import REL_TOL, parity_error, to_f64
 
     n, m, d_in, d_out, b = 2, 8, 512, 384, 264
     W = si.gaussian_bf16((d_out, d_in), 0.02, 511)
@@ -194,9 +194,9 @@ def test_emulated_2_8_layer_matches_oracle_on_the_masks(B, oracle):
     keep1 = oracle.mask_to_bool(mask1, d_in)
     want_dW = np.where(keep1, _dense_dw_from_oracle(oracle, dY, X, d_out, d_in), 0.0)
     errs = {
-        "Y": rel_fro(to_f64(B.bits_from_bf16(Y)), oracle.fwd_rows(X, W, mask1, rows)),
-        "dX": rel_fro(to_f64(B.bits_from_bf16(dX)), oracle.dx_rows(dY, W, mask2, rows)),
-        "dW": rel_fro(to_f64(B.bits_from_bf16(dW)), want_dW),
+        "Y": parity_error(to_f64(B.bits_from_bf16(Y)), oracle.fwd_rows(X, W, mask1, rows)),
+        "dX": parity_error(to_f64(B.bits_from_bf16(dX)), oracle.dx_rows(dY, W, mask2, rows)),
+        "dW": parity_error(to_f64(B.bits_from_bf16(dW)), want_dW),
     }
     print(errs)
     for k, v in errs.items():

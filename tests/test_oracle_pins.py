@@ -310,6 +310,34 @@ def test_p8_metadata_layout_spot_values(oracle):
     assert np.count_nonzero(hw) == 5
 
 
+# The tensor-core order written out as a TABLE instead of a formula (a slip in the oracle's index
+# arithmetic fails here on the CPU; the GPU exact case X = I pins the same order through the MMA).
+# tcgen05.cp.128x128b moves 128 shared-memory rows of 16 bytes into 128 tensor-memory lanes x 4
+# 32-bit columns: byte 16*lane + 4*column + 2*half of a 2 KB block.  One column serves two
+# consecutive K = 32 sparse MMAs of a 128-row operand; within each run of 16 operand rows the
+# metadata of a 16-column slot sits as follows (row within the 16 -> lane within the 16, half-word):
+_LANE_EVEN_SLOT = (0, 1, 2, 3, 4, 5, 6, 7, 0, 1, 2, 3, 4, 5, 6, 7)          # slots 0, 2, 4, 6 of a block
+_LANE_ODD_SLOT = (8, 9, 10, 11, 12, 13, 14, 15, 8, 9, 10, 11, 12, 13, 14, 15)  # slots 1, 3, 5, 7
+_HALF_WORD = (0, 0, 0, 0, 0, 0, 0, 0, 1, 1, 1, 1, 1, 1, 1, 1)
+_COLUMN_OF_SLOT = (0, 0, 1, 1, 2, 2, 3, 3)
+
+
+def test_p8_metadata_layout_against_the_lane_table(oracle):
+    rng = np.random.Generator(np.random.PCG64(8))
+    rows, cols = 384, 256
+    canon = rng.integers(0, 1 << 16, size=(rows, cols // 16), dtype=np.uint16)
+    want = np.zeros(rows * cols // 8, np.uint8)
+    for i in range(rows):
+        for u in range(cols // 16):
+            block = (i // 128) * (cols // 128) + u // 8
+            r16, slot = i % 16, u % 8
+            lane = 16 * ((i % 128) // 16) + (_LANE_ODD_SLOT if slot % 2 else _LANE_EVEN_SLOT)[r16]
+            byte = 2048 * block + 16 * lane + 4 * _COLUMN_OF_SLOT[slot] + 2 * _HALF_WORD[r16]
+            want[byte] = int(canon[i, u]) & 0xFF
+            want[byte + 1] = int(canon[i, u]) >> 8
+    assert np.array_equal(oracle.canonical_to_hw(canon), want)
+
+
 def test_pack_canonical(oracle):
     nib = np.array([[0x4, 0xD, 0x9, 0xE]], np.uint8)
     assert oracle.pack_canonical(nib).tolist() == [[0xE9D4]]
