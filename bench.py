@@ -147,7 +147,7 @@ class LayerState:
                                   dtype=torch.uint8, device=dev)
 
 
-OPS = ("prune_24", "double_prune", "adapter_T", "linear_fwd", "adapter_bwd", "linear_bwd_dx", "linear_bwd_dw_masked")
+OPS = ("prune_24_double", "adapter_T", "linear_fwd", "adapter_bwd", "linear_bwd_dx", "linear_bwd_dw_masked")
 
 
 def run_layer(B, s: LayerState, rec=None):
@@ -158,9 +158,10 @@ def run_layer(B, s: LayerState, rec=None):
         else:
             rec(op, s, fn)
 
-    stage("prune_24", lambda: B.slope_prune_24(s.W, s.Wc_vals, s.Wc_meta, s.mask1))
-    # the second-pass mask is an optional diagnostic output (no kernel of the step reads it)
-    stage("double_prune", lambda: B.slope_double_prune(s.W, s.mask1, s.WTc_vals, s.WTc_meta, None))
+    # both pruning passes in one launch (same outputs as slope_prune_24 + slope_double_prune, W read
+    # once); the second-pass mask is an optional diagnostic output that no kernel of the step reads
+    stage("prune_24_double", lambda: B.slope_prune_24_double(s.W, s.Wc_vals, s.Wc_meta, s.mask1, s.WTc_vals,
+                                                             s.WTc_meta, None))
     if s.r:
         stage("adapter_T", lambda: B.slope_adapter_fwd_bwd(0, s.X, None, s.L, None, s.b, s.d_out, s.d_in, s.r, T=s.T))
         stage("linear_fwd", lambda: B.slope_linear_fwd(s.X, s.Wc_vals, s.Wc_meta, s.d_out, s.Y, s.T, s.R))
@@ -343,7 +344,7 @@ def headline(args, wl, b, world, value, ms_step, executed_tflops, launches, cloc
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl.key, "tokens": b, "rank": wl.rank, "parallelism": "replicas" if world > 1 else "1 GPU",
                    "l2": "inputs larger than L2",
-                   "step": f"prune, double prune, adapters, fwd, dX, masked dW x {len(wl.layers)} layers"},
+                   "step": f"prune+double prune, adapters, fwd, dX, masked dW x {len(wl.layers)} layers"},
         "executed_tflops": round(executed_tflops, 2),
         "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
         "roofline_other": None if other is None else {k: other[k] for k in (
@@ -521,8 +522,9 @@ def main():
             t_star = max(fl / (burst * 1e12), nbytes / (pk["hbm_gbs"] * 1e9))
             row.update({"tflops_dense_eq": round(tf, 1), "tflops_executed": round(tf if kind == "dense" else tf / 2, 1),
                         "frac_of_burst_peak": round(tf / burst, 4), "roofline_frac_t_star": round(t_star / (ms * 1e-3), 4)})
-        elif op in ("prune_24", "double_prune"):
-            gbs = 3.25 * n_el / (ms * 1e-3) / 1e9
+        elif op == "prune_24_double":
+            # W in (2 B), two compressed copies out (1 + 1/8 B each), first mask out (1/8 B)
+            gbs = 4.375 * n_el / (ms * 1e-3) / 1e9
             row.update({"gbs": round(gbs, 1), "frac_of_hbm_peak": round(gbs / pk["hbm_gbs"], 4)})
         elif op in ("adapter_T", "adapter_bwd"):
             # T = X L streams X once; the backward streams dY once for dT (X and dY for dL, dR ride in the dW launch
@@ -610,6 +612,8 @@ def per_op_probe(torch, B, layers, stream, pk, launches=200, warm=20):
         seen.add((s.d_in, s.d_out))
         calls = {"prune_24": lambda s=s: B.slope_prune_24(s.W, s.Wc_vals, s.Wc_meta, s.mask1),
                  "double_prune": lambda s=s: B.slope_double_prune(s.W, s.mask1, s.WTc_vals, s.WTc_meta, None),
+                 "prune_24_double": lambda s=s: B.slope_prune_24_double(s.W, s.Wc_vals, s.Wc_meta, s.mask1, s.WTc_vals,
+                                                                        s.WTc_meta, None),
                  "linear_bwd_dw_masked": lambda s=s: B.slope_linear_bwd_dw_masked(s.dY, s.X, s.mask1, s.dWc)}
         if s.r:
             calls["adapter_T"] = lambda s=s: B.slope_adapter_fwd_bwd(0, s.X, None, s.L, None, s.b, s.d_out, s.d_in, s.r, T=s.T)
@@ -638,6 +642,9 @@ def per_op_probe(torch, B, layers, stream, pk, launches=200, warm=20):
                 t_star = max(fl / (peak * 1e12), nbytes / (pk["hbm_gbs"] * 1e9))
                 row.update({"tflops_dense_eq": round(fl / ms / 1e9, 1), "frac_of_burst_peak": round(fl / ms / 1e9 / peak, 4),
                             "roofline_frac_t_star": round(t_star / (ms * 1e-3), 4)})
+            elif op in ("prune_24", "double_prune", "prune_24_double"):
+                nbytes = (4.375 if op == "prune_24_double" else 3.25) * s.d_in * s.d_out
+                row.update({"gbs": round(nbytes / ms / 1e6, 1), "frac_of_hbm_peak": round(nbytes / ms / 1e6 / pk["hbm_gbs"], 4)})
             rows.append(row)
     return {"what": f"median of {launches} launches after {warm} warm-ups, each launch between its own CUDA events; "
                     f"peaks: dense {pk['bf16']} TFLOP/s burst ({pk['src']}), sparse := 2 x dense", "rows": rows}

@@ -86,6 +86,17 @@ slope_status_t slope_double_prune(const void* W, const void* mask1_bits, int d_o
                                   void* WTc_vals, void* WTc_meta, void* mask2_bits, void* stream);
 
 /*
+ * Both pruning passes in one launch (Algorithm 1 calls "backend.setup" twice, once for W and once
+ * for its transpose; Section "Double-pruned Backward Pass" makes the second a function of the
+ * first): every output of slope_prune_24 followed by slope_double_prune, bit for bit, while W is
+ * read once and the first mask is never read back (4.375 instead of 6.5 bytes of HBM traffic per
+ * weight element).  mask1_bits and mask2_bits may be NULL.
+ */
+slope_status_t slope_prune_24_double(const void* W, int d_out, int d_in,
+                                     void* Wc_vals, void* Wc_meta, void* mask1_bits,
+                                     void* WTc_vals, void* WTc_meta, void* mask2_bits, void* stream);
+
+/*
  * Forward, Eq. (sparse_forward), optionally with the lazy adapter fused as in
  * Eq. (concat):  Y[b x d_out] = X[b x d_in] (W^R)^T  (+ T[b x r] R[r x d_out]).
  * Wc_vals / Wc_meta come from slope_prune_24.  T = X L is produced by

@@ -31,7 +31,7 @@ EXPORTS = (
     "slope_sparse_add", "slope_update_sparse_matrix", "slope_selftest_wait_timeout",
     "slope_prune_nm", "slope_double_prune_nm", "slope_apply_mask",
     "slope_dense_linear_fwd", "slope_dense_linear_bwd_dx", "slope_dense_linear_bwd_dw", "slope_mask_difference",
-    "slope_linear_fwd_adapter",
+    "slope_linear_fwd_adapter", "slope_prune_24_double",
 )
 
 
@@ -55,6 +55,8 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).argtypes = [ci, ci]
         L.slope_prune_24.argtypes = [vp, ci, ci, vp, vp, vp, vp]
         L.slope_double_prune.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp]
+        L.slope_prune_24_double.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, vp, vp]
+        L.slope_prune_24_double.restype = ci
         L.slope_linear_fwd.argtypes = [vp, ci, vp, vp, ci, ci, vp, vp, ci, vp, vp]
         L.slope_linear_bwd_dx.argtypes = [vp, ci, vp, vp, ci, ci, vp, vp, ci, vp, vp]
         L.slope_linear_fwd_adapter.argtypes = [vp, ci, vp, vp, ci, ci, vp, vp, ci, vp, vp, vp]
@@ -145,6 +147,13 @@ def slope_double_prune(W, mask1_bits, WTc_vals, WTc_meta, mask2_bits=None):
     d_out, d_in = W.shape
     _check("slope_double_prune", lib().slope_double_prune(_ptr(W), _ptr(mask1_bits), d_out, d_in, _ptr(WTc_vals),
                                                           _ptr(WTc_meta), _ptr(mask2_bits), _stream()))
+
+
+def slope_prune_24_double(W, Wc_vals, Wc_meta, mask1_bits, WTc_vals, WTc_meta, mask2_bits=None):
+    d_out, d_in = W.shape
+    _check("slope_prune_24_double", lib().slope_prune_24_double(_ptr(W), d_out, d_in, _ptr(Wc_vals), _ptr(Wc_meta),
+                                                                _ptr(mask1_bits), _ptr(WTc_vals), _ptr(WTc_meta),
+                                                                _ptr(mask2_bits), _stream()))
 
 
 def slope_linear_fwd(X, Wc_vals, Wc_meta, d_out, Y, T=None, R=None):

@@ -27,6 +27,7 @@ struct PackedPick {
     uint32_t out0, out1;      // kept pair of group 0 / group 1: first kept in the low half
     uint32_t mask_byte;       // 4 keep bits of group 0 | 4 keep bits of group 1 << 4
     uint32_t meta_byte;       // code p0 | p1<<2 of group 0 | code of group 1 << 4
+    uint32_t keep[4];         // element i kept: 0xFFFF in the low half (group 0) / high half (group 1)
 };
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
@@ -61,6 +62,7 @@ __device__ __forceinline__ PackedPick pick2of4_packed(uint32_t E0, uint32_t E1, 
     const uint32_t p1 = bitsel(m3, 0x00030003u, bitsel(m2, 0x00020002u, 0x00010001u));
     const uint32_t c = p0 | (p1 << 2);
     r.meta_byte = (c | (c >> 12)) & 0xFFu;
+    r.keep[0] = m0; r.keep[1] = m1; r.keep[2] = m2; r.keep[3] = m3;
     return r;
 }
 
@@ -200,6 +202,103 @@ __global__ void __launch_bounds__(256, 4) double_prune_kernel(const uint4* __res
     if (tid < 128) {
         const size_t blk = static_cast<size_t>(cb) * (d_out >> 7) + rb;
         metaT[blk * 128 + tid] = reinterpret_cast<const uint4*>(s_meta)[tid];
+    }
+}
+
+// Both passes in one launch.  The second pass of a 128 x 128 tile needs nothing but what the first
+// pass makes of that same tile (groups of four rows never straddle a tile), so a CTA reads its tile
+// of W once, runs the first pass on it in registers, writes the forward copy, and feeds the masked
+// tile straight into the second pass: W is read once instead of twice and the first mask is never
+// read back (4.375 bytes per weight element for both compressed copies and both masks instead of
+// 6.5).  Thread layout of the second-pass kernel: 8 rows x 8 columns per thread, so a thread's row
+// holds exactly two first-pass groups, the pair the packed selection works on.
+// Outputs are bit for bit those of prune24_kernel followed by double_prune_kernel.
+__global__ void __launch_bounds__(256, 4) prune24_double_kernel(const uint4* __restrict__ W, int d_out, int d_in,
+                                                              uint2* __restrict__ vals, uint4* __restrict__ meta,
+                                                              uint4* __restrict__ mask1 /* may be null */,
+                                                              uint4* __restrict__ valsT, uint4* __restrict__ metaT,
+                                                              uint8_t* __restrict__ mask2 /* may be null */) {
+    __shared__ __align__(16) uint8_t s_out[128 * 128];       // [column j][16 slots of 8 B], slot index XOR (j >> 3)
+    __shared__ __align__(16) uint8_t s_metaT[2048];
+    __shared__ __align__(16) uint8_t s_meta[2048];
+    __shared__ __align__(16) uint8_t s_mask[2048];           // [row][16 bytes]
+
+    const int cb = blockIdx.x, rb = blockIdx.y;
+    const int tid = threadIdx.x;
+    const int c8 = tid & 15;                                 // 8-column slot of the tile
+    const int ig = tid >> 4;                                 // 8-row slot of the tile
+    const size_t row_u4 = static_cast<size_t>(d_in) >> 3;
+    const size_t mrow = static_cast<size_t>(d_in) >> 3;      // mask bytes (= uint2 of values) per row
+    const size_t at0 = (static_cast<size_t>(rb) * 128 + ig * 8) * row_u4 + cb * 16 + c8;
+
+    uint4 w[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) w[t] = __ldg(W + at0 + t * row_u4);
+
+    // ---- first pass: the two groups of this thread's 8 columns, row by row; W becomes W^R in place
+    uint32_t mb[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+        const PackedPick a = pick2of4_packed(prmt(w[t].x, w[t].z, 0x5410u), prmt(w[t].x, w[t].z, 0x7632u),
+                                             prmt(w[t].y, w[t].w, 0x5410u), prmt(w[t].y, w[t].w, 0x7632u));
+        const int rr = ig * 8 + t;
+        vals[at0 + t * mrow] = make_uint2(a.out0, a.out1);
+        s_meta[meta_byte_offset(rr, c8)] = static_cast<uint8_t>(a.meta_byte);
+        s_mask[rr * 16 + c8] = static_cast<uint8_t>(a.mask_byte);
+        mb[t] = a.mask_byte;
+        w[t].x &= prmt(a.keep[0], a.keep[1], 0x5410u);
+        w[t].y &= prmt(a.keep[2], a.keep[3], 0x5410u);
+        w[t].z &= prmt(a.keep[0], a.keep[1], 0x7632u);
+        w[t].w &= prmt(a.keep[2], a.keep[3], 0x7632u);
+    }
+
+    // ---- second pass on the masked tile (see double_prune_kernel)
+    uint32_t sel_bits[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const int meta_base = meta_byte_offset(c8 * 8, ig);
+#pragma unroll
+    for (int wi = 0; wi < 4; ++wi) {
+        uint32_t e[8];
+#pragma unroll
+        for (int t = 0; t < 8; ++t) e[t] = wi == 0 ? w[t].x : (wi == 1 ? w[t].y : (wi == 2 ? w[t].z : w[t].w));
+        const PackedPick a = pick2of4_packed(e[0], e[1], e[2], e[3]);
+        const PackedPick b = pick2of4_packed(e[4], e[5], e[6], e[7]);
+        const int j0 = c8 * 8 + 2 * wi;
+        const int slot = (ig ^ c8) * 8;
+        *reinterpret_cast<uint2*>(s_out + j0 * 128 + slot) = make_uint2(a.out0, b.out0);
+        *reinterpret_cast<uint2*>(s_out + (j0 + 1) * 128 + slot) = make_uint2(a.out1, b.out1);
+        s_metaT[meta_base + 16 * (2 * wi)] = static_cast<uint8_t>((a.meta_byte & 0xFu) | ((b.meta_byte & 0xFu) << 4));
+        s_metaT[meta_base + 16 * (2 * wi + 1)] = static_cast<uint8_t>((a.meta_byte >> 4) | (b.meta_byte & 0xF0u));
+        if (mask2 != nullptr) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                sel_bits[i] |= (((a.mask_byte >> i) & 1u) << (2 * wi)) | (((a.mask_byte >> (4 + i)) & 1u) << (2 * wi + 1));
+                sel_bits[4 + i] |= (((b.mask_byte >> i) & 1u) << (2 * wi)) | (((b.mask_byte >> (4 + i)) & 1u) << (2 * wi + 1));
+            }
+        }
+    }
+    if (mask2 != nullptr) {
+#pragma unroll
+        for (int t = 0; t < 8; ++t)
+            mask2[(static_cast<size_t>(rb) * 128 + ig * 8 + t) * mrow + cb * 16 + c8] =
+                static_cast<uint8_t>(sel_bits[t] & mb[t]);
+    }
+    __syncthreads();
+
+    const size_t vrow_u4 = static_cast<size_t>(d_out) >> 4;        // uint4 per row of valsT (d_out/2 bf16)
+#pragma unroll
+    for (int pass = 0; pass < 4; ++pass) {
+        const int jr = pass * 32 + (tid >> 3), seg = tid & 7;
+        const int x = (jr >> 3) & 15;
+        const uint4 v = *reinterpret_cast<const uint4*>(s_out + jr * 128 + (((2 * seg) ^ x) >> 1) * 16);
+        const uint4 o = (x & 1) ? make_uint4(v.z, v.w, v.x, v.y) : v;
+        valsT[(static_cast<size_t>(cb) * 128 + jr) * vrow_u4 + rb * 8 + seg] = o;
+    }
+    if (tid < 128) {
+        metaT[(static_cast<size_t>(cb) * (d_out >> 7) + rb) * 128 + tid] = reinterpret_cast<const uint4*>(s_metaT)[tid];
+        meta[(static_cast<size_t>(rb) * (d_in >> 7) + cb) * 128 + tid] = reinterpret_cast<const uint4*>(s_meta)[tid];
+    } else if (mask1 != nullptr) {
+        const int rr = tid - 128;
+        mask1[(static_cast<size_t>(rb) * 128 + rr) * (d_in >> 7) + cb] = reinterpret_cast<const uint4*>(s_mask)[rr];
     }
 }
 

@@ -46,7 +46,7 @@ def to_f64(bits: np.ndarray) -> np.ndarray:
 class GpuLayer:
     """Device-side state of one SLoPe layer driven through the C ABI."""
 
-    def __init__(self, W_bits, device="cuda"):
+    def __init__(self, W_bits, device="cuda", fused_setup=False):
         import torch
         from paper_2608_24070_b200 import binding as B
 
@@ -57,8 +57,12 @@ class GpuLayer:
         self.Wc_vals, self.Wc_meta, self.mask1 = B.alloc_compressed(self.d_out, self.d_in, device)
         self.WTc_vals, self.WTc_meta, _ = B.alloc_compressed(self.d_in, self.d_out, device)
         self.mask2 = torch.empty_like(self.mask1)
-        B.slope_prune_24(self.W, self.Wc_vals, self.Wc_meta, self.mask1)
-        B.slope_double_prune(self.W, self.mask1, self.WTc_vals, self.WTc_meta, self.mask2)
+        if fused_setup:      # both pruning passes in one launch
+            B.slope_prune_24_double(self.W, self.Wc_vals, self.Wc_meta, self.mask1, self.WTc_vals, self.WTc_meta,
+                                    self.mask2)
+        else:
+            B.slope_prune_24(self.W, self.Wc_vals, self.Wc_meta, self.mask1)
+            B.slope_double_prune(self.W, self.mask1, self.WTc_vals, self.WTc_meta, self.mask2)
 
     def canonical(self, meta, rows, cols):
         out = self.torch.empty((rows, cols // 16), dtype=self.torch.int16, device=meta.device)

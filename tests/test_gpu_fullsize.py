@@ -36,7 +36,8 @@ def test_full_size_layer(B, oracle, key, idx):
     b, d_in, d_out, r = wl.tokens, lay.d_in, lay.d_out, wl.rank
     t = si.layer_tensors(wl, idx)
     W, X, dY, L, R = t["W"], t["X"], t["dY"], t.get("L"), t.get("R")
-    layer = GpuLayer(W)
+    check_selection(oracle, GpuLayer(W), W)               # the two separate calls
+    layer = GpuLayer(W, fused_setup=True)                 # the one-call set-up the benchmark's step uses
     mask1, mask2 = check_selection(oracle, layer, W)
     Xd, dYd = B.bf16_from_bits(X), B.bf16_from_bits(dY)
     if r:
@@ -157,7 +158,8 @@ def test_more_than_2_31_activation_elements(B, oracle):
         assert bool(torch.isfinite(t[-extra:].float()).all())
 
 
-def test_pruning_a_matrix_of_more_than_2_31_elements(B, oracle):
+@pytest.mark.parametrize("fused", [False, True], ids=["two_calls", "one_call"])
+def test_pruning_a_matrix_of_more_than_2_31_elements(B, oracle, fused):
     """W[65792 x 32768] (2^31 + 8.4 M elements, 4.3 GB): a seeded 256-row block repeated 257 times.  Both
     pruning passes work on groups inside 128 x 128 tiles, so every 256-row slab of the outputs must equal
     the oracle's outputs for the block; the first, a middle and the last slab are compared bit for bit."""
@@ -177,8 +179,11 @@ def test_pruning_a_matrix_of_more_than_2_31_elements(B, oracle):
     vals, meta, mask1 = B.alloc_compressed(d_out, d_in)
     valsT, metaT, _ = B.alloc_compressed(d_in, d_out)
     mask2 = torch.empty_like(mask1)
-    B.slope_prune_24(W, vals, meta, mask1)
-    B.slope_double_prune(W, mask1, valsT, metaT, mask2)
+    if fused:
+        B.slope_prune_24_double(W, vals, meta, mask1, valsT, metaT, mask2)
+    else:
+        B.slope_prune_24(W, vals, meta, mask1)
+        B.slope_double_prune(W, mask1, valsT, metaT, mask2)
     assert B.slope_poll_status() == 0
     meta_rows = meta.view(d_out // 128, (d_in // 128) * 2048)
     metaT_blocks = metaT.view(d_in // 128, d_out // 128, 2048)

@@ -30,14 +30,33 @@ def dev(B, bits):
 
 
 # ------------------------------------------------------------------ selection / compression
+@pytest.mark.parametrize("fused", [False, True], ids=["two_calls", "one_call"])
 @pytest.mark.parametrize("d_out,d_in,seed", [(512, 512, 1), (384, 640, 2), (128, 1152, 3), (1280, 128, 4)])
-def test_prune_and_double_prune_bit_exact(B, oracle, d_out, d_in, seed):
+def test_prune_and_double_prune_bit_exact(B, oracle, d_out, d_in, seed, fused):
     W = si.gaussian_bf16((d_out, d_in), 0.02, seed)
-    layer = GpuLayer(W)
+    layer = GpuLayer(W, fused_setup=fused)
     check_selection(oracle, layer, W)
 
 
-def test_prune_ties_zeros_and_specials(B, oracle):
+def test_both_passes_in_one_call_without_the_optional_masks(B, oracle):
+    """slope_prune_24_double with mask1 / mask2 left out writes the same compressed copies."""
+    import torch
+
+    W = si.gaussian_bf16((384, 512), 0.02, 9)
+    ref = GpuLayer(W, fused_setup=True)
+    check_selection(oracle, ref, W)
+    Wd = dev(B, W)
+    vals, meta, _ = B.alloc_compressed(384, 512)
+    valsT, metaT, _ = B.alloc_compressed(512, 384)
+    B.slope_prune_24_double(Wd, vals, meta, None, valsT, metaT, None)
+    assert B.slope_poll_status() == 0
+    for a, b_ in ((vals, ref.Wc_vals), (valsT, ref.WTc_vals)):
+        assert torch.equal(a.view(torch.int16), b_.view(torch.int16))
+    assert torch.equal(meta, ref.Wc_meta) and torch.equal(metaT, ref.WTc_meta)
+
+
+@pytest.mark.parametrize("fused", [False, True], ids=["two_calls", "one_call"])
+def test_prune_ties_zeros_and_specials(B, oracle, fused):
     """All 4-tuples over {+0,-0,+-1,+-2} (ties everywhere), plus inf / nan / denormal patterns."""
     alphabet = si.f32_to_bf16_bits(np.array([0.0, -0.0, 1.0, -1.0, 2.0, -2.0], np.float32))
     groups = np.array(list(itertools.product(alphabet, repeat=4)), np.uint16).reshape(-1)
@@ -46,7 +65,7 @@ def test_prune_ties_zeros_and_specials(B, oracle):
     special = np.array([0x7F80, 0xFF80, 0x7FC0, 0x0001, 0x8001, 0x7F7F, 0x0080, 0xFFFF], np.uint16)
     rng = np.random.Generator(np.random.PCG64(5))
     W[128:, :] = rng.choice(special, size=(128, 256))
-    layer = GpuLayer(W)
+    layer = GpuLayer(W, fused_setup=fused)
     check_selection(oracle, layer, W)
 
 
