@@ -79,9 +79,6 @@ struct DenseGemmParams {
     void* out;
     const uint8_t* mask;          // kEpiMasked: [M x N/8]
     int pdl_mode;                 // 1: producer of a fused pair of launches (wait first, release dependents afterwards)
-    int tile_rows;                // 1-CTA kernel: rows of D a tile owns (0 = 128).  Fewer than 128: tiles start every
-                                  // tile_rows rows, still compute 128 and store only their own, so that a launch
-                                  // bound by what each SM can pull in spreads over every SM in one wave
 };
 
 template <int BLOCK_N, int STAGES>
@@ -112,9 +109,8 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    auto rows_of = [](const DenseGemmParams& q) { return q.tile_rows > 0 ? q.tile_rows : kBlockM; };
-    auto tiles_of = [&](const DenseGemmParams& q) {
-        return q.M == 0 ? 0 : ((q.M + rows_of(q) - 1) / rows_of(q)) * ((q.N + BLOCK_N - 1) / BLOCK_N) * q.k_splits;
+    auto tiles_of = [](const DenseGemmParams& q) {
+        return q.M == 0 ? 0 : ((q.M + kBlockM - 1) / kBlockM) * ((q.N + BLOCK_N - 1) / BLOCK_N) * q.k_splits;
     };
     const int tiles0 = tiles_of(p0);
     const int num_tiles = tiles0 + tiles_of(p1);
@@ -148,7 +144,7 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
         const bool second = tile >= tiles0;
         const DenseGemmParams& q = second ? p1 : p0;
         if (second) tile -= tiles0;
-        const int num_m = (q.M + rows_of(q) - 1) / rows_of(q);
+        const int num_m = (q.M + kBlockM - 1) / kBlockM;
         const int num_n = (q.N + BLOCK_N - 1) / BLOCK_N;
         const int num_kb_total = (q.K + 63) / 64;
         const int kb_per_split = (num_kb_total + q.k_splits - 1) / q.k_splits;
@@ -172,7 +168,6 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
                 const bool second = (decode(tile, m_blk, n_blk, kb0, kb1) & 0x10000) != 0;
                 const CUtensorMap* tmA = second ? &tmA1 : &tmA0;
                 const CUtensorMap* tmB = second ? &tmB1 : &tmB0;
-                const int m_row0 = m_blk * rows_of(second ? p1 : p0);
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (!mbar_wait(&empty_bar[ps.stage], ps.phase ^ 1u, abort_flag)) { ok = false; break; }
                     uint8_t* sA = smem + ps.stage * Cfg::kStageBytes;
@@ -180,10 +175,10 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
                     uint64_t* bar = &full_bar[ps.stage];
                     mbar_expect_tx(bar, Cfg::kStageBytes);
                     if (A_MN) {
-                        tma_load_2d(sA, tmA, bar, m_row0, kb * 64);
-                        tma_load_2d(sA + 8192, tmA, bar, m_row0 + 64, kb * 64);
+                        tma_load_2d(sA, tmA, bar, m_blk * kBlockM, kb * 64);
+                        tma_load_2d(sA + 8192, tmA, bar, m_blk * kBlockM + 64, kb * 64);
                     } else {
-                        tma_load_2d(sA, tmA, bar, kb * 64, m_row0);
+                        tma_load_2d(sA, tmA, bar, kb * 64, m_blk * kBlockM);
                     }
                     if (B_MN) {
 #pragma unroll
@@ -243,15 +238,14 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
             if (!mbar_wait(&tfull_bar[acc], acc_phase, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t t_row = tmem_base + acc * BLOCK_N + (static_cast<uint32_t>(q * 32) << 16);
-            const int m = m_blk * rows_of(p) + q * 32 + lane;
-            const bool mine = q * 32 + lane < rows_of(p);             // rows past tile_rows belong to the next tile
+            const int m = m_blk * kBlockM + q * 32 + lane;
 #pragma unroll 1
             for (int c0 = 0; c0 < BLOCK_N; c0 += 16) {
                 uint32_t v[16];
                 tmem_ld_16(t_row + c0, v);
                 tmem_ld_wait();
                 const int n0 = n_blk * BLOCK_N + c0;
-                if (!mine || m >= p.M || n0 >= p.N) continue;
+                if (m >= p.M || n0 >= p.N) continue;
                 if (EPI == kEpiStore) {
                     uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + static_cast<size_t>(m) * p.N + n0);
                     uint32_t w[8];

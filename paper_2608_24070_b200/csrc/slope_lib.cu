@@ -260,22 +260,7 @@ struct DenseProblem {
     void* out = nullptr;
     const void* mask = nullptr;
     int pdl_mode = 0;
-    int tile_rows = 0;            // rows of the output a tile owns (0 = 128), see DenseGemmParams
 };
-
-// Row count per tile for the skinny adapter products T = X L and dT = dY R^T ([tokens x r], r <= 256):
-// they stream the activations once and are bound by what each SM can pull in, so the tiles should
-// cover every SM in ONE wave.  16384 tokens in 128-row tiles are 128 CTAs on 148 SMs; 112-row tiles
-// (each still computes 128 rows and stores its own 112) are 147.
-static int skinny_tile_rows(int M, int col_tiles, const DeviceInfo& info) {
-    const int tiles128 = (M + kBlockM - 1) / kBlockM;
-    if (col_tiles <= 0 || tiles128 * col_tiles >= info.sm_count) return 0;       // already a full wave (or more)
-    const int m_tiles = info.sm_count / col_tiles;
-    if (m_tiles <= tiles128) return 0;
-    int rows = (M + m_tiles - 1) / m_tiles;
-    rows = (rows + 7) & ~7;
-    return rows >= 64 && rows < kBlockM ? rows : 0;
-}
 
 // One launch of the 1-CTA dense kernel over one or two problems of the same kind.
 template <bool A_MN, bool B_MN, int BLOCK_N, int EPI, int STAGES>
@@ -295,9 +280,7 @@ static slope_status_t launch_dense2(const DenseProblem& q0, const DenseProblem& 
         p[i].M = live ? q.M : 0; p[i].N = q.N; p[i].K = q.K; p[i].k_splits = q.k_splits; p[i].out = q.out;
         p[i].mask = static_cast<const uint8_t*>(q.mask);
         p[i].pdl_mode = q0.pdl_mode;
-        p[i].tile_rows = A_MN ? 0 : q.tile_rows;
-        const int rows = p[i].tile_rows > 0 ? p[i].tile_rows : kBlockM;
-        if (live) tiles += ((q.M + rows - 1) / rows) * ((q.N + BLOCK_N - 1) / BLOCK_N) * q.k_splits;
+        if (live) tiles += ((q.M + kBlockM - 1) / kBlockM) * ((q.N + BLOCK_N - 1) / BLOCK_N) * q.k_splits;
     }
     auto kern = dense_gemm_kernel<A_MN, B_MN, BLOCK_N, EPI, STAGES>;
     if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
@@ -317,8 +300,6 @@ static slope_status_t launch_dense(const void* A, const void* B, int M, int N, i
     DenseProblem q;
     q.A = A; q.B = B; q.M = M; q.N = N; q.K = K; q.k_splits = k_splits; q.out = out; q.mask = mask;
     q.pdl_mode = pdl_mode;
-    // (not beside the consumer of a fused pair: there the launch must stay within the SMs reserved for it)
-    if (EPI == kEpiStore && !A_MN && k_splits == 1 && pdl_mode == 0) q.tile_rows = skinny_tile_rows(M, (N + BLOCK_N - 1) / BLOCK_N, info);
     return launch_dense2<A_MN, B_MN, BLOCK_N, EPI, STAGES>(q, DenseProblem{}, stream, info);
 }
 
