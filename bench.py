@@ -143,11 +143,15 @@ class LayerState:
             self.dT = torch.empty((b, self.r), dtype=bf, device=dev)
             self.dL = torch.empty((self.d_in, self.r), dtype=bf, device=dev)
             self.dR = torch.empty((self.r, self.d_out), dtype=bf, device=dev)
-            self.ws = torch.empty(B.slope_adapter_workspace_bytes(b, self.d_out, self.d_in, self.r),
+            self.ws = torch.empty(max(B.slope_adapter_workspace_bytes(b, self.d_out, self.d_in, self.r),
+                                      B.slope_bwd_dw_adapter_workspace_bytes(b, self.d_out, self.d_in, self.r)),
                                   dtype=torch.uint8, device=dev)
 
 
 OPS = ("prune_24_double", "adapter_T", "linear_fwd", "adapter_bwd", "linear_bwd_dx", "linear_bwd_dw_masked")
+
+
+FUSED_ADAPTER_GRADS = True      # dL, dR ride in the weight-gradient launch (False: separate launches, for comparison)
 
 
 def run_layer(B, s: LayerState, rec=None):
@@ -165,9 +169,17 @@ def run_layer(B, s: LayerState, rec=None):
     if s.r:
         stage("adapter_T", lambda: B.slope_adapter_fwd_bwd(0, s.X, None, s.L, None, s.b, s.d_out, s.d_in, s.r, T=s.T))
         stage("linear_fwd", lambda: B.slope_linear_fwd(s.X, s.Wc_vals, s.Wc_meta, s.d_out, s.Y, s.T, s.R))
-        stage("adapter_bwd", lambda: B.slope_adapter_fwd_bwd(1, s.X, s.dY, s.L, s.R, s.b, s.d_out, s.d_in, s.r,
-                                                             T=s.T, dT=s.dT, dL=s.dL, dR=s.dR, workspace=s.ws))
+        if FUSED_ADAPTER_GRADS:     # dT here; dL and dR come out of the weight-gradient launch below
+            stage("adapter_bwd", lambda: B.slope_adapter_fwd_bwd(2, None, s.dY, None, s.R, s.b, s.d_out, s.d_in, s.r,
+                                                                 dT=s.dT))
+        else:
+            stage("adapter_bwd", lambda: B.slope_adapter_fwd_bwd(1, s.X, s.dY, s.L, s.R, s.b, s.d_out, s.d_in, s.r,
+                                                                 T=s.T, dT=s.dT, dL=s.dL, dR=s.dR, workspace=s.ws))
         stage("linear_bwd_dx", lambda: B.slope_linear_bwd_dx(s.dY, s.WTc_vals, s.WTc_meta, s.d_in, s.dX, s.dT, s.L))
+        if FUSED_ADAPTER_GRADS:
+            stage("linear_bwd_dw_masked", lambda: B.slope_linear_bwd_dw_adapter(s.dY, s.X, s.T, s.dT, s.mask1, s.dWc,
+                                                                                 s.dL, s.dR, s.ws))
+            return
     else:
         stage("linear_fwd", lambda: B.slope_linear_fwd(s.X, s.Wc_vals, s.Wc_meta, s.d_out, s.Y))
         stage("linear_bwd_dx", lambda: B.slope_linear_bwd_dx(s.dY, s.WTc_vals, s.WTc_meta, s.d_in, s.dX))
@@ -383,12 +395,17 @@ def main():
                          "write it to the side file")
     ap.add_argument("--side-file", default=os.path.join(ROOT, "gpurun_out", "bench_extras.json"),
                     help="where the per-stage table and the probe results go (not printed)")
+    ap.add_argument("--separate-adapter-grads", action="store_true",
+                    help="compute dL, dR by their own launches (slope_adapter_fwd_bwd phase 1) instead of inside the "
+                         "weight-gradient launch; for comparison")
     ap.add_argument("--cusparselt-context", action="store_true",
                     help="with --extras: also time the forward GEMMs through torch's semi-structured sparse matmul "
                          "(cuSPARSELt, the library the paper builds on); context only")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "slope" and not args.tokens else args.warmup
 
+    global FUSED_ADAPTER_GRADS
+    FUSED_ADAPTER_GRADS = not args.separate_adapter_grads
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

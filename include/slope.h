@@ -160,6 +160,7 @@ slope_status_t slope_linear_bwd_dw_masked(const void* dY, const void* X, int b, 
  *   phase 0:  T[b x r]  = X L
  *   phase 1:  dT[b x r] = dY R^T,  dL[d_in x r] = X^T dT,  dR[r x d_out] = T^T dY
  *             (dT and T are the bf16 tensors written by this call / phase 0).
+ *   phase 2:  dT[b x r] = dY R^T only (dL and dR then come from slope_linear_bwd_dw_adapter).
  * `workspace` is device scratch of at least slope_adapter_workspace_bytes()
  * bytes, used by phase 1 for fixed-order split-K partial sums; unused pointers
  * of the other phase may be NULL.
@@ -170,6 +171,26 @@ slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY,
                                      int b, int d_out, int d_in, int r,
                                      void* T, void* dT, void* dL, void* dR,
                                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Weight gradient and the adapter's factor gradients in one pass over X and dY:
+ *   dWc          as slope_linear_bwd_dw_masked              Eq. (sparse_backward_weight)
+ *   dL[d_in x r]  = X^T dT,  dR[r x d_out] = T^T dY          chain rule on Eq. (concat), as phase 1
+ * T and dT are the bf16 tensors of slope_adapter_fwd_bwd phases 0 and 2.  All three products contract
+ * over the tokens and the two small ones use the operand tiles the weight-gradient GEMM has staged
+ * anyway, so X and dY are not streamed from HBM a second time (Sec. "Efficient implementation" names
+ * the adapter's extra low-intensity kernel calls as what limits the speed-up).  For r <= 128 and
+ * weight matrices large enough for the 256 x 256 tile kernel the work is one GEMM launch plus the
+ * fixed-order reduction of fp32 partial sums; other shapes run the separate launches.  Same sums as
+ * the separate calls; dL and dR may differ from phase 1 in the last bit because the token
+ * reduction is cut into different slices, and are deterministic like every other output.
+ * `workspace`: device scratch of at least slope_bwd_dw_adapter_workspace_bytes() bytes.
+ */
+size_t slope_bwd_dw_adapter_workspace_bytes(int b, int d_out, int d_in, int r);
+slope_status_t slope_linear_bwd_dw_adapter(const void* dY, const void* X, const void* T, const void* dT,
+                                           int b, int d_out, int d_in, int r,
+                                           const void* mask1_bits, void* dWc_vals, void* dL, void* dR,
+                                           void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Optimizer tail of Algorithm 1 ("sparseAdd", supplementary "Sparse matrix addition"):

@@ -32,6 +32,7 @@ EXPORTS = (
     "slope_prune_nm", "slope_double_prune_nm", "slope_apply_mask",
     "slope_dense_linear_fwd", "slope_dense_linear_bwd_dx", "slope_dense_linear_bwd_dw", "slope_mask_difference",
     "slope_linear_fwd_adapter", "slope_prune_24_double",
+    "slope_bwd_dw_adapter_workspace_bytes", "slope_linear_bwd_dw_adapter",
 )
 
 
@@ -57,6 +58,10 @@ def lib() -> ctypes.CDLL:
         L.slope_double_prune.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp]
         L.slope_prune_24_double.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, vp, vp]
         L.slope_prune_24_double.restype = ci
+        L.slope_bwd_dw_adapter_workspace_bytes.restype = sz
+        L.slope_bwd_dw_adapter_workspace_bytes.argtypes = [ci, ci, ci, ci]
+        L.slope_linear_bwd_dw_adapter.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, vp, sz, vp]
+        L.slope_linear_bwd_dw_adapter.restype = ci
         L.slope_linear_fwd.argtypes = [vp, ci, vp, vp, ci, ci, vp, vp, ci, vp, vp]
         L.slope_linear_bwd_dx.argtypes = [vp, ci, vp, vp, ci, ci, vp, vp, ci, vp, vp]
         L.slope_linear_fwd_adapter.argtypes = [vp, ci, vp, vp, ci, ci, vp, vp, ci, vp, vp, vp]
@@ -183,6 +188,18 @@ def slope_linear_bwd_dw_masked(dY, X, mask1_bits, dWc_vals):
     d_in = X.shape[1]
     _check("slope_linear_bwd_dw_masked", lib().slope_linear_bwd_dw_masked(_ptr(dY), _ptr(X), b, d_out, d_in,
                                                                           _ptr(mask1_bits), _ptr(dWc_vals), _stream()))
+
+
+def slope_bwd_dw_adapter_workspace_bytes(b: int, d_out: int, d_in: int, r: int) -> int:
+    return int(lib().slope_bwd_dw_adapter_workspace_bytes(b, d_out, d_in, r))
+
+
+def slope_linear_bwd_dw_adapter(dY, X, T, dT, mask1_bits, dWc_vals, dL, dR, workspace):
+    b, d_out = dY.shape
+    d_in, r = X.shape[1], T.shape[1]
+    _check("slope_linear_bwd_dw_adapter", lib().slope_linear_bwd_dw_adapter(
+        _ptr(dY), _ptr(X), _ptr(T), _ptr(dT), b, d_out, d_in, r, _ptr(mask1_bits), _ptr(dWc_vals), _ptr(dL), _ptr(dR),
+        _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()))
 
 
 def slope_adapter_workspace_bytes(b: int, d_out: int, d_in: int, r: int) -> int:

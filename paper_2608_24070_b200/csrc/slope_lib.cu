@@ -8,6 +8,7 @@
 #include <mutex>
 #include <utility>
 
+#include "dw_adapter_kernel.cuh"
 #include "gemm_kernels.cuh"
 #include "nm_kernels.cuh"
 #include "prune_kernels.cuh"
@@ -939,11 +940,41 @@ static bool adapter_narrow_tiles(int b, int r, const DeviceInfo& info) {
     return 2 * wide_tiles <= info.sm_count;
 }
 
+// dT[b x r] = dY[b x d_out] * R[r x d_out]^T   (both K contiguous)
+static slope_status_t launch_adapter_dT(const void* dY, const void* R, int b, int d_out, int r, void* dT,
+                                        cudaStream_t stream, const DeviceInfo& info) {
+    return b <= kSkinnyMaxTokens
+               ? launch_skinny(nullptr, b, nullptr, nullptr, r, 0, dY, R, d_out, false, dT, stream, info)
+           : adapter_narrow_tiles(b, r, info)
+               ? launch_dense<false, false, 64, kEpiStore, 9>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info)
+               : launch_dense<false, false, 128, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info);
+}
+
+// dL[d_in x r] = X^T dT and dR^T[d_out x r] = dY^T T: operands stored [K x M] / [K x N] with
+// K = tokens, split into fixed slices; both problems share one launch, their fp32 partial
+// sums are reduced in slice order by one more launch (dR written transposed).
+static slope_status_t launch_adapter_grads(const void* X, const void* dY, const void* T, const void* dT, int b,
+                                           int d_out, int d_in, int r, void* dL, void* dR, void* workspace,
+                                           cudaStream_t stream, const DeviceInfo& info) {
+    float* ws_l = static_cast<float*>(workspace);
+    float* ws_r = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + adapter_partial_bytes(b, d_in, r));
+    DenseProblem ql, qr;
+    ql.A = X; ql.B = dT; ql.M = d_in; ql.N = r; ql.K = b; ql.k_splits = adapter_splits(b, d_in); ql.out = ws_l;
+    qr.A = dY; qr.B = T; qr.M = d_out; qr.N = r; qr.K = b; qr.k_splits = adapter_splits(b, d_out); qr.out = ws_r;
+    slope_status_t st = r <= 64 ? launch_dense2<true, true, 64, kEpiPartial, 6>(ql, qr, stream, info)
+                                : launch_dense2<true, true, 128, kEpiPartial, 6>(ql, qr, stream, info);
+    if (st) return st;
+    const SplitKReduce rl{ws_l, static_cast<uint16_t*>(dL), d_in, r, ql.k_splits, 0};
+    const SplitKReduce rr{ws_r, static_cast<uint16_t*>(dR), d_out, r, qr.k_splits, 1};
+    splitk_reduce_kernel<<<info.sm_count * 4, 256, 0, stream>>>(rl, rr);
+    return launch_result();
+}
+
 slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY, const void* L, const void* R, int b,
                                      int d_out, int d_in, int r, void* T, void* dT, void* dL, void* dR,
                                      void* workspace, size_t workspace_bytes, void* stream_) {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    if (phase != 0 && phase != 1) return SLOPE_ERR_INVALID_ARG;
+    if (phase < 0 || phase > 2) return SLOPE_ERR_INVALID_ARG;
     if (!dims_ok(d_out, d_in) || b < 1 || !rank_ok(r) || r == 0) return SLOPE_ERR_SHAPE;
     DeviceInfo info;
     if (phase == 0) {
@@ -957,33 +988,111 @@ slope_status_t slope_adapter_fwd_bwd(int phase, const void* X, const void* dY, c
                    ? launch_dense<false, true, 64, kEpiStore, 9>(X, L, b, r, d_in, 1, T, nullptr, stream, info)
                    : launch_dense<false, true, 128, kEpiStore, 6>(X, L, b, r, d_in, 1, T, nullptr, stream, info);
     }
+    if (phase == 2) {
+        if (!dY || !R || !dT) return SLOPE_ERR_INVALID_ARG;
+        if (!aligned16(dY) || !aligned16(R) || !aligned16(dT)) return SLOPE_ERR_ALIGNMENT;
+        if (slope_status_t st = check_arch(info)) return st;
+        return launch_adapter_dT(dY, R, b, d_out, r, dT, stream, info);
+    }
     if (!X || !dY || !R || !T || !dT || !dL || !dR || !workspace) return SLOPE_ERR_INVALID_ARG;
     if (!aligned16(X) || !aligned16(dY) || !aligned16(R) || !aligned16(T) || !aligned16(dT) || !aligned16(dL) ||
         !aligned16(dR) || !aligned16(workspace))
         return SLOPE_ERR_ALIGNMENT;
     if (workspace_bytes < slope_adapter_workspace_bytes(b, d_out, d_in, r)) return SLOPE_ERR_INVALID_ARG;
     if (slope_status_t st = check_arch(info)) return st;
-    slope_status_t st;
-    // dT[b x r] = dY[b x d_out] * R[r x d_out]^T   (both K contiguous)
-    st = b <= kSkinnyMaxTokens
-             ? launch_skinny(nullptr, b, nullptr, nullptr, r, 0, dY, R, d_out, false, dT, stream, info)
-         : adapter_narrow_tiles(b, r, info)
-             ? launch_dense<false, false, 64, kEpiStore, 9>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info)
-             : launch_dense<false, false, 128, kEpiStore, 6>(dY, R, b, r, d_out, 1, dT, nullptr, stream, info);
-    if (st) return st;
-    // dL[d_in x r] = X^T dT and dR^T[d_out x r] = dY^T T: operands stored [K x M] / [K x N] with
-    // K = tokens, split into fixed slices; both problems share one launch, their fp32 partial
-    // sums are reduced in slice order by one more launch (dR written transposed).
-    float* ws_l = static_cast<float*>(workspace);
-    float* ws_r = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + adapter_partial_bytes(b, d_in, r));
-    DenseProblem ql, qr;
-    ql.A = X; ql.B = dT; ql.M = d_in; ql.N = r; ql.K = b; ql.k_splits = adapter_splits(b, d_in); ql.out = ws_l;
-    qr.A = dY; qr.B = T; qr.M = d_out; qr.N = r; qr.K = b; qr.k_splits = adapter_splits(b, d_out); qr.out = ws_r;
-    st = r <= 64 ? launch_dense2<true, true, 64, kEpiPartial, 6>(ql, qr, stream, info)
-                 : launch_dense2<true, true, 128, kEpiPartial, 6>(ql, qr, stream, info);
-    if (st) return st;
-    const SplitKReduce rl{ws_l, static_cast<uint16_t*>(dL), d_in, r, ql.k_splits, 0};
-    const SplitKReduce rr{ws_r, static_cast<uint16_t*>(dR), d_out, r, qr.k_splits, 1};
+    if (slope_status_t st = launch_adapter_dT(dY, R, b, d_out, r, dT, stream, info)) return st;
+    return launch_adapter_grads(X, dY, T, dT, b, d_out, d_in, r, dL, dR, workspace, stream, info);
+}
+
+// ------------------------------------------------------------------ masked dW with dL, dR riding along
+namespace slope {
+constexpr int kCarrySplits = 8;            // partial sums per row block of dR^T / dL in the fused launch
+
+struct DwAdapterPlan {
+    bool fused;
+    int splits_r, splits_l;
+};
+
+// The fused launch serves the shapes of the CTA-pair 256 x 256 weight-gradient kernel with r <= 128,
+// provided no tile that carries adapter work lies among the halved items of the last wave (those run
+// at half width, too narrow to serve as the A operand of the dL product).  Everything else takes the
+// separate launches.
+static DwAdapterPlan dw_adapter_plan(int b, int d_out, int d_in, int r, int sm_count) {
+    DwAdapterPlan plan{false, 1, 1};
+    const int num_m = (d_out + 255) / 256, num_n = (d_in + 255) / 256, num_kb = (b + 63) / 64;
+    if (r > 128 || num_m * num_n * 2 <= sm_count) return plan;
+    plan.splits_r = num_n < kCarrySplits ? num_n : kCarrySplits;
+    plan.splits_l = num_m < kCarrySplits ? num_m : kCarrySplits;
+    if (plan.splits_r > num_kb) plan.splits_r = num_kb;
+    if (plan.splits_l > num_kb) plan.splits_l = num_kb;
+    const int num_pairs = sm_count / 2, num_tiles = num_m * num_n;
+    const int full = (num_tiles / num_pairs) * num_pairs, rem = num_tiles - full;
+    if (rem > 0 && 2 * rem <= num_pairs) {
+        for (int tile = full; tile < num_tiles; ++tile) {            // the raster order of raster_tile()
+            const int group_size = kRasterGroupM * num_n, g = tile / group_size, first_m = g * kRasterGroupM;
+            const int gm = num_m - first_m < kRasterGroupM ? num_m - first_m : kRasterGroupM;
+            const int local = tile - g * group_size;
+            const int m = first_m + local % gm, n = local / gm;
+            if (m < plan.splits_l || n < plan.splits_r) return plan;
+        }
+    }
+    plan.fused = true;
+    return plan;
+}
+
+static size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+}  // namespace slope
+
+size_t slope_bwd_dw_adapter_workspace_bytes(int b, int d_out, int d_in, int r) {
+    if (b <= 0 || d_out <= 0 || d_in <= 0 || r <= 0) return 0;
+    const DwAdapterPlan plan = dw_adapter_plan(b, d_out, d_in, r, 148);
+    const size_t fused = align256(static_cast<size_t>(plan.splits_r) * d_out * r * sizeof(float)) +
+                         align256(static_cast<size_t>(plan.splits_l) * d_in * r * sizeof(float));
+    const size_t separate = slope_adapter_workspace_bytes(b, d_out, d_in, r);
+    return fused > separate ? fused : separate;
+}
+
+slope_status_t slope_linear_bwd_dw_adapter(const void* dY, const void* X, const void* T, const void* dT, int b,
+                                           int d_out, int d_in, int r, const void* mask1_bits, void* dWc_vals,
+                                           void* dL, void* dR, void* workspace, size_t workspace_bytes,
+                                           void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!dY || !X || !T || !dT || !mask1_bits || !dWc_vals || !dL || !dR || !workspace) return SLOPE_ERR_INVALID_ARG;
+    if (!dims_ok(d_out, d_in) || b < 1 || !rank_ok(r) || r == 0) return SLOPE_ERR_SHAPE;
+    if (!aligned16(dY) || !aligned16(X) || !aligned16(T) || !aligned16(dT) || !aligned16(mask1_bits) ||
+        !aligned16(dWc_vals) || !aligned16(dL) || !aligned16(dR) || !aligned16(workspace))
+        return SLOPE_ERR_ALIGNMENT;
+    if (workspace_bytes < slope_bwd_dw_adapter_workspace_bytes(b, d_out, d_in, r)) return SLOPE_ERR_INVALID_ARG;
+    DeviceInfo info;
+    if (slope_status_t st = check_arch(info)) return st;
+    const DwAdapterPlan plan = dw_adapter_plan(b, d_out, d_in, r, info.sm_count);
+    if (!plan.fused || info.sm_count != 148) {
+        // the separate launches: masked dW, then the dL / dR partial products and their reduction
+        if (slope_status_t st = slope_linear_bwd_dw_masked(dY, X, b, d_out, d_in, mask1_bits, dWc_vals, stream_)) return st;
+        return launch_adapter_grads(X, dY, T, dT, b, d_out, d_in, r, dL, dR, workspace, stream, info);
+    }
+    using Cfg = DwAdapterCfg<5>;
+    CUtensorMap tmA, tmB, tmT, tmDT;
+    if (!make_tmap(&tmA, dY, b, d_out, 64, 64) || !make_tmap(&tmB, X, b, d_in, 64, 64) ||
+        !make_tmap(&tmT, T, b, r, 64, 64) || !make_tmap(&tmDT, dT, b, r, 64, 64))
+        return SLOPE_ERR_CUDA;
+    DwAdapterParams p = {};
+    p.M = d_out; p.N = d_in; p.K = b; p.r = r;
+    p.splits_r = plan.splits_r; p.splits_l = plan.splits_l;
+    p.dWc = static_cast<uint16_t*>(dWc_vals);
+    p.mask = static_cast<const uint8_t*>(mask1_bits);
+    p.ws_r = static_cast<float*>(workspace);
+    p.ws_l = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) +
+                                      align256(static_cast<size_t>(plan.splits_r) * d_out * r * sizeof(float)));
+    auto kern = dw_adapter_pair_kernel<5>;
+    if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
+    const int tiles = ((d_out + 255) / 256) * ((d_in + 255) / 256);
+    const int max_pairs = info.sm_count / 2;
+    const int pairs = tiles < max_pairs ? tiles : max_pairs;
+    if (slope_status_t st = launch_pairs(kern, 2 * pairs, Cfg::kThreads, Cfg::kSmemBytes, stream, tmA, tmB, tmT, tmDT, p))
+        return st;
+    const SplitKReduce rl{p.ws_l, static_cast<uint16_t*>(dL), d_in, r, plan.splits_l, 0};
+    const SplitKReduce rr{p.ws_r, static_cast<uint16_t*>(dR), d_out, r, plan.splits_r, 1};
     splitk_reduce_kernel<<<info.sm_count * 4, 256, 0, stream>>>(rl, rr);
     return launch_result();
 }

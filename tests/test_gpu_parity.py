@@ -692,3 +692,62 @@ def test_chain_of_fused_adapter_forwards_in_a_cuda_graph(B, oracle):
             assert torch.equal(acts[4].view(torch.int16), eager.view(torch.int16))
     torch.cuda.current_stream().wait_stream(side)
     layers[0].poll()
+
+
+# ------------------------------------------------------------------ weight gradient with dL, dR riding along
+@pytest.mark.parametrize("d_in,d_out,b,r", [
+    (3328, 3072, 1100, 64),      # 13 x 12 tiles on 74 pairs: fused launch, ragged tokens, 8 partial sums each way
+    (3328, 3072, 200, 16),       # fewer k-blocks (4) than carriers: the split count follows the k-blocks
+    (3072, 3328, 520, 128),      # widest rank of the fused launch
+    (3200, 2944, 330, 32),       # d_in, d_out not multiples of 256: half-empty last tile row and column
+    (4096, 4096, 300, 64),       # 256 tiles: the last wave's tiles are halved, none of them a carrier
+    (1024, 1024, 300, 64),       # too few tiles for the 256 x 256 kernel: separate launches
+    (3328, 3072, 300, 256),      # rank beyond the fused launch: separate launches
+])
+def test_weight_gradient_with_adapter_gradients_in_one_call(B, oracle, d_in, d_out, b, r):
+    """slope_linear_bwd_dw_adapter against the oracle (dWc, dL, dR) and against the separate calls
+    (dWc bit for bit: same kernel arithmetic, same reduction order)."""
+    import torch
+
+    W = si.gaussian_bf16((d_out, d_in), 0.02, 701)
+    Xb, dYb = si.gaussian_bf16((b, d_in), 1.0, 702), si.gaussian_bf16((b, d_out), 1.0, 703)
+    Lb, Rb = si.gaussian_bf16((d_in, r), 0.01, 704), si.gaussian_bf16((r, d_out), 0.01, 705)
+    layer = GpuLayer(W, fused_setup=True)
+    X, dY, L, R = dev(B, Xb), dev(B, dYb), dev(B, Lb), dev(B, Rb)
+    T = layer.adapter_T(X, L)
+    bf = torch.bfloat16
+    dT = torch.empty((b, r), dtype=bf, device="cuda")
+    B.slope_adapter_fwd_bwd(2, None, dY, None, R, b, d_out, d_in, r, dT=dT)
+    dT_ref, dL_ref, dR_ref = layer.adapter_bwd(X, dY, L, R, T)
+    assert torch.equal(dT.view(torch.int16), dT_ref.view(torch.int16))
+    dWc_ref = layer.dw(dY, X)
+    nan = float("nan")
+    dWc = torch.full((d_out, d_in // 2), nan, dtype=bf, device="cuda")
+    dL = torch.full((d_in, r), nan, dtype=bf, device="cuda")
+    dR = torch.full((r, d_out), nan, dtype=bf, device="cuda")
+    ws = torch.empty(B.slope_bwd_dw_adapter_workspace_bytes(b, d_out, d_in, r), dtype=torch.uint8, device="cuda")
+    launches = B.slope_launch_count()
+    for _ in range(2):                       # twice: stale partial sums in the workspace must not matter
+        B.slope_linear_bwd_dw_adapter(dY, X, T, dT, layer.mask1, dWc, dL, dR, ws)
+    layer.poll()
+    # one GEMM launch + the reduction when the shape takes the fused launch, else dW, partial products, reduction
+    fused = r <= 128 and d_in >= 2048
+    assert B.slope_launch_count() - launches == 2 * (2 if fused else 3)
+    assert torch.equal(dWc.view(torch.int16), dWc_ref.view(torch.int16))
+    g = lambda t: to_f64(B.bits_from_bf16(t))
+    _, _, mask1 = oracle.prune24(W)
+    orows = si.sample_indices(d_out, 48, 11)
+    jrows = si.sample_indices(d_in, 48, 12)
+    icols = si.sample_indices(d_out, 96, 13)
+    errs = {
+        "dWc": parity_error(g(dWc)[orows], oracle.dw_rows(dYb, Xb, mask1, orows)),
+        "dL": parity_error(g(dL)[jrows], oracle.adapter_dL_rows(Xb, dYb, Rb, jrows), roundings=2),
+        "dR": parity_error(g(dR)[:, icols], oracle.adapter_dR_cols(Xb, Lb, dYb, icols), roundings=2),
+        # against the separate launches: the same sums cut into other slices
+        "dL_vs_separate": rel_fro(g(dL), g(dL_ref)),
+        "dR_vs_separate": rel_fro(g(dR), g(dR_ref)),
+    }
+    print(errs)
+    for k, v in errs.items():
+        assert v <= (REL_TOL if "separate" not in k else 2.5e-3), (k, v, errs)
+    assert np.isfinite(g(dL)).all() and np.isfinite(g(dR)).all()
