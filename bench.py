@@ -151,7 +151,7 @@ class LayerState:
 OPS = ("prune_24_double", "adapter_T", "linear_fwd", "adapter_bwd", "linear_bwd_dx", "linear_bwd_dw_masked")
 
 
-FUSED_ADAPTER_GRADS = True      # dL, dR ride in the weight-gradient launch (False: separate launches, for comparison)
+FUSED_ADAPTER_GRADS = False     # True: dL, dR ride in the weight-gradient launch (measured: no faster, see --fused-adapter-grads)
 
 
 def run_layer(B, s: LayerState, rec=None):
@@ -395,9 +395,9 @@ def main():
                          "write it to the side file")
     ap.add_argument("--side-file", default=os.path.join(ROOT, "gpurun_out", "bench_extras.json"),
                     help="where the per-stage table and the probe results go (not printed)")
-    ap.add_argument("--separate-adapter-grads", action="store_true",
-                    help="compute dL, dR by their own launches (slope_adapter_fwd_bwd phase 1) instead of inside the "
-                         "weight-gradient launch; for comparison")
+    ap.add_argument("--fused-adapter-grads", action="store_true",
+                    help="compute dL, dR inside the weight-gradient launch (slope_linear_bwd_dw_adapter) instead of by "
+                         "their own launches; for comparison (measured: the step is no faster)")
     ap.add_argument("--cusparselt-context", action="store_true",
                     help="with --extras: also time the forward GEMMs through torch's semi-structured sparse matmul "
                          "(cuSPARSELt, the library the paper builds on); context only")
@@ -405,7 +405,7 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "slope" and not args.tokens else args.warmup
 
     global FUSED_ADAPTER_GRADS
-    FUSED_ADAPTER_GRADS = not args.separate_adapter_grads
+    FUSED_ADAPTER_GRADS = args.fused_adapter_grads
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -1071,7 +1071,7 @@ slope_status_t slope_linear_bwd_dw_adapter(const void* dY, const void* X, const 
         if (slope_status_t st = slope_linear_bwd_dw_masked(dY, X, b, d_out, d_in, mask1_bits, dWc_vals, stream_)) return st;
         return launch_adapter_grads(X, dY, T, dT, b, d_out, d_in, r, dL, dR, workspace, stream, info);
     }
-    using Cfg = DwAdapterCfg<5>;
+    using Cfg = DwAdapterCfg<6>;
     CUtensorMap tmA, tmB, tmT, tmDT;
     if (!make_tmap(&tmA, dY, b, d_out, 64, 64) || !make_tmap(&tmB, X, b, d_in, 64, 64) ||
         !make_tmap(&tmT, T, b, r, 64, 64) || !make_tmap(&tmDT, dT, b, r, 64, 64))
@@ -1084,7 +1084,7 @@ slope_status_t slope_linear_bwd_dw_adapter(const void* dY, const void* X, const 
     p.ws_r = static_cast<float*>(workspace);
     p.ws_l = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) +
                                       align256(static_cast<size_t>(plan.splits_r) * d_out * r * sizeof(float)));
-    auto kern = dw_adapter_pair_kernel<5>;
+    auto kern = dw_adapter_pair_kernel<6>;
     if (!set_smem(kern, Cfg::kSmemBytes)) return SLOPE_ERR_CUDA;
     const int tiles = ((d_out + 255) / 256) * ((d_in + 255) / 256);
     const int max_pairs = info.sm_count / 2;
