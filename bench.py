@@ -279,29 +279,33 @@ def replica_throughput(world, flops_per_replica, ms_step):
     return world * flops_per_replica / (ms_step * 1e-3) / 1e12
 
 
+GEMM_SOURCES = ("gemm_kernels.cuh", "ptx.cuh", "slope_lib.cu")     # the GEMM kernels, their PTX wrappers, the kernel choice
+
+
 def kernel_sources_sha256():
-    """Hash of the CUDA sources the library is built from: the ncu-recorded DRAM traffic below is
-    reported only while it describes the kernels that actually ran."""
+    """Hash of the CUDA sources that decide what the two tensor-core kernels do: the ncu-recorded
+    DRAM traffic below is reported only while it describes the kernels that actually ran."""
     import hashlib
 
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2608_24070_b200", "csrc")
-    for name in sorted(os.listdir(csrc)):
-        if name.endswith((".cu", ".cuh")):
-            with open(os.path.join(csrc, name), "rb") as f:
-                h.update(name.encode() + b"\0" + f.read())
+    for name in GEMM_SOURCES:
+        with open(os.path.join(csrc, name), "rb") as f:
+            h.update(name.encode() + b"\0" + f.read())
     return h.hexdigest()
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, from an ncu capture of the two tensor-core
-# kernels at 4096 tokens (one pass, --clock-control none), scaled by tokens to the bench's launch.
-# `sources` is kernel_sources_sha256() of the build that was captured; a build with other sources
-# reports traffic = null (tests/test_bench_line.py fails until the capture is refreshed or cleared).
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the two tensor-core kernels, from a
+# one-pass ncu capture (--clock-control none) of this benchmark's own workload at full size: the 21
+# GEMM launches of one step of c4_llama7b_adapter at 16384 tokens (profiles/ has the summary and the
+# command).  `sources` is kernel_sources_sha256() of the build that was captured; a build with other
+# sources reports traffic = null (tests/test_bench_line.py fails until the capture is refreshed or
+# cleared).
 NCU_TRAFFIC = {
-    "sources": None,
-    "captured_tokens": 4096,
-    "sparse_bytes_per_launch": None,      # mean over the 14 sparse GEMM launches of one step
-    "dense_bytes_per_launch": None,       # mean over the 7 weight-gradient launches of one step
+    "sources": "180996c6082f7d6d09f6ef82df813d953b7d492a5443c3f3ce17f6c78828a191",
+    "captured_tokens": 16384,
+    "sparse_bytes_per_launch": 493127643,     # mean over the 14 sparse GEMM launches of one step
+    "dense_bytes_per_launch": 1391460242,     # mean over the 7 weight-gradient launches of one step
 }
 
 
