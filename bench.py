@@ -186,6 +186,45 @@ def run_layer(B, s: LayerState, rec=None):
     stage("linear_bwd_dw_masked", lambda: B.slope_linear_bwd_dw_masked(s.dY, s.X, s.mask1, s.dWc))
 
 
+def stage_ms_by_graph(torch, B, layers, replays=5):
+    """Device time of every op without the launch gaps that per-call events add: per op one CUDA graph
+    holding that op's launches of all layers back to back (each layer has its own buffers, together far
+    larger than L2, so the launches run cold as in the step), median of `replays` replays."""
+    class Collect:
+        def __init__(self):
+            self.calls = {}
+
+        def __call__(self, op, s, fn):
+            self.calls.setdefault(op, []).append(fn)
+
+    col = Collect()
+    for s in layers:
+        run_layer(B, s, rec=col)                 # collects the closures, launches nothing
+    side = torch.cuda.Stream()
+    out = {}
+    for op, fns in col.calls.items():
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            for fn in fns:
+                fn()
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for fn in fns:
+                    fn()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(replays):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); graph.replay(); e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        out[op] = round(statistics.median(ts), 4)
+    return out
+
+
 def cpu_baseline_sample(wl, seconds_hint=15.0):
     """Time the oracle, as it stands, on the workload: in full where that takes about half a
     minute at the oracle's ~0.02 TFLOP/s (the two small configurations), else on a bounded sample
@@ -371,8 +410,11 @@ def headline(args, wl, b, world, value, ms_step, executed_tflops, launches, cloc
     }
 
 
-def attach_extras(out, dl, e2e, cb):
+def attach_extras(out, dl, e2e, cb, stage_graph=None):
     """Dense comparison, end-to-end run and CPU baseline, cut down to what the line carries."""
+    if stage_graph:
+        out["adapter_share_graph"] = round((stage_graph.get("adapter_T", 0.0) + stage_graph.get("adapter_bwd", 0.0)) /
+                                           sum(stage_graph.values()), 4)
     if dl is not None:
         out["dense_layer"] = {"cublas_ms": dl["dense_ms"], "inhouse_ms": dl["inhouse_dense_ms"], "slope_ms": dl["slope_ms"],
                               "speedup": dl["speedup"], "speedup_vs_inhouse": dl["speedup_vs_inhouse_dense"]}
@@ -590,8 +632,12 @@ def main():
     if rank == 0 and not args.no_extras and world == 1:
         dl = dense_comparison(torch, B, layers, stream)
         side["dense_layer"] = dl
+        sg = stage_ms_by_graph(torch, B, layers)
+        side["stage_ms_graph"] = {"what": "ms per step and op from one CUDA graph per op (all layers back to back, no events "
+                                          "between launches), median of 5 replays", **sg}
         if args.extras:
             side["per_op_200"] = per_op_probe(torch, B, layers, stream, pk)
+            side["hbm_kernels_cold"] = hbm_kernel_probe(torch, B, pk)
             side["optimizer_tail"] = optimizer_tail_probe(torch, B, layers, stream, pk)
             side["burst"] = burst_probe(torch, B, layers, stream, pk)
             side["inference_forward"] = inference_forward_probe(torch, B, wl, pk)
@@ -606,7 +652,7 @@ def main():
         side["e2e"] = e2e
         cb = cpu_baseline_sample(wl)
         side["cpu_baseline"] = cb
-        attach_extras(out, dl, e2e, cb)
+        attach_extras(out, dl, e2e, cb, sg)
     elif rank == 0:
         attach_extras(out, None, None, None)
     if rank == 0:
@@ -669,6 +715,71 @@ def per_op_probe(torch, B, layers, stream, pk, launches=200, warm=20):
             rows.append(row)
     return {"what": f"median of {launches} launches after {warm} warm-ups, each launch between its own CUDA events; "
                     f"peaks: dense {pk['bf16']} TFLOP/s burst ({pk['src']}), sparse := 2 x dense", "rows": rows}
+
+
+def hbm_kernel_probe(torch, B, pk, sets=3, launches=12, replays=5):
+    """The HBM-bound kernels (both pruning passes separately and in one launch, the optimizer tail)
+    timed COLD and without launch gaps: a CUDA graph of `launches` back-to-back launches that cycle
+    through `sets` separate buffer sets (inputs and outputs of one set are 60-450 MB, so a set has left
+    the 126 MB L2 long before its turn comes again), best of `replays` replays.  Events around single
+    launches of 15-50 us kernels add 5-15 us of launch gap each, which is what the per-stage table of
+    the step shows for them."""
+    dev = torch.device("cuda")
+    side = torch.cuda.Stream()
+
+    def graph_us(calls):
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            for fn in calls[:sets]:
+                fn()
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for fn in calls:
+                    fn()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(replays):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); graph.replay(); e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        return best * 1e3 / len(calls)
+
+    rows = []
+    for d_out, d_in in ((4096, 4096), (11008, 4096), (4096, 11008), (13824, 5120)):
+        n = d_out * d_in
+        bufs = []
+        for i in range(sets):
+            W = B.bf16_from_bits(si.gaussian_bf16((d_out, d_in), 0.02, si.seed_for(7, i, "W")), dev)
+            vals, meta, mask1 = B.alloc_compressed(d_out, d_in, dev)
+            valsT, metaT, _ = B.alloc_compressed(d_in, d_out, dev)
+            B.slope_prune_24_double(W, vals, meta, mask1, valsT, metaT, None)
+            bufs.append({"W": W, "vals": vals, "meta": meta, "mask1": mask1, "valsT": valsT, "metaT": metaT,
+                         "g": torch.randn_like(vals), "out": torch.empty_like(vals), "newT": torch.empty_like(valsT)})
+        ops = {
+            "prune_24": (lambda q: B.slope_prune_24(q["W"], q["vals"], q["meta"], q["mask1"]), 3.25),
+            "double_prune": (lambda q: B.slope_double_prune(q["W"], q["mask1"], q["valsT"], q["metaT"], None), 3.25),
+            "prune_24_double": (lambda q: B.slope_prune_24_double(q["W"], q["vals"], q["meta"], q["mask1"], q["valsT"],
+                                                                  q["metaT"], None), 4.375),
+            "sparse_add": (lambda q: B.slope_sparse_add(q["g"], q["vals"], 1.0 / 1024.0, 0.01, q["out"]), 3.0),
+            "update_sparse_matrix": (lambda q: B.slope_update_sparse_matrix(q["vals"], q["mask1"], q["metaT"], q["newT"]),
+                                     2.25),
+        }
+        for op, (fn, bytes_per_el) in ops.items():
+            us = graph_us([lambda fn=fn, q=bufs[i % sets]: fn(q) for i in range(launches)])
+            gbs = bytes_per_el * n / us / 1e3
+            rows.append({"op": op, "d_out": d_out, "d_in": d_in, "us": round(us, 2), "bytes_per_element": bytes_per_el,
+                         "gbs": round(gbs, 1), "frac_of_hbm_peak": round(gbs / pk["hbm_gbs"], 4)})
+        del bufs
+    st = B.slope_poll_status()
+    if st != 0:
+        raise SystemExit(f"device status after the HBM kernel probe: {B.slope_status_string(st)}")
+    return {"what": f"us per launch from a CUDA graph of {launches} launches cycling through {sets} buffer sets (cold), best "
+                    f"of {replays} replays; algorithmic bytes per weight element as listed; HBM peak {pk['hbm_gbs']} GB/s "
+                    f"({pk['src']})", "rows": rows}
 
 
 def optimizer_tail_probe(torch, B, layers, stream, pk, reps=20):

@@ -46,7 +46,7 @@ def _worst_case_line():
     cb = {"value": 0.020512345, "unit": "TFLOP/s", "cores": 128, "kind": "oracle", "seconds": 15.21,
           "sample": "bounded sample: down 11008->4096 b=16384: fwd+dX 1024 token rows, dW 1024 rows",
           "full_workload": False, "extrapolated_step_seconds": 990.1, "extrapolation": "e" * 200}
-    bench.attach_extras(out, dl, e2e, cb)
+    bench.attach_extras(out, dl, e2e, cb, {op: 12.3456 for op in bench.OPS})
     return out, bench.compact_line(out)
 
 
