@@ -63,6 +63,16 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     assert lib.slope_prune_nm(a, 128, 128, 4, 4, a, null, null) == 2                   # n must be below m
     assert lib.slope_sparse_add(a, a, 1.0, 1.0, 128, 100, a, null) == 2
     assert lib.slope_update_sparse_matrix(a, a, a, 128, 128, null, null) == 1
+    # the one-launch set-up and the weight gradient with the adapter gradients riding along
+    assert lib.slope_prune_24_double(a, 128, 128, a, a, null, a, null, null, null) == 1          # a compressed copy missing
+    assert lib.slope_prune_24_double(a, 128, 192, a, a, null, a, a, null, null) == 2             # d_in not a multiple of 128
+    assert lib.slope_prune_24_double(a, 128, 128, a, a, a + 8, a, a, null, null) == 3            # misaligned mask
+    assert lib.slope_bwd_dw_adapter_workspace_bytes(16384, 4096, 4096, 64) >= lib.slope_adapter_workspace_bytes(16384, 4096, 4096, 64)
+    assert lib.slope_bwd_dw_adapter_workspace_bytes(16384, 4096, 4096, 0) == 0
+    assert lib.slope_linear_bwd_dw_adapter(a, a, a, a, 16, 128, 128, 16, a, a, a, a, a, 0, null) == 1   # workspace too small
+    assert lib.slope_linear_bwd_dw_adapter(a, a, a, a, 16, 128, 128, 24, a, a, a, a, a, 1 << 30, null) == 2   # rank
+    assert lib.slope_linear_bwd_dw_adapter(a, a, a, null, 16, 128, 128, 16, a, a, a, a, a, 1 << 30, null) == 1   # dT missing
+    assert lib.slope_adapter_fwd_bwd(2, null, a, null, a, 16, 128, 128, 16, null, null, null, null, null, 0, null) == 1  # phase 2 needs dT
 
 
 def test_binding_refuses_to_run_without_the_library(monkeypatch, tmp_path):
