@@ -341,10 +341,10 @@ def kernel_sources_sha256():
 # sources reports traffic = null (tests/test_bench_line.py fails until the capture is refreshed or
 # cleared).
 NCU_TRAFFIC = {
-    "sources": "180996c6082f7d6d09f6ef82df813d953b7d492a5443c3f3ce17f6c78828a191",
+    "sources": "38cb175c54c14813d37e626220845ad8cfddce57cf9e5b2bcdfaaf0f38d98251",
     "captured_tokens": 16384,
-    "sparse_bytes_per_launch": 493127643,     # mean over the 14 sparse GEMM launches of one step
-    "dense_bytes_per_launch": 1391460242,     # mean over the 7 weight-gradient launches of one step
+    "sparse_bytes_per_launch": 493483246,     # mean over the 14 sparse GEMM launches of one step
+    "dense_bytes_per_launch": 1388653641,     # mean over the 7 weight-gradient launches of one step
 }
 
 
@@ -357,7 +357,7 @@ def recorded_traffic(kind, wl_key, tokens):
     if v is None:
         return None, "no ncu capture recorded for this kernel"
     scale = tokens / NCU_TRAFFIC["captured_tokens"]
-    return round(v * scale), f"ncu at {NCU_TRAFFIC['captured_tokens']} tokens x{scale:g}, sources {NCU_TRAFFIC['sources'][:12]}"
+    return round(v * scale), f"ncu {NCU_TRAFFIC['captured_tokens']} tok x{scale:g}, src {NCU_TRAFFIC['sources'][:8]}"
 
 
 SM_COUNT = 148
@@ -387,34 +387,32 @@ def compact_line(out):
 
 
 def headline(args, wl, b, world, value, ms_step, executed_tflops, launches, clocks_full, roofline, other,
-             ms_step_staged, stage_ms):
+             ms_step_staged, stage_ms, kernel_mhz=None):
     """The compact record (pure function of measured numbers: also exercised without a GPU)."""
     clocks = None
     if clocks_full is not None:
         clocks = {k: clocks_full.get(k) for k in ("sm_mhz", "sm_mhz_min", "sm_max_mhz", "power_w_max", "reasons")}
+        clocks["kernel_mhz"] = kernel_mhz
     adapter_ms = stage_ms.get("adapter_T", 0.0) + stage_ms.get("adapter_bwd", 0.0)
     return {
         "impl": "slope", "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl.key, "tokens": b, "rank": wl.rank, "parallelism": "replicas" if world > 1 else "1 GPU",
-                   "l2": "inputs larger than L2",
-                   "step": f"prune+double prune, adapters, fwd, dX, masked dW x {len(wl.layers)} layers"},
+                   "l2": "inputs > L2",
+                   "step": f"prune x2, adapters, fwd, dX, masked dW x {len(wl.layers)} layers"},
         "executed_tflops": round(executed_tflops, 2),
         "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline,
         "roofline_other": None if other is None else {k: other[k] for k in (
-            "kernel", "achieved", "peak", "frac", "frac_sustained", "frac_clock", "kernel_ms_per_step")},
+            "kernel", "achieved", "peak", "frac", "frac_sustained", "frac_kernel_clock", "kernel_ms_per_step")},
         "ms_per_step_staged": round(ms_step_staged, 4),
         "stage_ms": stage_ms,
         "adapter_share": round(adapter_ms / sum(stage_ms.values()), 4) if stage_ms else None,
     }
 
 
-def attach_extras(out, dl, e2e, cb, stage_graph=None):
+def attach_extras(out, dl, e2e, cb):
     """Dense comparison, end-to-end run and CPU baseline, cut down to what the line carries."""
-    if stage_graph:
-        out["adapter_share_graph"] = round((stage_graph.get("adapter_T", 0.0) + stage_graph.get("adapter_bwd", 0.0)) /
-                                           sum(stage_graph.values()), 4)
     if dl is not None:
         out["dense_layer"] = {"cublas_ms": dl["dense_ms"], "inhouse_ms": dl["inhouse_dense_ms"], "slope_ms": dl["slope_ms"],
                               "speedup": dl["speedup"], "speedup_vs_inhouse": dl["speedup_vs_inhouse_dense"]}
@@ -526,6 +524,9 @@ def main():
     launches = B.slope_launch_count() - launches0
     ms_total = replica_max_ms(torch, dist, ev0.elapsed_time(ev1), dev)
     check_status("the timed region")
+    # the SM clock inside the last sparse / dense tile-kernel launch of the timed region (the power
+    # limiter moves it within microseconds; nvidia-smi's samples average over all kernels of the step)
+    kernel_mhz = {"sparse": round(B.slope_kernel_clock_mhz(0), 1), "dense": round(B.slope_kernel_clock_mhz(1), 1)}
     ms_step = ms_total / args.steps
     value = replica_throughput(world, de_flops, ms_step)
 
@@ -607,9 +608,11 @@ def main():
         r = {"kernel": kernel, "bound": "tensor", "achieved": round(tf, 1), "peak": round(peak_burst, 1),
              "unit": "TFLOP/s", "frac": round(tf / peak_burst, 4), "traffic": traffic,
              "algorithmic_bytes": round(nbytes / n), "traffic_source": source,
-             "peak_source": ("2 x " if kind == "sparse" else "") + f"{pk['src']} burst cuBLAS bf16",
+             "peak_source": ("2x " if kind == "sparse" else "") + f"{pk['src']} burst cuBLAS",
              "frac_sustained": round(tf / peak_sustained, 4), "frac_datasheet": round(tf / datasheet, 4),
              "frac_clock": round(fl / sec / (sm_mhz * 1e6 * SM_COUNT * flop_per_clk_sm), 4) if sm_mhz else None,
+             "frac_kernel_clock": round(fl / sec / (kernel_mhz[kind] * 1e6 * SM_COUNT * flop_per_clk_sm), 4)
+             if kernel_mhz[kind] else None,
              "tflop_per_step": round(fl / 1e12, 4), "kernel_ms_per_step": round(sec * 1e3, 4), "launches_per_step": n}
         return r
 
@@ -624,8 +627,9 @@ def main():
     other = roofline_dense if sparse_dominant else roofline_sparse
     stage_ms = {k: round(v, 3) for k, v in per_op_ms.items() if v > 0}
 
+    line_roofline = {k: v for k, v in roofline.items() if k not in ("launches_per_step",)}
     out = headline(args, wl, b, world, value, ms_step, world * ex_flops / (ms_step * 1e-3) / 1e12, launches,
-                   clocks_full, roofline, other, ms_step_staged, stage_ms)
+                   clocks_full, line_roofline, other, ms_step_staged, stage_ms, kernel_mhz)
 
     side = {"headline": dict(out), "clocks": clocks_full, "roofline_sparse": roofline_sparse,
             "roofline_dense": roofline_dense, "stages": stage_rows}
@@ -634,7 +638,9 @@ def main():
         side["dense_layer"] = dl
         sg = stage_ms_by_graph(torch, B, layers)
         side["stage_ms_graph"] = {"what": "ms per step and op from one CUDA graph per op (all layers back to back, no events "
-                                          "between launches), median of 5 replays", **sg}
+                                          "between launches), median of 5 replays", **sg,
+                                  "adapter_share": round((sg.get("adapter_T", 0.0) + sg.get("adapter_bwd", 0.0)) /
+                                                         sum(sg.values()), 4)}
         if args.extras:
             side["per_op_200"] = per_op_probe(torch, B, layers, stream, pk)
             side["hbm_kernels_cold"] = hbm_kernel_probe(torch, B, pk)
@@ -652,7 +658,7 @@ def main():
         side["e2e"] = e2e
         cb = cpu_baseline_sample(wl)
         side["cpu_baseline"] = cb
-        attach_extras(out, dl, e2e, cb, sg)
+        attach_extras(out, dl, e2e, cb)
     elif rank == 0:
         attach_extras(out, None, None, None)
     if rank == 0:

@@ -32,7 +32,7 @@ EXPORTS = (
     "slope_prune_nm", "slope_double_prune_nm", "slope_apply_mask",
     "slope_dense_linear_fwd", "slope_dense_linear_bwd_dx", "slope_dense_linear_bwd_dw", "slope_mask_difference",
     "slope_linear_fwd_adapter", "slope_prune_24_double",
-    "slope_bwd_dw_adapter_workspace_bytes", "slope_linear_bwd_dw_adapter",
+    "slope_bwd_dw_adapter_workspace_bytes", "slope_linear_bwd_dw_adapter", "slope_kernel_clock_mhz",
 )
 
 
@@ -95,6 +95,8 @@ def lib() -> ctypes.CDLL:
         L.slope_selftest_wait_timeout.argtypes = [ctypes.c_uint, vp, vp]
         L.slope_selftest_wait_timeout.restype = ci
         L.slope_poll_status.argtypes = [vp]
+        L.slope_kernel_clock_mhz.argtypes = [ci, vp, ctypes.POINTER(ctypes.c_double)]
+        L.slope_kernel_clock_mhz.restype = ci
         L.slope_launch_count.restype = ctypes.c_ulonglong
         L.slope_status_string.restype = ctypes.c_char_p
         L.slope_status_string.argtypes = [ci]
@@ -200,6 +202,13 @@ def slope_linear_bwd_dw_adapter(dY, X, T, dT, mask1_bits, dWc_vals, dL, dR, work
     _check("slope_linear_bwd_dw_adapter", lib().slope_linear_bwd_dw_adapter(
         _ptr(dY), _ptr(X), _ptr(T), _ptr(dT), b, d_out, d_in, r, _ptr(mask1_bits), _ptr(dWc_vals), _ptr(dL), _ptr(dR),
         _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()))
+
+
+def slope_kernel_clock_mhz(kind: int) -> float:
+    """SM clock (MHz) inside the last sparse (kind 0) / dense CTA-pair (kind 1) tile-kernel launch."""
+    mhz = ctypes.c_double(0.0)
+    _check("slope_kernel_clock_mhz", lib().slope_kernel_clock_mhz(int(kind), _stream(), ctypes.byref(mhz)))
+    return float(mhz.value)
 
 
 def slope_adapter_workspace_bytes(b: int, d_out: int, d_in: int, r: int) -> int:

@@ -487,6 +487,8 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             PipeState ps;
             bool ok = true;
             int it = 0;
+            ClockProbe probe;
+            if (pair_id == 0) probe.begin();
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
                 const int width = token_tile_width(p.Ntok, (tile / num_m) * BLOCK_N, BLOCK_N);
                 const uint32_t idesc_sp = make_idesc_bf16(2 * kBlockM, width, false, false, true);
@@ -528,6 +530,7 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 }
                 if (ok) umma_commit_pair(&tfull_bar[acc], 3);
             }
+            if (pair_id == 0) probe.end(kClockSparse);
         }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
@@ -731,6 +734,8 @@ dense_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
             bool ok = true;
             int it = 0;
             PairWork w;
+            ClockProbe probe;
+            if (pair_id == 0) probe.begin();
             for (int item = pair_id; ok && pair_work<BLOCK_N, kSplitTail>(item, num_pairs, num_m, num_n, w);
                  item += num_pairs, ++it) {
                 const uint32_t idesc = w.width == BLOCK_N ? idesc_full : idesc_half;
@@ -757,6 +762,7 @@ dense_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
                 }
                 if (ok) umma_commit_pair(&tfull_bar[acc], 3);
             }
+            if (pair_id == 0) probe.end(kClockDense);
         }
     } else {
         const int q = warp & 3;
@@ -1043,6 +1049,8 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             PipeState ps;                                     // stage that sub-tile 0 consumes next
             bool ok = true;
             int it = 0;
+            ClockProbe probe;
+            if (pair_id == 0) probe.begin();
             for (int tile = pair_id; ok && tile < num_tiles; tile += num_pairs, ++it) {
                 int mt, n_blk;
                 bool first_unused;
@@ -1093,6 +1101,7 @@ sparse_gemm_quad_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 }
                 if (ok && nsub == 1) umma_commit_pair(&tfull_bar[1], 3);        // keep both barriers in phase
             }
+            if (pair_id == 0) probe.end(kClockSparse);
         }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..9, both CTAs)

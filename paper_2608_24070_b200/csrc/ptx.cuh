@@ -24,6 +24,30 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
     return t;
 }
 
+// SM clock as the tensor-core kernels see it.  Under load the hardware's power limiter pulls the SM
+// clock down within the first kernel of a burst (1965 MHz idle, ~1.4 GHz in the first sparse GEMM
+// after a pause, 1.1-1.2 GHz in a sustained step) -- faster than any host-side sampler shows -- so a
+// fraction of the tensor peak only means something next to the clock the kernel actually ran at.
+// The MMA-issuing thread of the first CTA pair of a launch records its SM cycle counter and the
+// global nanosecond timer when it starts and when it has issued its last MMA; the host reads the
+// last launch's pair with slope_kernel_clock_mhz().  Two counter reads and one store per launch.
+constexpr int kClockSparse = 0, kClockDense = 1;
+__device__ unsigned long long g_kernel_clock[2][2];        // [kind][cycles, nanoseconds] of the last launch
+struct ClockProbe {
+    unsigned long long c0, t0;
+    __device__ __forceinline__ void begin() {
+        c0 = clock64();
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    }
+    __device__ __forceinline__ void end(int kind) const {
+        unsigned long long t1;
+        const unsigned long long c1 = clock64();
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+        g_kernel_clock[kind][0] = c1 - c0;
+        g_kernel_clock[kind][1] = t1 - t0;
+    }
+};
+
 __device__ __forceinline__ bool elect_one() {
     uint32_t pred;
     asm volatile(

@@ -720,6 +720,15 @@ const char* slope_status_string(slope_status_t s) {
     return "unknown status";
 }
 
+slope_status_t slope_kernel_clock_mhz(int kind, void* stream, double* mhz_host) {
+    if ((kind != 0 && kind != 1) || !mhz_host) return SLOPE_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return SLOPE_ERR_CUDA;
+    unsigned long long v[2][2];
+    if (cudaMemcpyFromSymbol(v, g_kernel_clock, sizeof(v)) != cudaSuccess) return SLOPE_ERR_CUDA;
+    *mhz_host = v[kind][1] ? static_cast<double>(v[kind][0]) / static_cast<double>(v[kind][1]) * 1e3 : 0.0;
+    return SLOPE_OK;
+}
+
 slope_status_t slope_poll_status(void* stream) {
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return SLOPE_ERR_CUDA;
     int st = 0;

@@ -30,15 +30,16 @@ def _worst_case_line():
     roof = {"kernel": "sparse_gemm_quad/pair_kernel (fwd, dX)", "bound": "tensor",
             "achieved": 2507.123, "peak": 3386.0, "unit": "TFLOP/s", "frac": 0.7404, "traffic": 507123456,
             "algorithmic_bytes": 398123456,
-            "traffic_source": "ncu at 4096 tokens x4, sources 0123456789ab",
-            "peak_source": "2 x measured burst cuBLAS bf16", "frac_sustained": 0.8906,
-            "frac_datasheet": 0.5571, "frac_clock": 0.7312, "tflop_per_step": 13.4269,
-            "kernel_ms_per_step": 5.3571, "launches_per_step": 14}
+            "traffic_source": "ncu 16384 tok x1, src 01234567", "peak_source": "2x measured burst cuBLAS",
+            "frac_sustained": 0.8906,
+            "frac_datasheet": 0.5571, "frac_clock": 0.7312, "frac_kernel_clock": 0.8912, "tflop_per_step": 13.4269,
+            "kernel_ms_per_step": 5.3571}
     other = dict(roof, kernel="dense_gemm_pair_kernel (masked dW)")
     clocks = {"sm_mhz": 1417.5, "sm_mhz_min": 1012.5, "sm_max_mhz": 1965.0, "power_w_max": 1002.02, "samples": 1234,
               "window": "x", "reasons": ["hw_slowdown", "hw_thermal_slowdown", "sw_power_cap", "sw_thermal_slowdown"]}
     stage_ms = {op: 12.345 for op in bench.OPS}
-    out = bench.headline(args, wl, 16384, 8, 12345.67, 11.6123, 1234.56, 123456, clocks, roof, other, 11.7123, stage_ms)
+    out = bench.headline(args, wl, 16384, 8, 12345.67, 11.6123, 1234.56, 123456, clocks, roof, other, 11.7123, stage_ms,
+                         {"sparse": 1172.5, "dense": 1095.5})
     dl = {"dense_ms": 14.4512, "inhouse_dense_ms": 13.9012, "slope_ms": 10.0212, "speedup": 1.443,
           "speedup_vs_inhouse_dense": 1.387}
     e2e = {"value": 431.12, "unit": "TFLOP/s", "ms_per_step": 47.291, "h2d_bytes_per_step": 2560000000,
@@ -46,7 +47,7 @@ def _worst_case_line():
     cb = {"value": 0.020512345, "unit": "TFLOP/s", "cores": 128, "kind": "oracle", "seconds": 15.21,
           "sample": "bounded sample: down 11008->4096 b=16384: fwd+dX 1024 token rows, dW 1024 rows",
           "full_workload": False, "extrapolated_step_seconds": 990.1, "extrapolation": "e" * 200}
-    bench.attach_extras(out, dl, e2e, cb, {op: 12.3456 for op in bench.OPS})
+    bench.attach_extras(out, dl, e2e, cb)
     return out, bench.compact_line(out)
 
 

@@ -751,3 +751,21 @@ def test_weight_gradient_with_adapter_gradients_in_one_call(B, oracle, d_in, d_o
     for k, v in errs.items():
         assert v <= (REL_TOL if "separate" not in k else 2.5e-3), (k, v, errs)
     assert np.isfinite(g(dL)).all() and np.isfinite(g(dR)).all()
+
+
+def test_kernel_clock_diagnostic_reports_a_plausible_sm_clock(B, oracle):
+    """slope_kernel_clock_mhz: the SM clock measured inside the last sparse / dense tile-kernel launch."""
+    import torch
+
+    W = si.gaussian_bf16((1024, 1024), 0.02, 801)
+    layer = GpuLayer(W, fused_setup=True)
+    X = dev(B, si.gaussian_bf16((2048, 1024), 1.0, 802))
+    dY = dev(B, si.gaussian_bf16((2048, 1024), 1.0, 803))
+    layer.fwd(X)                               # a CTA-pair sparse tile kernel
+    layer.dw(dY, X)                            # the CTA-pair dense kernel
+    layer.poll()
+    for kind in (0, 1):
+        mhz = B.slope_kernel_clock_mhz(kind)
+        assert 300.0 < mhz < 2100.0, (kind, mhz)        # B200: at most 1965 MHz, ~1.1-1.5 GHz under tensor load
+    with pytest.raises(B.SlopeError):
+        B.slope_kernel_clock_mhz(2)
