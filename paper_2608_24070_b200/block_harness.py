@@ -51,8 +51,7 @@ class SlopeLinear:
         self.d_out, self.d_in = W.shape
         self.Wc_vals, self.Wc_meta, self.mask1 = B.alloc_compressed(self.d_out, self.d_in)
         self.WTc_vals, self.WTc_meta, _ = B.alloc_compressed(self.d_in, self.d_out)
-        B.slope_prune_24(W, self.Wc_vals, self.Wc_meta, self.mask1)
-        B.slope_double_prune(W, self.mask1, self.WTc_vals, self.WTc_meta, None)
+        B.slope_prune_24_double(W, self.Wc_vals, self.Wc_meta, self.mask1, self.WTc_vals, self.WTc_meta, None)
         self.L, self.R = L, R
         self.r = 0 if L is None else L.shape[1]
         self.dWc = torch.empty_like(self.Wc_vals)

@@ -115,29 +115,31 @@ double_prune_nm_kernel(const uint4* W, const uint8_t* __restrict__ mask1, int d_
         const size_t h = idx / row_u4, c = idx % row_u4;
         const size_t base = h * M * row_u4 + c;
         uint32_t w[M][4];
-        uint32_t m1[M];
+        // first-pass mask bytes and second-pass keep bits of the M rows, four rows per register (the
+        // 16-row pattern otherwise needs more than 255 registers and spills)
+        constexpr int kPacked = (M + 3) / 4;
+        uint32_t m1p[kPacked], keep_p[kPacked];
+#pragma unroll
+        for (int i = 0; i < kPacked; ++i) { m1p[i] = 0; keep_p[i] = 0; }
 #pragma unroll
         for (int t = 0; t < M; ++t) {
             const uint4 v = __ldcs(W + base + static_cast<size_t>(t) * row_u4);
             w[t][0] = v.x; w[t][1] = v.y; w[t][2] = v.z; w[t][3] = v.w;
-            m1[t] = mask1[base + static_cast<size_t>(t) * row_u4];
+            m1p[t >> 2] |= static_cast<uint32_t>(mask1[base + static_cast<size_t>(t) * row_u4]) << (8 * (t & 3));
         }
-        uint32_t keep_row[M];
-#pragma unroll
-        for (int t = 0; t < M; ++t) keep_row[t] = 0;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             uint32_t key[M];
 #pragma unroll
             for (int t = 0; t < M; ++t)
-                key[t] = (m1[t] >> k) & 1u ? (w[t][k >> 1] >> (16 * (k & 1))) & 0x7FFFu : 0u;
+                key[t] = (m1p[t >> 2] >> (8 * (t & 3) + k)) & 1u ? (w[t][k >> 1] >> (16 * (k & 1))) & 0x7FFFu : 0u;
             const uint32_t keep = keep_n_of_m<M, (M >= 16)>(key, n);
 #pragma unroll
-            for (int t = 0; t < M; ++t) keep_row[t] |= ((keep >> t) & 1u) << k;
+            for (int t = 0; t < M; ++t) keep_p[t >> 2] |= ((keep >> t) & 1u) << (8 * (t & 3) + k);
         }
 #pragma unroll
         for (int t = 0; t < M; ++t) {
-            const uint32_t both = keep_row[t] & m1[t];
+            const uint32_t both = ((keep_p[t >> 2] & m1p[t >> 2]) >> (8 * (t & 3))) & 0xFFu;
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const uint32_t lo = (both >> (2 * q)) & 1u ? 0x0000FFFFu : 0u;
