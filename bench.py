@@ -437,7 +437,7 @@ def main():
                     help="also run the probe suite (per-op medians over 200 launches, burst, optimizer tail, N:M, "
                          "inference forward, decode block, shape sweep, small configurations, decoder block) and "
                          "write it to the side file")
-    ap.add_argument("--side-file", default=os.path.join(ROOT, "gpurun_out", "bench_extras.json"),
+    ap.add_argument("--side-file", default=os.path.join(ROOT, "bench_extras.json"),
                     help="where the per-stage table and the probe results go (not printed)")
     ap.add_argument("--fused-adapter-grads", action="store_true",
                     help="compute dL, dR inside the weight-gradient launch (slope_linear_bwd_dw_adapter) instead of by "
