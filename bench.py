@@ -341,10 +341,10 @@ def kernel_sources_sha256():
 # sources reports traffic = null (tests/test_bench_line.py fails until the capture is refreshed or
 # cleared).
 NCU_TRAFFIC = {
-    "sources": "38cb175c54c14813d37e626220845ad8cfddce57cf9e5b2bcdfaaf0f38d98251",
+    "sources": "d5acd425bbfd044583584d97afe9e5d7629458da7028d2bf4560be18c8dc3a9a",
     "captured_tokens": 16384,
-    "sparse_bytes_per_launch": 493483246,     # mean over the 14 sparse GEMM launches of one step
-    "dense_bytes_per_launch": 1388653641,     # mean over the 7 weight-gradient launches of one step
+    "sparse_bytes_per_launch": 493724818,     # mean over the 14 sparse GEMM launches of one step
+    "dense_bytes_per_launch": 1381888439,     # mean over the 7 weight-gradient launches of one step
 }
 
 
@@ -512,6 +512,7 @@ def main():
     launches0 = B.slope_launch_count()
     barrier()
     torch.cuda.synchronize()
+    B.slope_kernel_clock_mhz(0), B.slope_kernel_clock_mhz(1)        # start the in-kernel clock averages here
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t_begin = time.time()
     ev0.record(stream)
@@ -524,7 +525,7 @@ def main():
     launches = B.slope_launch_count() - launches0
     ms_total = replica_max_ms(torch, dist, ev0.elapsed_time(ev1), dev)
     check_status("the timed region")
-    # the SM clock inside the last sparse / dense tile-kernel launch of the timed region (the power
+    # the mean SM clock inside the sparse / dense tile-kernel launches of the timed region (the power
     # limiter moves it within microseconds; nvidia-smi's samples average over all kernels of the step)
     kernel_mhz = {"sparse": round(B.slope_kernel_clock_mhz(0), 1), "dense": round(B.slope_kernel_clock_mhz(1), 1)}
     ms_step = ms_total / args.steps

@@ -308,14 +308,16 @@ slope_status_t slope_meta_to_canonical(const void* meta_hw, int rows, int cols,
 slope_status_t slope_selftest_wait_timeout(unsigned int limit_us, void* gave_up_flag, void* stream);
 
 /*
- * Diagnostic (no counterpart in the paper): the SM clock in MHz that the last launch of a
- * tensor-core tile kernel actually ran at -- kind 0: the sparse forward / input-gradient tile
- * kernels, kind 1: the dense CTA-pair kernel (masked weight gradient, dense layer).  The MMA-issuing
- * thread of the launch's first CTA pair reads its SM cycle counter and the global timer at its
- * first and after its last MMA; the ratio is the clock.  Under the power cap the hardware lowers the
- * SM clock within microseconds of the tensor cores becoming busy, which no host-side sampler
- * resolves; a fraction of the tensor peak is only meaningful beside this clock.  Synchronises
- * `stream`; *mhz_host (host memory) is 0 when no such kernel has run yet.
+ * Diagnostic (no counterpart in the paper): the mean SM clock in MHz that the tensor-core tile
+ * kernels actually ran at, over all launches that completed on the current device since the
+ * previous call for that kind (or since the library was loaded) -- kind 0: the sparse forward /
+ * input-gradient tile kernels, kind 1: the dense CTA-pair kernel (masked weight gradient, dense
+ * layer).  The MMA-issuing thread of each launch's first CTA pair reads its SM cycle counter and
+ * the global timer at its first and after its last MMA; the ratio of the summed differences is the
+ * clock, weighted by kernel time.  Under the power cap the hardware lowers the SM clock within
+ * microseconds of the tensor cores becoming busy, which no host-side sampler resolves; a fraction of
+ * the tensor peak is only meaningful beside this clock.  Synchronises `stream`; *mhz_host (host
+ * memory) is 0 when no such kernel has run since the previous call.
  */
 slope_status_t slope_kernel_clock_mhz(int kind, void* stream, double* mhz_host);
 

@@ -205,7 +205,8 @@ def slope_linear_bwd_dw_adapter(dY, X, T, dT, mask1_bits, dWc_vals, dL, dR, work
 
 
 def slope_kernel_clock_mhz(kind: int) -> float:
-    """SM clock (MHz) inside the last sparse (kind 0) / dense CTA-pair (kind 1) tile-kernel launch."""
+    """Mean SM clock (MHz) inside the sparse (kind 0) / dense CTA-pair (kind 1) tile-kernel launches
+    since the previous call for that kind."""
     mhz = ctypes.c_double(0.0)
     _check("slope_kernel_clock_mhz", lib().slope_kernel_clock_mhz(int(kind), _stream(), ctypes.byref(mhz)))
     return float(mhz.value)

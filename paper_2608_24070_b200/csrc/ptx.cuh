@@ -28,11 +28,12 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
 // clock down within the first kernel of a burst (1965 MHz idle, ~1.4 GHz in the first sparse GEMM
 // after a pause, 1.1-1.2 GHz in a sustained step) -- faster than any host-side sampler shows -- so a
 // fraction of the tensor peak only means something next to the clock the kernel actually ran at.
-// The MMA-issuing thread of the first CTA pair of a launch records its SM cycle counter and the
-// global nanosecond timer when it starts and when it has issued its last MMA; the host reads the
-// last launch's pair with slope_kernel_clock_mhz().  Two counter reads and one store per launch.
+// The MMA-issuing thread of the first CTA pair of a launch reads its SM cycle counter and the
+// global nanosecond timer when it starts and when it has issued its last MMA and adds both
+// differences to running totals; slope_kernel_clock_mhz() turns the growth of the totals since its
+// previous call into a mean clock.  Four counter reads and two atomic adds per launch.
 constexpr int kClockSparse = 0, kClockDense = 1;
-__device__ unsigned long long g_kernel_clock[2][2];        // [kind][cycles, nanoseconds] of the last launch
+__device__ unsigned long long g_kernel_clock[2][2];        // [kind][cycles, nanoseconds], running totals
 struct ClockProbe {
     unsigned long long c0, t0;
     __device__ __forceinline__ void begin() {
@@ -43,8 +44,8 @@ struct ClockProbe {
         unsigned long long t1;
         const unsigned long long c1 = clock64();
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-        g_kernel_clock[kind][0] = c1 - c0;
-        g_kernel_clock[kind][1] = t1 - t0;
+        atomicAdd(&g_kernel_clock[kind][0], c1 - c0);
+        atomicAdd(&g_kernel_clock[kind][1], t1 - t0);
     }
 };
 

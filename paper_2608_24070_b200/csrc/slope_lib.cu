@@ -723,9 +723,18 @@ const char* slope_status_string(slope_status_t s) {
 slope_status_t slope_kernel_clock_mhz(int kind, void* stream, double* mhz_host) {
     if ((kind != 0 && kind != 1) || !mhz_host) return SLOPE_ERR_INVALID_ARG;
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return SLOPE_ERR_CUDA;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SLOPE_ERR_CUDA;
     unsigned long long v[2][2];
     if (cudaMemcpyFromSymbol(v, g_kernel_clock, sizeof(v)) != cudaSuccess) return SLOPE_ERR_CUDA;
-    *mhz_host = v[kind][1] ? static_cast<double>(v[kind][0]) / static_cast<double>(v[kind][1]) * 1e3 : 0.0;
+    // totals at the previous call, per device and kind
+    static std::mutex mu;
+    static unsigned long long seen[64][2][2] = {};
+    std::lock_guard<std::mutex> lock(mu);
+    const unsigned long long cycles = v[kind][0] - seen[dev][kind][0], ns = v[kind][1] - seen[dev][kind][1];
+    seen[dev][kind][0] = v[kind][0];
+    seen[dev][kind][1] = v[kind][1];
+    *mhz_host = ns ? static_cast<double>(cycles) / static_cast<double>(ns) * 1e3 : 0.0;
     return SLOPE_OK;
 }
 

@@ -754,13 +754,16 @@ def test_weight_gradient_with_adapter_gradients_in_one_call(B, oracle, d_in, d_o
 
 
 def test_kernel_clock_diagnostic_reports_a_plausible_sm_clock(B, oracle):
-    """slope_kernel_clock_mhz: the SM clock measured inside the last sparse / dense tile-kernel launch."""
+    """slope_kernel_clock_mhz: the SM clock measured inside the sparse / dense tile-kernel launches
+    since the previous call."""
     import torch
 
     W = si.gaussian_bf16((1024, 1024), 0.02, 801)
     layer = GpuLayer(W, fused_setup=True)
     X = dev(B, si.gaussian_bf16((2048, 1024), 1.0, 802))
     dY = dev(B, si.gaussian_bf16((2048, 1024), 1.0, 803))
+    B.slope_kernel_clock_mhz(0), B.slope_kernel_clock_mhz(1)          # forget earlier launches
+    assert B.slope_kernel_clock_mhz(0) == 0.0                          # nothing ran in between
     layer.fwd(X)                               # a CTA-pair sparse tile kernel
     layer.dw(dY, X)                            # the CTA-pair dense kernel
     layer.poll()
