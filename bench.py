@@ -336,8 +336,7 @@ def kernel_sources_sha256():
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the two tensor-core kernels, from a
 # one-pass ncu capture (--clock-control none) of this benchmark's own workload at full size: the 21
-# GEMM launches of one step of c4_llama7b_adapter at 16384 tokens (profiles/ has the summary and the
-# command).  `sources` is kernel_sources_sha256() of the build that was captured; a build with other
+# GEMM launches of one step of c4_llama7b_adapter at 16384 tokens.  `sources` is kernel_sources_sha256() of the build that was captured; a build with other
 # sources reports traffic = null (tests/test_bench_line.py fails until the capture is refreshed or
 # cleared).
 NCU_TRAFFIC = {
