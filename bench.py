@@ -377,10 +377,28 @@ def algorithmic_bytes(op, b, d_in, d_out, r):
     return 0.0
 
 
+LINE_LIMIT = 2000
+
+
 def compact_line(out):
-    """The one line the driver parses: short enough to survive a few-KB tail of stdout."""
+    """The one line the driver parses: short enough to survive a few-KB tail of stdout.  If a workload
+    with many layers makes it too long, the least important detail goes first (it stays in the side
+    file); a line that is still too long is an error."""
+    out = dict(out)
+    trims = (
+        lambda o: o.get("cpu_baseline") and o["cpu_baseline"].update(sample=o["cpu_baseline"]["sample"][:60] + "..."),
+        lambda o: o.pop("stage_ms", None),
+        lambda o: o.pop("roofline_other", None),
+    )
     line = json.dumps(out, separators=(",", ":"))
-    if len(line) > 2000:
+    for trim in trims:
+        if len(line) <= LINE_LIMIT:
+            break
+        if out.get("cpu_baseline"):
+            out["cpu_baseline"] = dict(out["cpu_baseline"])
+        trim(out)
+        line = json.dumps(out, separators=(",", ":"))
+    if len(line) > LINE_LIMIT:
         raise SystemExit(f"bench line grew to {len(line)} characters; move detail to the side file")
     return line
 

@@ -67,8 +67,14 @@ def test_slope_line_is_short_and_complete():
     assert "model" not in d["config"] and d["config"]["workload"] == "c4_llama7b_adapter"
 
 
-def test_an_overlong_line_is_refused():
-    out, _ = _worst_case_line()
+def test_an_overlong_line_sheds_detail_and_is_refused_only_when_that_is_not_enough():
+    out, line = _worst_case_line()
+    out["cpu_baseline"]["sample"] = "whole workload: " + "; ".join(["layer 768->3072 b=8192: fwd+dX 8192 token rows, dW 3072 rows"] * 6)
+    shorter = bench.compact_line(out)
+    assert len(shorter) <= LIMIT
+    d = json.loads(shorter)
+    assert d["value"] > 0 and d["roofline"]["frac"] > 0 and d["cpu_baseline"]["value"] > 0 and d["e2e"]["value"] > 0
+    assert d["cpu_baseline"]["sample"].endswith("...")
     out["junk"] = "x" * LIMIT
     with pytest.raises(SystemExit):
         bench.compact_line(out)
