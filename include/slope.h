@@ -209,7 +209,7 @@ slope_status_t slope_sparse_add(const void* A_vals, const void* B_vals, float be
  * transposed double-pruned copy from them: slot t of group h of row j of WTc_vals becomes
  * W_new[4h + q_t][j] if that element survived both pruning passes, else +0 (q_t from
  * WTc_meta; existence and position inside Wc_vals from mask1_bits).  Metadata and masks are
- * not modified.
+ * not modified.  d_out * d_in must stay below 2^35 (SLOPE_ERR_SHAPE otherwise).
  */
 slope_status_t slope_update_sparse_matrix(const void* Wc_vals, const void* mask1_bits, const void* WTc_meta,
                                           int d_out, int d_in, void* WTc_vals, void* stream);

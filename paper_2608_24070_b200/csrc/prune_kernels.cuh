@@ -364,73 +364,116 @@ __device__ __forceinline__ uint32_t expand_selector(uint32_t nib) {
     return sel;
 }
 
-__global__ void __launch_bounds__(256, 4) update_transposed_kernel(const uint2* __restrict__ Wc_new,
-                                                                   const uint8_t* __restrict__ mask1,
-                                                                   const uint4* __restrict__ metaT, int d_out, int d_in,
-                                                                   uint4* __restrict__ valsT) {
+// Blocks are persistent (three per SM) and walk over the tiles; the global loads of a block's
+// next tile are issued as soon as the registers of the current one have been expanded, so that
+// their latency is hidden behind the selection arithmetic instead of by other blocks.
+constexpr int kUpdateBlocksPerSm = 3;
+__global__ void __launch_bounds__(256, kUpdateBlocksPerSm)
+update_transposed_kernel(const uint2* __restrict__ Wc_new, const uint8_t* __restrict__ mask1,
+                         const uint4* __restrict__ metaT, int d_out, int d_in, uint4* __restrict__ valsT) {
     __shared__ __align__(16) uint8_t s_out[128 * 128];       // [column j][16 slots of 8 B], slot index XOR (j >> 3)
     __shared__ __align__(16) uint8_t s_meta[2048];
-    __shared__ uint32_t s_expand[16];
+    __shared__ __align__(8) uint2 s_expand[16];              // per 4-bit mask pattern: selectors of columns 0-1 and 2-3
 
-    const int cb = blockIdx.x, rb = blockIdx.y;
     const int tid = threadIdx.x;
     const int c8 = tid & 15;                                 // 8-column slot of the tile
     const int ig = tid >> 4;                                 // 8-row slot of the tile
-    const size_t row_u2 = static_cast<size_t>(d_in) >> 3;    // 8-byte units per compressed row = mask bytes per row
+    // 32-bit element offsets (the host refuses matrices of 2^35 elements or more): one integer add
+    // per load instead of a 64-bit address computation
+    const uint32_t row_u2 = static_cast<uint32_t>(d_in) >> 3;   // 8-byte units per compressed row = mask bytes per row
+    const uint32_t vrow_u4 = static_cast<uint32_t>(d_out) >> 4; // uint4 per row of valsT (d_out/2 bf16)
+    const int ncb = d_in >> 7, nrb = d_out >> 7;
+    const int num_tiles = ncb * nrb;
 
-    if (tid < 128) {
-        const size_t blk = static_cast<size_t>(cb) * (d_out >> 7) + rb;
-        reinterpret_cast<uint4*>(s_meta)[tid] = __ldg(metaT + blk * 128 + tid);
-    }
-    if (tid >= 128 && tid < 144) s_expand[tid - 128] = expand_selector(tid - 128);
+    if (tid < 16) s_expand[tid] = make_uint2(expand_selector(tid), expand_selector(tid) >> 16);
+
     uint2 cw[8];
     uint32_t mb[8];
+    uint4 m = make_uint4(0u, 0u, 0u, 0u);
+    auto fetch = [&](int cb, int rb) {
+        const uint32_t at = (static_cast<uint32_t>(rb) * 128u + ig * 8u) * row_u2 + cb * 16u + c8;
 #pragma unroll
-    for (int t = 0; t < 8; ++t) {
-        const size_t at = (static_cast<size_t>(rb) * 128 + ig * 8 + t) * row_u2 + cb * 16 + c8;
-        cw[t] = __ldg(Wc_new + at);
-        mb[t] = __ldg(mask1 + at);
-    }
-    __syncthreads();
-    uint32_t d[8][4];                                        // 8 rows x 4 column pairs of W^R
-#pragma unroll
-    for (int t = 0; t < 8; ++t) {
-        const uint32_t s0 = s_expand[mb[t] & 15u], s1 = s_expand[mb[t] >> 4];
-        d[t][0] = __byte_perm(cw[t].x, 0u, s0);
-        d[t][1] = __byte_perm(cw[t].x, 0u, s0 >> 16);
-        d[t][2] = __byte_perm(cw[t].y, 0u, s1);
-        d[t][3] = __byte_perm(cw[t].y, 0u, s1 >> 16);
-    }
-
-    const int meta_base = meta_byte_offset(c8 * 8, ig);      // + 16 per column inside the 8-column slot
-    const int slot = (ig ^ c8) * 8;
-#pragma unroll
-    for (int wi = 0; wi < 4; ++wi) {
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const int k = 2 * wi + half;
-            const uint32_t code = s_meta[meta_base + 16 * k];   // rows 0..3: low nibble, rows 4..7: high nibble
-            // column k of rows (0,1), (2,3), (4,5), (6,7) as four words, then one byte permute per
-            // row group picks rows q0 (low half) and q1 (high half): bytes 2q, 2q+1 of 8.
-            const uint32_t col = half ? 0x7632u : 0x5410u;
-            const uint32_t r01 = __byte_perm(d[0][wi], d[1][wi], col), r23 = __byte_perm(d[2][wi], d[3][wi], col);
-            const uint32_t r45 = __byte_perm(d[4][wi], d[5][wi], col), r67 = __byte_perm(d[6][wi], d[7][wi], col);
-            const uint32_t sel_a = 0x1010u + (code & 3u) * 0x22u + ((code >> 2) & 3u) * 0x2200u;
-            const uint32_t sel_b = 0x1010u + ((code >> 4) & 3u) * 0x22u + (code >> 6) * 0x2200u;
-            const uint32_t a = __byte_perm(r01, r23, sel_a), b = __byte_perm(r45, r67, sel_b);
-            *reinterpret_cast<uint2*>(s_out + (c8 * 8 + k) * 128 + slot) = make_uint2(a, b);
+        for (int t = 0; t < 8; ++t) {
+            cw[t] = __ldg(Wc_new + (at + t * row_u2));
+            mb[t] = __ldg(mask1 + (at + t * row_u2));
         }
-    }
-    __syncthreads();
+        if (tid < 128) m = __ldg(metaT + ((static_cast<uint32_t>(cb) * nrb + rb) * 128u + tid));
+    };
 
-    const size_t vrow_u4 = static_cast<size_t>(d_out) >> 4;        // uint4 per row of valsT (d_out/2 bf16)
+    // tile = blockIdx.x, blockIdx.x + gridDim.x, ...: (cb, rb) advance without a division per tile
+    const int step_rb = static_cast<int>(gridDim.x) / ncb, step_cb = static_cast<int>(gridDim.x) % ncb;
+    int tile = blockIdx.x;
+    int cb = tile % ncb, rb = tile / ncb;
+    if (tile < num_tiles) fetch(cb, rb);
+    __syncthreads();                                         // s_expand
+    for (; tile < num_tiles; tile += gridDim.x) {
+        int cb_next = cb + step_cb, rb_next = rb + step_rb;
+        if (cb_next >= ncb) { cb_next -= ncb; ++rb_next; }
+        if (tid < 128) {
+            // The metadata block goes to shared memory regrouped by reader: the eight code bytes a
+            // thread (ig, c8) needs (columns 8 c8 .. 8 c8 + 7 of row slot ig) lie 16 bytes apart in the
+            // block, all in one bank for a whole warp; stored as one 8-byte word per thread they are
+            // read back in a single conflict-free load.  16-byte unit `tid` of the block holds the
+            // codes of column k = tid % 8 of the slots c8 = 2 (tid / 16) + bit 1 of the byte index,
+            // ig = 4 (byte index / 4) + 2 ((tid / 8) % 2) + bit 0 of the byte index.
+            const uint32_t mw[4] = {m.x, m.y, m.z, m.w};
+            const int k = tid & 7, c8_0 = 2 * (tid >> 4), ig_0 = 2 * ((tid >> 3) & 1);
 #pragma unroll
-    for (int pass = 0; pass < 4; ++pass) {
-        const int jr = pass * 32 + (tid >> 3), seg = tid & 7;      // logical slots 2*seg, 2*seg+1
-        const int x = (jr >> 3) & 15;
-        const uint4 v = *reinterpret_cast<const uint4*>(s_out + jr * 128 + (((2 * seg) ^ x) >> 1) * 16);
-        const uint4 o = (x & 1) ? make_uint4(v.z, v.w, v.x, v.y) : v;
-        valsT[(static_cast<size_t>(cb) * 128 + jr) * vrow_u4 + rb * 8 + seg] = o;
+            for (int b = 0; b < 16; ++b) {
+                const int ig_b = ig_0 + 4 * (b >> 2) + (b & 1), c8_b = c8_0 + ((b >> 1) & 1);
+                s_meta[(ig_b * 16 + c8_b) * 8 + k] = static_cast<uint8_t>(mw[b >> 2] >> (8 * (b & 3)));
+            }
+        }
+        uint32_t d[8][4];                                    // 8 rows x 4 column pairs of W^R
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            const uint2 s0 = s_expand[mb[t] & 15u], s1 = s_expand[mb[t] >> 4];
+            d[t][0] = __byte_perm(cw[t].x, 0u, s0.x);
+            d[t][1] = __byte_perm(cw[t].x, 0u, s0.y);
+            d[t][2] = __byte_perm(cw[t].y, 0u, s1.x);
+            d[t][3] = __byte_perm(cw[t].y, 0u, s1.y);
+        }
+        if (tile + static_cast<int>(gridDim.x) < num_tiles) fetch(cb_next, rb_next);
+        __syncthreads();                                     // s_meta written; s_out no longer read
+
+        const uint2 codes = *reinterpret_cast<const uint2*>(s_meta + (ig * 16 + c8) * 8);   // byte k: column k of the slot
+        const int slot = (ig ^ c8) * 8;
+#pragma unroll
+        for (int wi = 0; wi < 4; ++wi) {
+            // A code byte holds four 2-bit row indices: q0, q1 (rows 0..3 -> slots 0, 1) and q2, q3
+            // (rows 4..7).  Index q selects bytes 2q, 2q + 1 of the eight bytes of a row quad, i.e.
+            // permute selector byte 0x10 + 0x22 q; the selector bytes of four columns are made at once.
+            const uint32_t c4 = wi < 2 ? codes.x : codes.y;
+            const uint32_t sq0 = (c4 & 0x03030303u) * 0x22u + 0x10101010u;
+            const uint32_t sq1 = ((c4 >> 2) & 0x03030303u) * 0x22u + 0x10101010u;
+            const uint32_t sq2 = ((c4 >> 4) & 0x03030303u) * 0x22u + 0x10101010u;
+            const uint32_t sq3 = ((c4 >> 6) & 0x03030303u) * 0x22u + 0x10101010u;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int k = 2 * wi + half;
+                // column k of rows (0,1), (2,3), (4,5), (6,7) as four words, then one byte permute per
+                // row group picks rows q0 (low half) and q1 (high half)
+                const uint32_t col = half ? 0x7632u : 0x5410u;
+                const uint32_t r01 = __byte_perm(d[0][wi], d[1][wi], col), r23 = __byte_perm(d[2][wi], d[3][wi], col);
+                const uint32_t r45 = __byte_perm(d[4][wi], d[5][wi], col), r67 = __byte_perm(d[6][wi], d[7][wi], col);
+                const uint32_t pick = static_cast<uint32_t>(k & 3) * 0x11u + 0x40u;      // byte k of the first, byte k of the second
+                const uint32_t sel_a = __byte_perm(sq0, sq1, pick), sel_b = __byte_perm(sq2, sq3, pick);
+                const uint32_t a = __byte_perm(r01, r23, sel_a), b = __byte_perm(r45, r67, sel_b);
+                *reinterpret_cast<uint2*>(s_out + (c8 * 8 + k) * 128 + slot) = make_uint2(a, b);
+            }
+        }
+        __syncthreads();
+
+#pragma unroll
+        for (int pass = 0; pass < 4; ++pass) {
+            const int jr = pass * 32 + (tid >> 3), seg = tid & 7;      // logical slots 2*seg, 2*seg+1
+            const int x = (jr >> 3) & 15;
+            const uint4 v = *reinterpret_cast<const uint4*>(s_out + jr * 128 + (((2 * seg) ^ x) >> 1) * 16);
+            const uint4 o = (x & 1) ? make_uint4(v.z, v.w, v.x, v.y) : v;
+            valsT[(static_cast<uint32_t>(cb) * 128u + jr) * vrow_u4 + rb * 8u + seg] = o;
+        }
+        cb = cb_next;
+        rb = rb_next;
     }
 }
 

@@ -1133,12 +1133,14 @@ slope_status_t slope_update_sparse_matrix(const void* Wc_vals, const void* mask1
                                           int d_out, int d_in, void* WTc_vals, void* stream) {
     if (!Wc_vals || !mask1_bits || !WTc_meta || !WTc_vals) return SLOPE_ERR_INVALID_ARG;
     if (!dims_ok(d_out, d_in)) return SLOPE_ERR_SHAPE;
+    // the kernel indexes its 8-byte and 16-byte units with 32 bits
+    if (static_cast<unsigned long long>(d_out) * static_cast<unsigned long long>(d_in) >= (1ull << 35)) return SLOPE_ERR_SHAPE;
     if (!aligned16(Wc_vals) || !aligned16(mask1_bits) || !aligned16(WTc_meta) || !aligned16(WTc_vals))
         return SLOPE_ERR_ALIGNMENT;
     DeviceInfo info;
     if (slope_status_t st = check_arch(info)) return st;
-    dim3 grid(d_in / 128, d_out / 128);
-    update_transposed_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+    const int tiles = (d_in / 128) * (d_out / 128), slots = info.sm_count * kUpdateBlocksPerSm;
+    update_transposed_kernel<<<tiles < slots ? tiles : slots, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint2*>(Wc_vals), static_cast<const uint8_t*>(mask1_bits),
         static_cast<const uint4*>(WTc_meta), d_out, d_in, static_cast<uint4*>(WTc_vals));
     return launch_result();

@@ -63,6 +63,7 @@ def test_host_side_argument_checks_need_no_gpu(lib):
     assert lib.slope_prune_nm(a, 128, 128, 4, 4, a, null, null) == 2                   # n must be below m
     assert lib.slope_sparse_add(a, a, 1.0, 1.0, 128, 100, a, null) == 2
     assert lib.slope_update_sparse_matrix(a, a, a, 128, 128, null, null) == 1
+    assert lib.slope_update_sparse_matrix(a, a, a, 262144, 131072, a, null) == 2       # 2^35 elements: beyond its 32-bit unit indices
     # the one-launch set-up and the weight gradient with the adapter gradients riding along
     assert lib.slope_prune_24_double(a, 128, 128, a, a, null, a, null, null, null) == 1          # a compressed copy missing
     assert lib.slope_prune_24_double(a, 128, 192, a, a, null, a, a, null, null) == 2             # d_in not a multiple of 128

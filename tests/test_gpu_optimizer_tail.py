@@ -48,7 +48,7 @@ def test_sparse_add(B, oracle, rows, cols):
     assert np.array_equal(B.bits_from_bf16(out), A)
 
 
-@pytest.mark.parametrize("d_out,d_in", [(512, 512), (384, 640), (1280, 128), (11008, 4096)])
+@pytest.mark.parametrize("d_out,d_in", [(512, 512), (384, 640), (1280, 128), (11008, 4096), (4096, 11008)])
 def test_update_sparse_matrix(B, oracle, d_out, d_in):
     import torch
 
