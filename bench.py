@@ -340,10 +340,10 @@ def kernel_sources_sha256():
 # sources reports traffic = null (tests/test_bench_line.py fails until the capture is refreshed or
 # cleared).
 NCU_TRAFFIC = {
-    "sources": "d5acd425bbfd044583584d97afe9e5d7629458da7028d2bf4560be18c8dc3a9a",
+    "sources": "29580e7bdfdde2b85c2b6fc0ef96f7ace4ecd81880759a788f213ca2aaaec8c4",
     "captured_tokens": 16384,
-    "sparse_bytes_per_launch": 493724818,     # mean over the 14 sparse GEMM launches of one step
-    "dense_bytes_per_launch": 1381888439,     # mean over the 7 weight-gradient launches of one step
+    "sparse_bytes_per_launch": 493399863,     # mean over the 14 sparse GEMM launches of one step
+    "dense_bytes_per_launch": 1370719854,     # mean over the 7 weight-gradient launches of one step
 }
 
 
