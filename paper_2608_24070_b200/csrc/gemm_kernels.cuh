@@ -535,9 +535,11 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
         // Warp w drains lane quadrant w%4; the two warps of a quadrant take alternate 32-token
-        // blocks.  A block is transposed through the warp's private staging buffer (lane =
-        // feature writes one bf16 per token row) and leaves as a TMA store of 32 tokens x 32
-        // features, so no warp waits for another and the stores cost no LSU issue slots.
+        // blocks.  A block (32 features x 32 tokens) is read from tensor memory as accumulator
+        // fragments, packed to bf16 pairs of adjacent tokens, and written transposed into the
+        // warp's private staging buffer by four stmatrix instructions ([token][32 features],
+        // 16-byte pieces XOR-swizzled as the store's tensor map expects); it leaves as a TMA store
+        // of 32 tokens x 32 features, so no warp waits for another.
         const int q = warp & 3;
         const int ew = warp - 2;
         const int half = ew >> 2;
@@ -557,18 +559,24 @@ sparse_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             const int width = token_tile_width(p.Ntok, n_blk * BLOCK_N, BLOCK_N);
 #pragma unroll 1
             for (int c0 = half * Cfg::kStoreRows; c0 < width; c0 += 2 * Cfg::kStoreRows) {
-                uint32_t v0[16], v1[16];
-                tmem_ld_16(t_row + c0, v0);
-                tmem_ld_16(t_row + c0 + 16, v1);
+                uint32_t v0[16], v1[16];                         // features 0..15 and 16..31 of the quadrant
+                tmem_ld_16x256b_x4(t_row + c0, v0);
+                tmem_ld_16x256b_x4(t_row + (16u << 16) + c0, v1);
                 // the staging buffer about to be overwritten must have been read by its TMA store
                 if (lane == 0) tma_store_wait_read<1>();
                 __syncwarp();
                 tmem_ld_wait();
-                uint16_t* sbuf = reinterpret_cast<uint16_t*>(my_buf + buf * Cfg::kStoreBytes) + lane;
+                // lane -> (matrix = feature group of 8, row = token within a group of 8): 64-byte token
+                // rows, 16-byte piece index XOR bits 7..8 of the address (the 64-byte swizzle)
+                const uint32_t row_addr = smem_u32(my_buf + buf * Cfg::kStoreBytes) + (lane & 7) * 64 +
+                                          (((lane >> 3) ^ ((lane >> 1) & 3)) << 4);
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    sbuf[c * Cfg::kStoreCols] = to_bf16(__uint_as_float(v0[c]));
-                    sbuf[(c + 16) * Cfg::kStoreCols] = to_bf16(__uint_as_float(v1[c]));
+                for (int j = 0; j < 4; ++j) {                    // tokens 8j .. 8j + 7
+                    stmatrix_x4_trans(row_addr + j * 512,
+                                      pack_bf16x2(__uint_as_float(v0[4 * j]), __uint_as_float(v0[4 * j + 1])),
+                                      pack_bf16x2(__uint_as_float(v0[4 * j + 2]), __uint_as_float(v0[4 * j + 3])),
+                                      pack_bf16x2(__uint_as_float(v1[4 * j]), __uint_as_float(v1[4 * j + 1])),
+                                      pack_bf16x2(__uint_as_float(v1[4 * j + 2]), __uint_as_float(v1[4 * j + 3])));
                 }
                 fence_proxy_async_smem();
                 __syncwarp();

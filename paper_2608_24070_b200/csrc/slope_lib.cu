@@ -132,17 +132,20 @@ static bool make_tmap_meta(CUtensorMap* tm, const void* base, size_t total_bytes
     });
 }
 
-// Plain (unswizzled) 2-D bf16 tensor map, used for TMA stores of output tiles.
-static bool make_tmap_plain(CUtensorMap* tm, const void* base, int rows, int cols, int box_rows, int box_cols) {
+// 2-D bf16 tensor map for TMA stores of output tiles: unswizzled, or (for a box 64 bytes wide) with
+// the 64-byte swizzle the transposing epilogues write their staging tiles in.
+static bool make_tmap_plain(CUtensorMap* tm, const void* base, int rows, int cols, int box_rows, int box_cols,
+                            bool swizzle64 = false) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
     const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(cols) * 2};
     const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
     const cuuint32_t estr[2] = {1, 1};
-    return tmap_memo(tm, TmapKey{base, rows, cols, box_rows, box_cols, 2}, [&](CUtensorMap* out) {
+    return tmap_memo(tm, TmapKey{base, rows, cols, box_rows, box_cols, swizzle64 ? 3 : 2}, [&](CUtensorMap* out) {
         return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_NONE,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
     });
 }
@@ -320,7 +323,7 @@ static slope_status_t launch_sparse_pair(const void* act, int ntok, const void* 
     if (!make_tmap(&tmA, vals, M, K / 2, kBlockM, 64)) return SLOPE_ERR_CUDA;
     if (!make_tmap(&tmB, act, ntok, K, Cfg::kHalfN, 64)) return SLOPE_ERR_CUDA;
     if (!make_tmap_meta(&tmE, meta, static_cast<size_t>(M) * K / 8)) return SLOPE_ERR_CUDA;
-    if (!make_tmap_plain(&tmO, out, ntok, M, Cfg::kStoreRows, Cfg::kStoreCols)) return SLOPE_ERR_CUDA;
+    if (!make_tmap_plain(&tmO, out, ntok, M, Cfg::kStoreRows, Cfg::kStoreCols, true)) return SLOPE_ERR_CUDA;
     if (r > 0) {
         const bool ok2 = a2_mn ? make_tmap(&tmA2, fac2, r, M, 64, 64) : make_tmap(&tmA2, fac2, M, r, kBlockM, 64);
         if (!ok2 || !make_tmap(&tmB2, act2, ntok, r, Cfg::kHalfN, 64)) return SLOPE_ERR_CUDA;
