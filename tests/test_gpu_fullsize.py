@@ -195,3 +195,12 @@ def test_pruning_a_matrix_of_more_than_2_31_elements(B, oracle, fused):
         assert np.array_equal(meta_rows[2 * t: 2 * t + 2].cpu().numpy().reshape(-1), meta_b.reshape(-1)), t
         assert np.array_equal(B.bits_from_bf16(valsT[:, t * (blk // 2): (t + 1) * (blk // 2)].contiguous()), valsT_b), t
         assert np.array_equal(metaT_blocks[:, 2 * t: 2 * t + 2].contiguous().cpu().numpy(), metaT_b), t
+    if fused:
+        # the optimizer tail's gather indexes its 8- and 16-byte units with 32 bits: same matrix, same slabs
+        # (unchanged forward values must give back the transposed copy)
+        del W
+        again = torch.zeros_like(valsT)
+        B.slope_update_sparse_matrix(vals, mask1, metaT, again)
+        assert B.slope_poll_status() == 0
+        for t in (0, 131, reps - 1):
+            assert np.array_equal(B.bits_from_bf16(again[:, t * (blk // 2): (t + 1) * (blk // 2)].contiguous()), valsT_b), t
