@@ -340,10 +340,10 @@ def kernel_sources_sha256():
 # sources reports traffic = null (tests/test_bench_line.py fails until the capture is refreshed or
 # cleared).
 NCU_TRAFFIC = {
-    "sources": "3577132d984e9be9659564230221706ea544d5a6f129c0d51699774a7fe018bc",
+    "sources": "e850cb677486eadb7dcfe7bb186a34c258c3387ea56bcab297d207fbd978d0fa",
     "captured_tokens": 16384,
-    "sparse_bytes_per_launch": 492941330,     # mean over the 14 sparse GEMM launches of one step
-    "dense_bytes_per_launch": 1384970277,     # mean over the 7 weight-gradient launches of one step
+    "sparse_bytes_per_launch": 493554889,     # mean over the 14 sparse GEMM launches of one step
+    "dense_bytes_per_launch": 1389503488,     # mean over the 7 weight-gradient launches of one step
 }
 
 

@@ -262,7 +262,7 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_saddr) {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_saddr) : "memory");
 }
 // 2-D tiled load into this CTA's shared memory whose completion bytes are counted on an
-// mbarrier that may live in the other CTA of the pair (`bar_cluster_saddr`).  No multicast.
+// mbarrier that may live in the other CTA of the pair (`bar_cluster_saddr`).  Each CTA issues its own copies.
 __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* tmap, uint32_t bar_cluster_saddr,
                                                  int x, int y) {
     asm volatile(
