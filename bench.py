@@ -318,6 +318,17 @@ def replica_throughput(world, flops_per_replica, ms_step):
     return world * flops_per_replica / (ms_step * 1e-3) / 1e12
 
 
+def replica_e2e(torch, dist, e2e_local, world, flops_per_replica, device):
+    """End-to-end record of `world` replicas from each rank's own: the slowest rank's time, all
+    replicas' work and bytes."""
+    ms = replica_max_ms(torch, dist, e2e_local["ms_per_step"], device)
+    out = dict(e2e_local)
+    out.update(ms_per_step=round(ms, 3), value=round(replica_throughput(world, flops_per_replica, ms), 2),
+               h2d_bytes_per_step=world * e2e_local["h2d_bytes_per_step"],
+               d2h_bytes_per_step=world * e2e_local["d2h_bytes_per_step"])
+    return out
+
+
 GEMM_SOURCES = ("gemm_kernels.cuh", "ptx.cuh", "slope_lib.cu")     # the GEMM kernels, their PTX wrappers, the kernel choice
 
 
@@ -677,6 +688,14 @@ def main():
         cb = cpu_baseline_sample(wl)
         side["cpu_baseline"] = cb
         attach_extras(out, dl, e2e, cb)
+    elif world > 1 and not args.no_extras:
+        # N replicas: every rank runs the host-buffer step on its own GPU and PCIe link; the job's
+        # end-to-end figure is all replicas' work over the slowest rank's time (no CPU baseline, no
+        # dense comparison at N > 1)
+        e2e = replica_e2e(torch, dist, e2e_run(torch, B, layers, de_flops, max(2, min(args.steps, 5))), world, de_flops, dev)
+        if rank == 0:
+            side["e2e"] = e2e
+            attach_extras(out, None, e2e, None)
     elif rank == 0:
         attach_extras(out, None, None, None)
     if rank == 0:

@@ -20,7 +20,10 @@ def _worker(rank, world, port, out):
     try:
         dist.barrier()
         ms = bench.replica_max_ms(torch, dist, 10.0 + 5.0 * rank, torch.device("cpu"))
-        out[rank] = (ms, bench.replica_throughput(world, 1e12, ms))
+        local = {"value": 0.0, "unit": "TFLOP/s", "ms_per_step": 40.0 + 10.0 * rank, "h2d_bytes_per_step": 1000,
+                 "d2h_bytes_per_step": 10}
+        e2e = bench.replica_e2e(torch, dist, local, world, 1e12, torch.device("cpu"))
+        out[rank] = (ms, bench.replica_throughput(world, 1e12, ms), e2e)
     finally:
         dist.destroy_process_group()
 
@@ -32,9 +35,12 @@ def test_two_replicas_report_slowest_time_and_summed_work():
         mp.spawn(_worker, args=(world, 29731, out), nprocs=world, join=True)
         res = dict(out)
     assert res[0] == res[1]
-    ms, tflops = res[0]
+    ms, tflops, e2e = res[0]
     assert ms == 15.0
     assert tflops == pytest.approx(2 * 1e12 / 15e-3 / 1e12)
+    # the end-to-end record of the job: slowest rank's time, both replicas' work and bytes
+    assert e2e["ms_per_step"] == 50.0 and e2e["h2d_bytes_per_step"] == 2000 and e2e["d2h_bytes_per_step"] == 20
+    assert e2e["value"] == pytest.approx(2 * 1e12 / 50e-3 / 1e12, rel=1e-3)
 
 
 def test_reference_arm_runs_on_rank0_only(monkeypatch, capsys):
